@@ -1,0 +1,10 @@
+"""Independent CPU oracle (float64) for the ToolSpec verify path and its drafters.
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, by the smoke check and by the benchmark's CPU-baseline
+leg.  The product package never imports it and shares no code with it.
+"""
+from .transformer import (OracleModel, KVCache, rmsnorm, rope, attention, swiglu,   # noqa: F401
+                          argmax_lowest, top2_gap)
+from .drafter import (SchemaFsm, Datastore, Drafter, suffix_match, validate_prefix,   # noqa: F401
+                      Q_O, Q_T, Q_P, Q_V, Q_DONE, SUFFIX_LENGTHS, DEFAULT_N_CAP)
+from .loop import prefill, vanilla_greedy, speculative_decode                        # noqa: F401
