@@ -1,0 +1,231 @@
+/*
+ * toolspec.h — C ABI of the B200-native verify path of ToolSpec (schema-aware, retrieval-augmented
+ * speculative decoding for tool calling).
+ *
+ * The calls follow the loop body of the paper's Algorithm 1:
+ *     draft (SuffixMatch, else SchemaAwareDraft)  ->  ts_draft      (host C++)
+ *     Verification (one forward over the packed chunk) + SelectLongestAcceptedPrefix
+ *                                                  ->  ts_verify     (sm_100a CUDA kernels)
+ *     y <- y (+) accepted span;  q <- delta(q, span) ->  ts_commit     (host C++)
+ * One candidate chain per step (causal mask inside the chunk) and greedy acceptance: the accepted
+ * length is the longest draft prefix equal to the per-position argmax of the target model, and one
+ * bonus token (the argmax after the last accepted draft) is always emitted, so an empty draft is
+ * exactly one vanilla decoding step.
+ *
+ * Conventions
+ *   - Every function returns a ts_status (0 = TS_OK, negative = error).  No exception crosses the
+ *     boundary.  ts_last_error() returns a thread-local description of the last failure.
+ *   - Handles (ts_model, ts_schema, ts_datastore, ts_session) are opaque, owned by the library and
+ *     released with the matching *_destroy.  A handle is not thread-safe.
+ *   - The library allocates NO device memory.  The caller allocates the four buffers whose sizes
+ *     ts_query_buffer_sizes() reports (three in device memory, one in pinned host memory) and
+ *     keeps them alive until ts_model_destroy().  All device work is enqueued on the cudaStream_t
+ *     given to ts_init_model (passed as void*).
+ *   - "host" / "device" below says where a pointer must point.  Token ids are int32.
+ *   - Without a usable CUDA device every call that needs one fails with TS_ERR_CUDA; there is no
+ *     CPU fallback for the verify path.
+ */
+#ifndef TOOLSPEC_H_
+#define TOOLSPEC_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TS_K_MAX 64          /* most rows (pending token + drafts) one sequence may verify per step */
+#define TS_PAGE_SIZE 16      /* tokens per KV page */
+
+typedef int32_t ts_status;
+enum {
+  TS_OK = 0,
+  TS_ERR_ARG = -1,            /* null pointer, size out of range, inconsistent configuration */
+  TS_ERR_STATE = -2,          /* call not valid in the handle's current state */
+  TS_ERR_OOM_PAGES = -3,      /* KV page pool exhausted */
+  TS_ERR_K_TOO_LARGE = -4,    /* chunk longer than k_max, or more rows than max_rows */
+  TS_ERR_TOKEN_RANGE = -5,    /* token id outside [0, vocab) */
+  TS_ERR_DEVICE_TIMEOUT = -6, /* a bounded device-side wait expired; the context stays usable */
+  TS_ERR_CUDA = -7,           /* CUDA runtime/driver error, or no device */
+  TS_ERR_UNIMPLEMENTED = -8
+};
+
+typedef struct ts_model ts_model;
+typedef struct ts_schema ts_schema;
+typedef struct ts_datastore ts_datastore;
+typedef struct ts_session ts_session;
+
+/* Decoder shape and capacity limits.  The layer recipe is pre-norm RMSNorm, rotary embedding in
+ * the rotate-half pairing, grouped-query attention, SwiGLU MLP, untied LM head, no biases. */
+typedef struct {
+  int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  float rope_theta, rms_eps;
+  int32_t max_pages;   /* KV pages in the pool (each TS_PAGE_SIZE tokens, all layers) */
+  int32_t max_batch;   /* most sequences per ts_verify call */
+  int32_t k_max;       /* most rows per sequence per call, <= TS_K_MAX */
+  int32_t max_rows;    /* most rows per call summed over the batch */
+  int32_t max_ctx;     /* most tokens per sequence (cache + chunk) */
+  int32_t act_split;   /* 1: GEMM activations are fed as a bf16 (hi, lo) pair; 0: hi only */
+} ts_model_config;
+
+typedef struct {
+  uint64_t weights_bytes;    /* device */
+  uint64_t kv_pool_bytes;    /* device */
+  uint64_t workspace_bytes;  /* device */
+  uint64_t host_io_bytes;    /* pinned host */
+} ts_buffer_sizes;
+
+typedef struct {
+  void *weights, *kv_pool, *workspace; /* device, 1024-byte aligned, sizes as queried */
+  void *host_io;                       /* pinned host */
+} ts_buffers;
+
+/* Sizes of the caller-allocated buffers for a configuration.  Host-only; needs no device. */
+ts_status ts_query_buffer_sizes(const ts_model_config *cfg, ts_buffer_sizes *out);
+
+/* ts_init_model — create the target model M of Algorithm 1 ("Require: target model M") over
+ * caller-owned buffers.  Zeroes the workspace, builds the TMA descriptors and the rotary table.
+ * Weights are loaded afterwards with ts_load_tensor.  `stream` is a cudaStream_t (0 = default).
+ * Errors: TS_ERR_ARG (bad shape: head_dim not 64/128, dims not multiples of 128, ...),
+ * TS_ERR_CUDA. */
+ts_status ts_init_model(const ts_model_config *cfg, const ts_buffers *bufs, void *stream,
+                        ts_model **out);
+
+enum { TS_W_EMBED = 0, TS_W_LM_HEAD = 1, TS_W_FINAL_GAIN = 2, TS_W_Q = 3, TS_W_K = 4, TS_W_V = 5,
+       TS_W_O = 6, TS_W_GATE = 7, TS_W_UP = 8, TS_W_DOWN = 9, TS_W_GAIN1 = 10, TS_W_GAIN2 = 11 };
+
+/* Upload one tensor.  Matrices are host bf16, row-major [out_features][in_features]; gains are
+ * host float32 [d_model].  `layer` is ignored for the three global tensors.  The library lays the
+ * matrix out for its kernels (Q,K,V rows concatenated; gate and up rows interleaved).  Synchronous.
+ * Errors: TS_ERR_ARG on a shape that does not match the configuration. */
+ts_status ts_load_tensor(ts_model *m, int32_t kind, int32_t layer, const void *host_data,
+                         int64_t rows, int64_t cols);
+
+ts_status ts_model_destroy(ts_model *m);
+
+/* ---- schema (Section 4.2: the parsed tool schema S; here supplied already parsed) -------------- */
+
+/* Fixed scaffolding strings of the tool-call format, as token ids:
+ *   <tool_call>  pfx name mid  key kvsep value  ( nxt key kvsep value )*  end
+ * e.g. pfx = {"name": "   mid = ", "parameters": {"   kvsep = ": "   nxt = ", "   end = "}}
+ * Each string has 1..8 ids; scaffolding ids must not occur inside names or keys. */
+typedef struct {
+  int32_t vocab, eos, tool_call;
+  int32_t pfx[8], mid[8], kvsep[8], nxt[8], end[8];
+  int32_t pfx_len, mid_len, kvsep_len, nxt_len, end_len;
+} ts_vocab_layout;
+
+ts_status ts_schema_create(const ts_vocab_layout *layout, ts_schema **out);
+/* key_tokens: all keys' ids concatenated; key_offsets[n_keys+1] delimits them (declared order). */
+ts_status ts_schema_add_tool(ts_schema *s, const int32_t *name, int32_t name_len,
+                             const int32_t *key_tokens, const int32_t *key_offsets, int32_t n_keys);
+ts_status ts_schema_destroy(ts_schema *s);
+
+/* ---- datastore (Section 4.3: historical invocations y_j; hidden states h_j are not stored) ---- */
+ts_status ts_datastore_create(int32_t n_tools, ts_datastore **out);
+/* Append one historical invocation (host ids, copied) and the tool it called (-1 = unknown).
+ * Not allowed while a session created over this datastore is between ts_draft calls of a step. */
+ts_status ts_datastore_add(ts_datastore *d, const int32_t *tokens, int32_t n, int32_t tool_id);
+ts_status ts_datastore_destroy(ts_datastore *d);
+
+/* ---- session: one sequence being decoded -------------------------------------------------------- */
+typedef struct {
+  int32_t n_cap;           /* longest retrieved continuation (paper: 32 for the first candidate) */
+  int32_t max_new_tokens;  /* generation budget */
+} ts_draft_config;
+
+/* `model` may be NULL for a host-only session (ts_draft / ts_commit_forced only). */
+ts_status ts_session_create(ts_model *model, const ts_schema *schema, const ts_datastore *store,
+                            const ts_draft_config *cfg, ts_session **out);
+/* Install the ranked candidate list I_k (indices into the datastore, best first) that Eq. 3's
+ * Top-K would produce.  n = 0 restores the default: every entry, in insertion order. */
+ts_status ts_session_set_ranks(ts_session *s, const int32_t *ranks, int32_t n);
+ts_status ts_session_destroy(ts_session *s);
+
+/* Feed the prompt: the KV of tokens[0..n-2] is computed with the verify kernels (chunks of k_max,
+ * LM head skipped) and tokens[n-1] becomes the pending token; every prompt id also passes through
+ * the FSM's delta.  With a host-only session only the FSM part happens. */
+ts_status ts_prefill(ts_model *m, ts_session *s, const int32_t *tokens, int32_t n);
+
+/* ts_draft — drafting part of Algorithm 1's loop body.  Retrieval first (Eq. 4: suffix lengths
+ * 7, 6, 5 of the generated output, candidates in rank order, first match position), and only if it
+ * yields nothing the schema FSM's deterministic filling (Eq. 2).  Writes at most max_draft ids to
+ * out_tokens (host, capacity max_draft), their count to *out_n (0 is not an error) and the source
+ * to *out_source: 0 none, 1 schema FSM, 2 retrieval.  Host only. */
+ts_status ts_draft(ts_session *s, int32_t max_draft, int32_t *out_tokens, int32_t *out_n,
+                   int32_t *out_source);
+
+typedef struct {
+  int32_t k;                   /* rows verified for this sequence = 1 + number of drafts */
+  int32_t accept_len;          /* l: drafts accepted, 0 <= l <= k-1 */
+  int32_t n_emitted;           /* l + 1 */
+  int32_t emitted[TS_K_MAX];   /* d_1..d_l followed by the bonus token t_l */
+  int32_t argmax[TS_K_MAX];    /* t_0..t_{k-1}: per-row argmax, lowest id on ties */
+  int32_t first_row;           /* index of this sequence's first row in the step's logits */
+} ts_verify_result;
+
+#define TS_FLAG_SKIP_LM_HEAD 1u  /* no logits, no acceptance: rows only extend the KV cache */
+
+/* ts_verify — Verification + SelectLongestAcceptedPrefix for B sequences in one batched forward.
+ * Sequence i's chunk is [pending_i, draft_tokens[draft_offsets[i] .. draft_offsets[i+1])], k_i rows
+ * at positions len_i .. len_i+k_i-1.  Allocates KV pages as needed, copies the step's inputs to the
+ * device, enqueues every kernel of the step, copies the result back and synchronises the stream.
+ * The sessions are not advanced: ts_commit does that.  out: host, B entries.
+ * Errors: TS_ERR_K_TOO_LARGE, TS_ERR_TOKEN_RANGE, TS_ERR_OOM_PAGES, TS_ERR_STATE (finished or
+ * unprefilled session), TS_ERR_DEVICE_TIMEOUT, TS_ERR_CUDA. */
+ts_status ts_verify(ts_model *m, ts_session *const *sessions, int32_t B,
+                    const int32_t *draft_tokens, const int32_t *draft_offsets, uint32_t flags,
+                    ts_verify_result *out);
+
+/* Enqueue again the device work of the last ts_verify call on its inputs, which are still resident
+ * in device memory; no host<->device copy, no synchronisation.  The step is idempotent because
+ * sessions advance only in ts_commit.  For timing the kernels alone. */
+ts_status ts_verify_replay(ts_model *m);
+
+/* ts_commit — y <- y (+) emitted, q <- delta(q, .) applied id by id (bonus token included), cache
+ * length and pending token advanced; stops at the first id that finishes the generation (call
+ * complete, EOS, or max_new_tokens) and drops the rest.  Host only. */
+ts_status ts_commit(ts_session *s, const ts_verify_result *r);
+/* Same, with an emitted span chosen by the caller (n >= 1): the cache keeps the pending token and
+ * the first n-1 ids, which must be the ids verified in the last step at those rows. */
+ts_status ts_commit_forced(ts_session *s, const int32_t *emitted, int32_t n);
+
+typedef struct {
+  int32_t cache_len, pending, n_output, finished;
+  int32_t fsm_kind;    /* 0 q_o, 1 q_t, 2 q_p, 3 q_v, 4 done */
+  int32_t fsm_tool;    /* chosen tool or -1 */
+  int32_t fsm_key;     /* index of the current key */
+  int32_t n_pages;
+} ts_session_info;
+ts_status ts_session_state(const ts_session *s, ts_session_info *out);
+/* Copy the generated output y (at most cap ids) to out (host); *n receives |y|. */
+ts_status ts_session_output(const ts_session *s, int32_t *out, int32_t cap, int32_t *n);
+
+/* ---- test / benchmark support ------------------------------------------------------------------- */
+/* Overwrite the session's cache for one layer with n_tokens rows of host bf16 K and V
+ * ([n_tokens][n_kv_heads][head_dim]).  After all layers were imported with the same n_tokens call
+ * ts_debug_set_cache(s, n_tokens, pending) to make them the session's context. */
+ts_status ts_debug_import_kv(ts_model *m, ts_session *s, int32_t layer, const void *k_bf16,
+                             const void *v_bf16, int32_t n_tokens);
+ts_status ts_debug_export_kv(ts_model *m, ts_session *s, int32_t layer, void *k_bf16, void *v_bf16,
+                             int32_t n_tokens);
+ts_status ts_debug_set_cache(ts_session *s, int32_t cache_len, int32_t pending);
+/* Copy rows [row0, row0+n_rows) of the last step's float32 logits [rows][vocab] to host memory. */
+ts_status ts_read_logits(ts_model *m, int32_t row0, int32_t n_rows, float *host_out);
+/* Copy the first `bytes` bytes of an internal activation buffer of the last step to host memory:
+ * 0 residual stream x (float32 [rows_alloc][d_model]); 1 normed activations (bf16
+ * [planes][rows_alloc][d_model]); 2 rotated queries (bf16 [rows_alloc][n_q_heads*head_dim]);
+ * 3 attention output (bf16 [planes][rows_alloc][n_q_heads*head_dim]); 4 SwiGLU output (bf16
+ * [planes][rows_alloc][d_ffn]).  rows_alloc = max_rows rounded up to 128; planes = 1 + act_split. */
+ts_status ts_debug_read_buffer(ts_model *m, int32_t which, void *host_out, uint64_t bytes);
+/* Counters: kernels launched since ts_init_model, bytes copied host->device and device->host by
+ * ts_verify since then. */
+ts_status ts_model_counters(const ts_model *m, int64_t *launches, int64_t *h2d_bytes,
+                            int64_t *d2h_bytes);
+
+const char *ts_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TOOLSPEC_H_ */

@@ -1,0 +1,9 @@
+"""B200-native verify path of ToolSpec (schema-aware, retrieval-augmented speculative decoding).
+
+The product is the C-ABI shared library built from csrc/ (see include/toolspec.h); this package holds
+its ctypes binding and the in-tree build step.  Importing the package does not load the library;
+`binding.lib()` does, and raises if it has not been built.
+"""
+from . import binding                     # noqa: F401
+from .binding import (Model, Schema, Datastore, Session, TsError, ts_prefill, ts_draft, ts_verify,   # noqa: F401
+                      ts_verify_replay, ts_commit, ts_commit_forced, TS_FLAG_SKIP_LM_HEAD, TS_K_MAX)

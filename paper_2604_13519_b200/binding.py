@@ -1,0 +1,361 @@
+"""Thin ctypes binding over the C ABI in include/toolspec.h.
+
+Argument marshalling only: every step of the verify path runs in the library's CUDA kernels and
+host C++.  PyTorch is used to allocate the caller-owned device / pinned buffers and to own the
+stream.  There is no fallback: if the shared library is missing the import of `lib()` raises.
+"""
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtoolspec.so")
+
+TS_K_MAX = 64
+TS_PAGE_SIZE = 16
+TS_FLAG_SKIP_LM_HEAD = 1
+
+STATUS = {0: "TS_OK", -1: "TS_ERR_ARG", -2: "TS_ERR_STATE", -3: "TS_ERR_OOM_PAGES",
+          -4: "TS_ERR_K_TOO_LARGE", -5: "TS_ERR_TOKEN_RANGE", -6: "TS_ERR_DEVICE_TIMEOUT",
+          -7: "TS_ERR_CUDA", -8: "TS_ERR_UNIMPLEMENTED"}
+
+(TS_W_EMBED, TS_W_LM_HEAD, TS_W_FINAL_GAIN, TS_W_Q, TS_W_K, TS_W_V, TS_W_O, TS_W_GATE, TS_W_UP,
+ TS_W_DOWN, TS_W_GAIN1, TS_W_GAIN2) = range(12)
+
+
+class TsError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__(f"{STATUS.get(code, code)}: {msg}")
+        self.code = code
+
+
+class ts_model_config(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim",
+                                         "d_ffn", "vocab")] + \
+               [("rope_theta", C.c_float), ("rms_eps", C.c_float)] + \
+               [(n, C.c_int32) for n in ("max_pages", "max_batch", "k_max", "max_rows", "max_ctx",
+                                         "act_split")]
+
+
+class ts_buffer_sizes(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in ("weights_bytes", "kv_pool_bytes", "workspace_bytes",
+                                          "host_io_bytes")]
+
+
+class ts_buffers(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("weights", "kv_pool", "workspace", "host_io")]
+
+
+class ts_vocab_layout(C.Structure):
+    _fields_ = [("vocab", C.c_int32), ("eos", C.c_int32), ("tool_call", C.c_int32)] + \
+               [(n, C.c_int32 * 8) for n in ("pfx", "mid", "kvsep", "nxt", "end")] + \
+               [(n, C.c_int32) for n in ("pfx_len", "mid_len", "kvsep_len", "nxt_len", "end_len")]
+
+
+class ts_draft_config(C.Structure):
+    _fields_ = [("n_cap", C.c_int32), ("max_new_tokens", C.c_int32)]
+
+
+class ts_verify_result(C.Structure):
+    _fields_ = [("k", C.c_int32), ("accept_len", C.c_int32), ("n_emitted", C.c_int32),
+                ("emitted", C.c_int32 * TS_K_MAX), ("argmax", C.c_int32 * TS_K_MAX),
+                ("first_row", C.c_int32)]
+
+
+class ts_session_info(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("cache_len", "pending", "n_output", "finished", "fsm_kind",
+                                         "fsm_tool", "fsm_key", "n_pages")]
+
+
+_P = C.c_void_p
+_I32P = C.POINTER(C.c_int32)
+_SIGNATURES = {
+    "ts_query_buffer_sizes": [C.POINTER(ts_model_config), C.POINTER(ts_buffer_sizes)],
+    "ts_init_model": [C.POINTER(ts_model_config), C.POINTER(ts_buffers), _P, C.POINTER(_P)],
+    "ts_load_tensor": [_P, C.c_int32, C.c_int32, _P, C.c_int64, C.c_int64],
+    "ts_model_destroy": [_P],
+    "ts_schema_create": [C.POINTER(ts_vocab_layout), C.POINTER(_P)],
+    "ts_schema_add_tool": [_P, _I32P, C.c_int32, _I32P, _I32P, C.c_int32],
+    "ts_schema_destroy": [_P],
+    "ts_datastore_create": [C.c_int32, C.POINTER(_P)],
+    "ts_datastore_add": [_P, _I32P, C.c_int32, C.c_int32],
+    "ts_datastore_destroy": [_P],
+    "ts_session_create": [_P, _P, _P, C.POINTER(ts_draft_config), C.POINTER(_P)],
+    "ts_session_set_ranks": [_P, _I32P, C.c_int32],
+    "ts_session_destroy": [_P],
+    "ts_prefill": [_P, _P, _I32P, C.c_int32],
+    "ts_draft": [_P, C.c_int32, _I32P, _I32P, _I32P],
+    "ts_verify": [_P, C.POINTER(_P), C.c_int32, _I32P, _I32P, C.c_uint32, C.POINTER(ts_verify_result)],
+    "ts_verify_replay": [_P],
+    "ts_commit": [_P, C.POINTER(ts_verify_result)],
+    "ts_commit_forced": [_P, _I32P, C.c_int32],
+    "ts_session_state": [_P, C.POINTER(ts_session_info)],
+    "ts_session_output": [_P, _I32P, C.c_int32, _I32P],
+    "ts_debug_import_kv": [_P, _P, C.c_int32, _P, _P, C.c_int32],
+    "ts_debug_export_kv": [_P, _P, C.c_int32, _P, _P, C.c_int32],
+    "ts_debug_set_cache": [_P, C.c_int32, C.c_int32],
+    "ts_read_logits": [_P, C.c_int32, C.c_int32, C.POINTER(C.c_float)],
+    "ts_debug_read_buffer": [_P, C.c_int32, _P, C.c_uint64],
+    "ts_model_counters": [_P, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64)],
+}
+EXPORTED = sorted(list(_SIGNATURES) + ["ts_last_error"])
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library.  Raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with "
+                               f"`python -m paper_2604_13519_b200.build` (needs nvcc)")
+        L = C.CDLL(LIB_PATH)
+        for name, args in _SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.argtypes = args
+            fn.restype = C.c_int32
+        L.ts_last_error.restype = C.c_char_p
+        L.ts_last_error.argtypes = []
+        _lib = L
+    return _lib
+
+
+def _check(code):
+    if code != 0:
+        raise TsError(code, lib().ts_last_error().decode())
+
+
+def _i32(seq: Sequence[int]):
+    arr = (C.c_int32 * max(1, len(seq)))(*seq)
+    return arr
+
+
+# ---- the same names as the C ABI, with Python-friendly arguments ----------------------------------
+class Schema:
+    def __init__(self, vocab_layout, tools):
+        """vocab_layout: object with size, eos, tool_call, pfx, mid, kvsep, nxt, end;
+        tools: iterable of objects with .name (ids) and .keys (list of id lists)."""
+        v = ts_vocab_layout()
+        v.vocab, v.eos, v.tool_call = vocab_layout.size, vocab_layout.eos, vocab_layout.tool_call
+        for f in ("pfx", "mid", "kvsep", "nxt", "end"):
+            ids = list(getattr(vocab_layout, f))
+            setattr(v, f + "_len", len(ids))
+            arr = getattr(v, f)
+            for i, t in enumerate(ids):
+                arr[i] = t
+        self.h = _P()
+        _check(lib().ts_schema_create(C.byref(v), C.byref(self.h)))
+        self.n_tools = 0
+        for t in tools:
+            flat, offs = [], [0]
+            for k in t.keys:
+                flat += list(k)
+                offs.append(len(flat))
+            _check(lib().ts_schema_add_tool(self.h, _i32(t.name), len(t.name), _i32(flat), _i32(offs),
+                                            len(t.keys)))
+            self.n_tools += 1
+
+    def __del__(self):
+        if getattr(self, "h", None) and _lib is not None:
+            _lib.ts_schema_destroy(self.h)
+            self.h = None
+
+
+class Datastore:
+    def __init__(self, n_tools: int):
+        self.h = _P()
+        _check(lib().ts_datastore_create(n_tools, C.byref(self.h)))
+        self.n = 0
+
+    def add(self, tokens: Sequence[int], tool_id: int):
+        _check(lib().ts_datastore_add(self.h, _i32(tokens), len(tokens), tool_id))
+        self.n += 1
+
+    def __del__(self):
+        if getattr(self, "h", None) and _lib is not None:
+            _lib.ts_datastore_destroy(self.h)
+            self.h = None
+
+
+class Model:
+    """ts_init_model + ts_load_tensor over buffers allocated with torch."""
+
+    def __init__(self, shape, max_pages: int, max_batch: int, k_max: int, max_rows: int, max_ctx: int,
+                 act_split: bool = True, device="cuda:0", stream=None):
+        import torch
+        self.torch = torch
+        self.shape = shape
+        c = ts_model_config()
+        for n in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab",
+                  "rope_theta", "rms_eps"):
+            setattr(c, n, getattr(shape, n))
+        c.max_pages, c.max_batch, c.k_max, c.max_rows, c.max_ctx = max_pages, max_batch, k_max, max_rows, max_ctx
+        c.act_split = 1 if act_split else 0
+        self.cfg = c
+        sizes = ts_buffer_sizes()
+        _check(lib().ts_query_buffer_sizes(C.byref(c), C.byref(sizes)))
+        self.sizes = sizes
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        mk = lambda n: torch.empty(int(n) + 1024, dtype=torch.uint8, device=self.device)
+        self._raw = [mk(sizes.weights_bytes), mk(sizes.kv_pool_bytes), mk(sizes.workspace_bytes)]
+        self._host = torch.empty(int(sizes.host_io_bytes), dtype=torch.uint8).pin_memory()
+        al = lambda t: (t.data_ptr() + 1023) // 1024 * 1024
+        self.kv_pool_ptr = al(self._raw[1])
+        b = ts_buffers(al(self._raw[0]), self.kv_pool_ptr, al(self._raw[2]), self._host.data_ptr())
+        self.stream = stream
+        sp = stream.cuda_stream if stream is not None else torch.cuda.current_stream().cuda_stream
+        self.stream_ptr = sp
+        self.h = _P()
+        _check(lib().ts_init_model(C.byref(c), C.byref(b), _P(sp), C.byref(self.h)))
+
+    def kv_pool_tensor(self):
+        """The caller-owned KV pool viewed as a bf16 tensor (e.g. to fill it with synthetic data)."""
+        torch = self.torch
+        off = self.kv_pool_ptr - self._raw[1].data_ptr()
+        n = int(self.sizes.kv_pool_bytes)
+        return self._raw[1][off:off + n].view(torch.bfloat16)
+
+    def load_tensor(self, kind: int, layer: int, t):
+        t = t.contiguous()
+        rows, cols = (t.shape if t.dim() == 2 else (1, t.shape[0]))
+        _check(lib().ts_load_tensor(self.h, kind, layer, _P(t.data_ptr()), rows, cols))
+
+    def load_weights(self, w: dict):
+        """w: name -> CPU tensor, names as produced by the synthetic generator."""
+        self.load_tensor(TS_W_EMBED, 0, w["embed"])
+        self.load_tensor(TS_W_LM_HEAD, 0, w["lm_head"])
+        self.load_tensor(TS_W_FINAL_GAIN, 0, w["gf"].float())
+        kinds = dict(wq=TS_W_Q, wk=TS_W_K, wv=TS_W_V, wo=TS_W_O, wg=TS_W_GATE, wu=TS_W_UP, wd=TS_W_DOWN,
+                     g1=TS_W_GAIN1, g2=TS_W_GAIN2)
+        for l in range(self.shape.n_layers):
+            for n, kind in kinds.items():
+                t = w[f"l{l}.{n}"]
+                self.load_tensor(kind, l, t.float() if n[0] == "g" else t)
+
+    def read_logits(self, row0: int, n_rows: int):
+        import numpy as np
+        out = np.empty((n_rows, self.cfg.vocab), dtype=np.float32)
+        _check(lib().ts_read_logits(self.h, row0, n_rows, out.ctypes.data_as(C.POINTER(C.c_float))))
+        return out
+
+    def read_buffer(self, which: int):
+        """Internal activation buffer `which` of the last step as a CPU tensor (test support)."""
+        torch = self.torch
+        s, R = self.shape, (self.cfg.max_rows + 127) // 128 * 128
+        P = 1 + self.cfg.act_split
+        Nq = s.n_q_heads * s.head_dim
+        shape, dt = {0: ((R, s.d_model), torch.float32), 1: ((P, R, s.d_model), torch.bfloat16),
+                     2: ((R, Nq), torch.bfloat16), 3: ((P, R, Nq), torch.bfloat16),
+                     4: ((P, R, s.d_ffn), torch.bfloat16)}[which]
+        out = torch.empty(shape, dtype=dt)
+        _check(lib().ts_debug_read_buffer(self.h, which, _P(out.data_ptr()), out.numel() * out.element_size()))
+        return out
+
+    def counters(self):
+        a, b, c = C.c_int64(), C.c_int64(), C.c_int64()
+        _check(lib().ts_model_counters(self.h, C.byref(a), C.byref(b), C.byref(c)))
+        return a.value, b.value, c.value
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib().ts_model_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Session:
+    def __init__(self, model: Optional[Model], schema: Optional[Schema], store: Optional[Datastore],
+                 n_cap: int = 32, max_new_tokens: int = 1 << 30):
+        self.model, self.schema, self.store = model, schema, store      # keep handles alive
+        cfg = ts_draft_config(n_cap, max_new_tokens)
+        self.h = _P()
+        _check(lib().ts_session_create(model.h if model else None, schema.h if schema else None,
+                                       store.h if store else None, C.byref(cfg), C.byref(self.h)))
+
+    def set_ranks(self, ranks: Sequence[int]):
+        _check(lib().ts_session_set_ranks(self.h, _i32(ranks), len(ranks)))
+
+    def state(self) -> ts_session_info:
+        info = ts_session_info()
+        _check(lib().ts_session_state(self.h, C.byref(info)))
+        return info
+
+    def output(self) -> List[int]:
+        n = C.c_int32()
+        _check(lib().ts_session_output(self.h, None, 0, C.byref(n)))
+        buf = (C.c_int32 * max(1, n.value))()
+        _check(lib().ts_session_output(self.h, buf, n.value, C.byref(n)))
+        return list(buf[:n.value])
+
+    def set_cache(self, cache_len: int, pending: int):
+        _check(lib().ts_debug_set_cache(self.h, cache_len, pending))
+
+    def import_kv(self, layer: int, k, v):
+        """k, v: CPU bf16 tensors [n_tokens][n_kv_heads][head_dim]."""
+        k, v = k.contiguous(), v.contiguous()
+        _check(lib().ts_debug_import_kv(self.model.h, self.h, layer, _P(k.data_ptr()), _P(v.data_ptr()),
+                                        k.shape[0]))
+
+    def export_kv(self, layer: int, n_tokens: int):
+        torch = self.model.torch
+        s = self.model.shape
+        k = torch.empty(n_tokens, s.n_kv_heads, s.head_dim, dtype=torch.bfloat16)
+        v = torch.empty_like(k)
+        _check(lib().ts_debug_export_kv(self.model.h, self.h, layer, _P(k.data_ptr()), _P(v.data_ptr()),
+                                        n_tokens))
+        return k, v
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib().ts_session_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def ts_prefill(model: Optional[Model], session: Session, tokens: Sequence[int]):
+    _check(lib().ts_prefill(model.h if model else None, session.h, _i32(tokens), len(tokens)))
+
+
+def ts_draft(session: Session, max_draft: int):
+    """Returns (draft ids, source) with source 0 none, 1 schema FSM, 2 retrieval."""
+    buf = (C.c_int32 * max(1, max_draft))()
+    n, src = C.c_int32(), C.c_int32()
+    _check(lib().ts_draft(session.h, max_draft, buf, C.byref(n), C.byref(src)))
+    return list(buf[:n.value]), src.value
+
+
+def ts_verify(model: Model, sessions: Sequence[Session], drafts: Sequence[Sequence[int]], flags: int = 0):
+    """Returns a list of ts_verify_result, one per session."""
+    B = len(sessions)
+    hs = (_P * B)(*[s.h for s in sessions])
+    flat, offs = [], [0]
+    for d in drafts:
+        flat += list(d)
+        offs.append(len(flat))
+    out = (ts_verify_result * B)()
+    _check(lib().ts_verify(model.h, hs, B, _i32(flat), _i32(offs), flags, out))
+    return list(out)
+
+
+def ts_verify_replay(model: Model):
+    _check(lib().ts_verify_replay(model.h))
+
+
+def ts_commit(session: Session, result: ts_verify_result):
+    _check(lib().ts_commit(session.h, C.byref(result)))
+
+
+def ts_commit_forced(session: Session, emitted: Sequence[int]):
+    _check(lib().ts_commit_forced(session.h, _i32(emitted), len(emitted)))

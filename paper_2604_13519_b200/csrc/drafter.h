@@ -1,0 +1,75 @@
+// Host-side drafting structures: tool schema with a name trie, the schema finite-state machine
+// (Section 4.2 of the paper), and the datastore of historical invocations with a 5-gram index for
+// suffix matching (Section 4.3, Eq. 4).
+#pragma once
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "toolspec.h"
+
+namespace ts {
+
+struct ToolDef {
+  std::vector<int32_t> name;
+  std::vector<std::vector<int32_t>> keys;
+};
+
+struct TrieNode {
+  std::vector<std::pair<int32_t, int32_t>> next;  // (token, child), kept sorted by token
+  int32_t tool_exact = -1;                        // tool whose full name ends here
+  int32_t min_tool = -1;                          // lowest tool id in this subtree
+  std::vector<int32_t> tools;                     // every tool id in this subtree (ascending)
+};
+
+}  // namespace ts
+
+struct ts_schema {
+  ts_vocab_layout v{};
+  std::vector<ts::ToolDef> tools;
+  std::vector<ts::TrieNode> trie;  // node 0 = root
+  int32_t child(int32_t node, int32_t token) const;
+  int32_t walk(const std::vector<int32_t> &prefix) const;  // -1 if no tool has this prefix
+};
+
+struct ts_datastore {
+  std::vector<int32_t> tokens;       // all entries concatenated
+  std::vector<int64_t> offset{0};    // entry e = tokens[offset[e] .. offset[e+1])
+  std::vector<int32_t> tool_of;
+  std::vector<int64_t> freq;         // per tool
+  // index over every position m with a 5-gram ending at m and a non-empty continuation
+  struct Posting { uint64_t key; int32_t entry; int32_t m; };
+  mutable std::vector<Posting> index;
+  mutable int64_t indexed_entries = 0;
+  void ensure_index() const;
+  int32_t n_entries() const { return (int32_t)tool_of.size(); }
+  const int32_t *entry(int32_t e, int32_t *len) const {
+    *len = (int32_t)(offset[e + 1] - offset[e]);
+    return tokens.data() + offset[e];
+  }
+};
+
+namespace ts {
+
+enum FsmKind : int32_t { Q_O = 0, Q_T = 1, Q_P = 2, Q_V = 3, Q_DONE = 4 };
+enum FsmStage : int32_t { ST_NONE = 0, ST_PFX, ST_NAME, ST_MID, ST_KEY, ST_SEP, ST_VAL, ST_NXT, ST_END };
+
+// State of the schema FSM F = (Q, Sigma_schema, delta, q0), q0 = q_o.
+struct Fsm {
+  const ts_schema *s = nullptr;
+  int32_t kind = Q_O, stage = ST_NONE, i = 0, tool = -1, key = 0, node = 0;
+  int32_t name_len = 0;
+  void reset() { kind = Q_O; stage = ST_NONE; i = 0; tool = -1; key = 0; node = 0; name_len = 0; }
+  void step(int32_t token);                         // delta
+  // deterministic schema filling from the current state; guess = tool to assume while the name is open
+  void draft(int32_t guess, std::vector<int32_t> *out) const;
+ private:
+  void to_o(int32_t token);
+  int expect(const int32_t *seq, int32_t len, int32_t token);  // -1 mismatch, 0 more, 1 complete
+};
+
+// Eq. 4 over the store: returns the continuation (possibly empty).
+void suffix_match(const std::vector<int32_t> &y, const ts_datastore &d, const std::vector<int32_t> *ranks,
+                  int32_t n, std::vector<int32_t> *out);
+
+}  // namespace ts

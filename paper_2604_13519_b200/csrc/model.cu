@@ -1,0 +1,880 @@
+// Host side of the library: handles, buffer layout, weight upload, the verify step's kernel sequence,
+// sessions (page lists, drafter state) and every extern "C" entry point declared in toolspec.h.
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "drafter.h"
+#include "kernels.h"
+#include "toolspec.h"
+
+namespace {
+
+thread_local std::string g_err;
+
+ts_status fail(ts_status code, const char *fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  g_err = buf;
+  return code;
+}
+
+#define CU_TRY(expr)                                                                          \
+  do {                                                                                        \
+    cudaError_t e__ = (expr);                                                                 \
+    if (e__ != cudaSuccess)                                                                   \
+      return fail(TS_ERR_CUDA, "%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e__), __FILE__, __LINE__); \
+  } while (0)
+
+inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+constexpr int kMaxSplits = 12;
+constexpr int kMaxAttnSplits = 32;
+constexpr int kMcOptions[4] = {16, 32, 64, 128};
+
+struct Layout {
+  // weights buffer (byte offsets)
+  uint64_t embed, lm_head, gf;
+  std::vector<uint64_t> wqkv, wo, wgu, wd, g1, g2;
+  uint64_t weights_bytes;
+  // kv pool
+  uint64_t kv_layer_stride, kv_v_offset, kv_bytes;   // in bf16 elements / bytes
+  // workspace (byte offsets)
+  uint64_t x, h, part, q, attn_o, attn_ml, attn, act, logits, amax, rope, d_in, d_out, workspace_bytes;
+  // step io (int32 offsets inside d_in / h_in)
+  int o_tokens, o_pos, o_rowseq, o_cu, o_len, o_tile_seq, o_tile_row0, o_btab, in_ints;
+  // step out (int32 offsets)
+  int o_argmax, o_accept, o_emitted, o_newlen, o_newpend, o_err, out_ints;
+  int rows_alloc, pages_per_seq, max_tiles, Nqkv, n_vocab_tiles;
+  uint64_t host_io_bytes;
+};
+
+bool config_ok(const ts_model_config &c, const char **why) {
+#define REQ(cond, msg) if (!(cond)) { *why = msg; return false; }
+  REQ(c.n_layers > 0 && c.d_model > 0 && c.vocab > 0 && c.d_ffn > 0, "non-positive dimension");
+  REQ(c.head_dim == 64 || c.head_dim == 128, "head_dim must be 64 or 128");
+  REQ(c.n_q_heads > 0 && c.n_kv_heads > 0 && c.n_q_heads % c.n_kv_heads == 0, "q heads not a multiple of kv heads");
+  REQ(c.d_model % 128 == 0 && c.d_ffn % 64 == 0 && c.vocab % 128 == 0, "d_model, vocab must be multiples of 128, d_ffn of 64");
+  REQ(((c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim) % 128 == 0, "QKV width must be a multiple of 128");
+  REQ((c.n_q_heads * c.head_dim) % 64 == 0, "attention width must be a multiple of 64");
+  REQ(c.k_max >= 1 && c.k_max <= TS_K_MAX, "k_max out of range");
+  REQ(c.max_batch >= 1 && c.max_rows >= c.k_max && c.max_rows <= c.max_batch * c.k_max, "max_rows out of range");
+  REQ(c.max_ctx >= c.k_max && c.max_pages >= 1, "max_ctx / max_pages out of range");
+  REQ(c.act_split == 0 || c.act_split == 1, "act_split must be 0 or 1");
+  REQ(c.rope_theta > 1.f && c.rms_eps > 0.f, "rope_theta / rms_eps out of range");
+#undef REQ
+  return true;
+}
+
+void make_layout(const ts_model_config &c, Layout *L) {
+  const uint64_t d = c.d_model, F = c.d_ffn, V = c.vocab, hd = c.head_dim;
+  L->Nqkv = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+  const uint64_t Nq = (uint64_t)c.n_q_heads * hd;
+  uint64_t o = 0;
+  auto take = [&](uint64_t bytes) { uint64_t r = o; o = align_up(o + bytes, 1024); return r; };
+  L->embed = take(V * d * 2);
+  L->lm_head = take(V * d * 2);
+  L->wqkv.resize(c.n_layers); L->wo.resize(c.n_layers); L->wgu.resize(c.n_layers); L->wd.resize(c.n_layers);
+  L->g1.resize(c.n_layers); L->g2.resize(c.n_layers);
+  for (int l = 0; l < c.n_layers; ++l) {
+    L->wqkv[l] = take((uint64_t)L->Nqkv * d * 2);
+    L->wo[l] = take(d * Nq * 2);
+    L->wgu[l] = take(2 * F * d * 2);
+    L->wd[l] = take(d * F * 2);
+  }
+  for (int l = 0; l < c.n_layers; ++l) { L->g1[l] = take(d * 4); L->g2[l] = take(d * 4); }
+  L->gf = take(d * 4);
+  L->weights_bytes = o;
+
+  const uint64_t page_elems = (uint64_t)c.n_kv_heads * TS_PAGE_SIZE * hd;
+  L->kv_v_offset = (uint64_t)c.max_pages * page_elems;
+  L->kv_layer_stride = 2 * L->kv_v_offset;
+  L->kv_bytes = (uint64_t)c.n_layers * L->kv_layer_stride * 2;
+
+  L->rows_alloc = (int)align_up(c.max_rows, 128);
+  L->pages_per_seq = (c.max_ctx + TS_PAGE_SIZE - 1) / TS_PAGE_SIZE;
+  const int G = c.n_q_heads / c.n_kv_heads;
+  L->max_tiles = c.max_batch * ((c.k_max * G + 63) / 64);
+  L->n_vocab_tiles = c.vocab / 128;
+  const uint64_t R = L->rows_alloc, planes = c.act_split ? 2 : 1;
+  o = 0;
+  L->x = take(R * d * 4);
+  L->h = take(planes * R * d * 2);
+  const uint64_t part_cols = std::max<uint64_t>(L->Nqkv, d);
+  L->part = take((uint64_t)kMaxSplits * R * part_cols * 4);
+  L->q = take(R * Nq * 2);
+  L->attn_o = take(R * c.n_q_heads * kMaxAttnSplits * hd * 4);
+  L->attn_ml = take(R * c.n_q_heads * kMaxAttnSplits * 8);
+  L->attn = take(planes * R * Nq * 2);
+  L->act = take(planes * R * F * 2);
+  L->logits = take(R * V * 4);
+  L->amax = take(R * (uint64_t)L->n_vocab_tiles * 4 * 8);
+  L->rope = take((uint64_t)c.max_ctx * (hd / 2) * 8);
+  int io = 0;
+  auto itake = [&](int n) { int r = io; io += (n + 3) / 4 * 4; return r; };
+  L->o_tokens = itake(c.max_rows); L->o_pos = itake(c.max_rows); L->o_rowseq = itake(c.max_rows);
+  L->o_cu = itake(c.max_batch + 1); L->o_len = itake(c.max_batch);
+  L->o_tile_seq = itake(L->max_tiles); L->o_tile_row0 = itake(L->max_tiles);
+  L->o_btab = itake(c.max_batch * L->pages_per_seq);
+  L->in_ints = io;
+  io = 0;
+  L->o_argmax = itake(c.max_rows); L->o_accept = itake(c.max_batch); L->o_emitted = itake(c.max_batch * c.k_max);
+  L->o_newlen = itake(c.max_batch); L->o_newpend = itake(c.max_batch); L->o_err = itake(4);
+  L->out_ints = io;
+  L->d_in = take((uint64_t)L->in_ints * 4);
+  L->d_out = take((uint64_t)L->out_ints * 4);
+  L->workspace_bytes = o;
+  L->host_io_bytes = align_up((uint64_t)(L->in_ints + L->out_ints) * 4, 4096);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+}  // namespace
+
+struct ts_model {
+  ts_model_config c{};
+  ts_buffers b{};
+  Layout L{};
+  cudaStream_t st = nullptr;
+  int planes = 1, n_sms = 148;
+  size_t gemm_smem_budget = 100 * 1024;
+  std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_d;
+  CUtensorMap tm_lm{}, tm_h[4]{}, tm_attn[4]{}, tm_act[4]{};
+  std::vector<int32_t> free_pages;
+  // last staged step
+  int last_B = 0, last_M = 0, last_tiles = 0;
+  uint32_t last_flags = 0;
+  bool have_step = false;
+  int64_t launches = 0, h2d = 0, d2h = 0;
+  bool use_pdl = true;
+
+  uint8_t *W(uint64_t off) const { return (uint8_t *)b.weights + off; }
+  uint8_t *WS(uint64_t off) const { return (uint8_t *)b.workspace + off; }
+  int32_t *h_in() const { return (int32_t *)b.host_io; }
+  int32_t *h_out() const { return (int32_t *)b.host_io + L.in_ints; }
+  int32_t *d_in() const { return (int32_t *)WS(L.d_in); }
+  int32_t *d_out() const { return (int32_t *)WS(L.d_out); }
+  __nv_bfloat16 *k_pages(int l) const { return (__nv_bfloat16 *)b.kv_pool + (uint64_t)l * L.kv_layer_stride; }
+  __nv_bfloat16 *v_pages(int l) const { return k_pages(l) + L.kv_v_offset; }
+};
+
+struct ts_session {
+  ts_model *m = nullptr;
+  const ts_schema *schema = nullptr;
+  const ts_datastore *store = nullptr;
+  ts_draft_config cfg{};
+  ts::Fsm fsm;
+  std::vector<int32_t> y, ranks, pages, last_chunk;
+  bool have_ranks = false;
+  int32_t cache_len = -1, pending = -1;
+  bool finished = false;
+};
+
+namespace {
+
+ts_status make_map(EncodeTiledFn enc, CUtensorMap *out, void *base, int rank, const uint64_t *dims,
+                   const uint32_t *box) {
+  cuuint64_t gdim[3], gstride[2];
+  cuuint32_t bx[3], es[3] = {1, 1, 1};
+  for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bx[i] = box[i]; }
+  gstride[0] = dims[0] * 2;
+  if (rank == 3) gstride[1] = dims[0] * dims[1] * 2;
+  CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, base, gdim, gstride, bx, es,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(TS_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+  return TS_OK;
+}
+
+ts_status weight_map(EncodeTiledFn enc, CUtensorMap *out, void *base, uint64_t N, uint64_t K) {
+  const uint64_t dims[2] = {K, N};
+  const uint32_t box[2] = {64, 128};
+  return make_map(enc, out, base, 2, dims, box);
+}
+
+ts_status act_maps(EncodeTiledFn enc, CUtensorMap *out4, void *base, uint64_t K, uint64_t rows, int planes) {
+  for (int i = 0; i < 4; ++i) {
+    const uint64_t dims[3] = {K, rows, (uint64_t)planes};
+    const uint32_t box[3] = {64, (uint32_t)kMcOptions[i], (uint32_t)planes};
+    ts_status s = make_map(enc, &out4[i], base, 3, dims, box);
+    if (s) return s;
+  }
+  return TS_OK;
+}
+
+int pick_mc_index(int M) {
+  for (int i = 0; i < 3; ++i)
+    if (M <= kMcOptions[i]) return i;
+  return 3;
+}
+
+// split-K factor: fill about two CTAs per SM, at least 4 k-blocks per slice
+int pick_splits(const ts_model *m, int n_tiles, int m_chunks, int n_kblocks, bool allow) {
+  if (!allow) return 1;
+  const int ctas = n_tiles * m_chunks;
+  int s = (2 * m->n_sms) / std::max(1, ctas);
+  s = std::max(1, std::min(s, std::min(kMaxSplits, n_kblocks / 4)));
+  return std::max(1, s);
+}
+
+struct GemmPlan { int splits, kb_per_split; };
+
+ts_status run_gemm(ts_model *m, int epi, const CUtensorMap &tw, const CUtensorMap *ta4, int N, int K, int M,
+                   float *out, __nv_bfloat16 *act_out, float2 *amax, GemmPlan *plan) {
+  const int mi = pick_mc_index(M);
+  ts::GemmArgs g{};
+  g.N = N; g.K = K; g.M = M; g.Mc = kMcOptions[mi]; g.planes = m->planes;
+  g.n_kblocks = K / 64;
+  const int m_chunks = (M + g.Mc - 1) / g.Mc;
+  int splits = pick_splits(m, N / 128, m_chunks, g.n_kblocks, epi == ts::EPI_PARTIAL);
+  g.kb_per_split = (g.n_kblocks + splits - 1) / splits;
+  splits = (g.n_kblocks + g.kb_per_split - 1) / g.kb_per_split;
+  g.out = out; g.out_rows = m->L.rows_alloc;
+  g.act_out = act_out; g.act_rows = m->L.rows_alloc; g.out_planes = m->planes;
+  g.amax = amax;
+  g.err = m->d_out() + m->L.o_err;
+  if (plan) { plan->splits = splits; plan->kb_per_split = g.kb_per_split; }
+  CU_TRY(ts::launch_gemm(epi, tw, ta4[mi], g, splits, m->gemm_smem_budget, m->st, m->use_pdl));
+  ++m->launches;
+  return TS_OK;
+}
+
+ts_status run_step(ts_model *m) {
+  const ts_model_config &c = m->c;
+  const Layout &L = m->L;
+  const int M = m->last_M, B = m->last_B;
+  const int d = c.d_model, F = c.d_ffn, Nq = c.n_q_heads * c.head_dim;
+  ts::StepIn in{};
+  int32_t *di = m->d_in();
+  in.tokens = di + L.o_tokens; in.pos = di + L.o_pos; in.row_seq = di + L.o_rowseq; in.cu_rows = di + L.o_cu;
+  in.seq_len = di + L.o_len; in.block_tab = di + L.o_btab; in.pages_per_seq = L.pages_per_seq;
+  in.B = B; in.M = M;
+  float *x = (float *)m->WS(L.x);
+  __nv_bfloat16 *h = (__nv_bfloat16 *)m->WS(L.h);
+  float *part = (float *)m->WS(L.part);
+  __nv_bfloat16 *q = (__nv_bfloat16 *)m->WS(L.q);
+  __nv_bfloat16 *attn = (__nv_bfloat16 *)m->WS(L.attn);
+  __nv_bfloat16 *act = (__nv_bfloat16 *)m->WS(L.act);
+  const float2 *rope = (const float2 *)m->WS(L.rope);
+  const int R = L.rows_alloc;
+
+  ts::AttnArgs aa{};
+  aa.in = in; aa.q = q; aa.Hq = c.n_q_heads; aa.Hkv = c.n_kv_heads; aa.hd = c.head_dim;
+  aa.n_row_tiles_total = m->last_tiles;
+  aa.tile_seq = di + L.o_tile_seq; aa.tile_row0 = di + L.o_tile_row0;
+  aa.part_o = (float *)m->WS(L.attn_o); aa.part_ml = (float2 *)m->WS(L.attn_ml);
+  aa.out = attn; aa.out_rows = R; aa.planes = m->planes;
+  {
+    // enough CTAs for about two per SM, each split at least one 64-position block
+    int max_total = 0;
+    const int32_t *hi = m->h_in();
+    for (int i = 0; i < B; ++i)
+      max_total = std::max(max_total, hi[L.o_len + i] + (hi[L.o_cu + i + 1] - hi[L.o_cu + i]));
+    const int nblk = (max_total + 63) / 64;
+    int s = (2 * m->n_sms + c.n_kv_heads * m->last_tiles - 1) / (c.n_kv_heads * m->last_tiles);
+    aa.n_splits = std::max(1, std::min(std::min(s, kMaxAttnSplits), nblk));
+  }
+
+  CU_TRY(ts::launch_embed_norm(in, (const __nv_bfloat16 *)m->W(L.embed), (const float *)m->W(L.g1[0]), c.rms_eps,
+                               d, x, h, R, m->planes, m->st));
+  ++m->launches;
+  GemmPlan plan{};
+  for (int l = 0; l < c.n_layers; ++l) {
+    if (l > 0) {
+      CU_TRY(ts::launch_add_norm(M, d, part, plan.splits, R, (const float *)m->W(L.g1[l]), c.rms_eps, x, h, R,
+                                 m->planes, m->st));
+      ++m->launches;
+    }
+    ts_status s = run_gemm(m, ts::EPI_PARTIAL, m->tm_qkv[l], m->tm_h, L.Nqkv, d, M, part, nullptr, nullptr, &plan);
+    if (s) return s;
+    CU_TRY(ts::launch_rope_kv(in, part, plan.splits, R, c.n_q_heads, c.n_kv_heads, c.head_dim, rope, q,
+                              m->k_pages(l), m->v_pages(l), m->st));
+    ++m->launches;
+    aa.k_pages = m->k_pages(l); aa.v_pages = m->v_pages(l);
+    CU_TRY(ts::launch_attention(aa, m->st));
+    m->launches += 2;
+    s = run_gemm(m, ts::EPI_PARTIAL, m->tm_o[l], m->tm_attn, d, Nq, M, part, nullptr, nullptr, &plan);
+    if (s) return s;
+    CU_TRY(ts::launch_add_norm(M, d, part, plan.splits, R, (const float *)m->W(L.g2[l]), c.rms_eps, x, h, R,
+                               m->planes, m->st));
+    ++m->launches;
+    s = run_gemm(m, ts::EPI_SWIGLU, m->tm_gu[l], m->tm_h, 2 * F, d, M, nullptr, act, nullptr, nullptr);
+    if (s) return s;
+    s = run_gemm(m, ts::EPI_PARTIAL, m->tm_d[l], m->tm_act, d, F, M, part, nullptr, nullptr, &plan);
+    if (s) return s;
+  }
+  if (m->last_flags & TS_FLAG_SKIP_LM_HEAD) return TS_OK;
+  CU_TRY(ts::launch_add_norm(M, d, part, plan.splits, R, (const float *)m->W(L.gf), c.rms_eps, x, h, R, m->planes,
+                             m->st));
+  ++m->launches;
+  float2 *amax = (float2 *)m->WS(L.amax);
+  ts_status s = run_gemm(m, ts::EPI_LOGITS, m->tm_lm, m->tm_h, c.vocab, d, M, (float *)m->WS(L.logits), nullptr,
+                         amax, nullptr);
+  if (s) return s;
+  ts::AcceptArgs ac{};
+  int32_t *dout = m->d_out();
+  ac.in = in; ac.amax = amax; ac.n_part = L.n_vocab_tiles * 4;
+  ac.argmax = dout + L.o_argmax; ac.accept_len = dout + L.o_accept; ac.emitted = dout + L.o_emitted;
+  ac.new_len = dout + L.o_newlen; ac.new_pending = dout + L.o_newpend; ac.k_max = c.k_max;
+  CU_TRY(ts::launch_accept(ac, m->st));
+  ++m->launches;
+  return TS_OK;
+}
+
+ts_status ensure_pages(ts_session *s, int tokens) {
+  ts_model *m = s->m;
+  const int need = (tokens + TS_PAGE_SIZE - 1) / TS_PAGE_SIZE;
+  if (need > m->L.pages_per_seq) return fail(TS_ERR_ARG, "sequence of %d tokens exceeds max_ctx %d", tokens, m->c.max_ctx);
+  while ((int)s->pages.size() < need) {
+    if (m->free_pages.empty()) return fail(TS_ERR_OOM_PAGES, "KV page pool exhausted (%d pages)", m->c.max_pages);
+    s->pages.push_back(m->free_pages.back());
+    m->free_pages.pop_back();
+  }
+  return TS_OK;
+}
+
+// Stage one step: rows[i] = chunk ids of sequence i.  Copies inputs, runs, copies results back, syncs.
+ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::vector<std::vector<int32_t>> &rows,
+                        uint32_t flags) {
+  const ts_model_config &c = m->c;
+  const Layout &L = m->L;
+  int32_t *hi = m->h_in();
+  const int G = c.n_q_heads / c.n_kv_heads;
+  int M = 0, tiles = 0;
+  hi[L.o_cu] = 0;
+  for (int i = 0; i < B; ++i) {
+    ts_session *s = ss[i];
+    const int k = (int)rows[i].size();
+    if (k < 1 || k > c.k_max) return fail(TS_ERR_K_TOO_LARGE, "sequence %d: chunk of %d rows, k_max is %d", i, k, c.k_max);
+    if (M + k > c.max_rows) return fail(TS_ERR_K_TOO_LARGE, "step has more than max_rows = %d rows", c.max_rows);
+    if (s->cache_len + k > c.max_ctx) return fail(TS_ERR_ARG, "sequence %d would exceed max_ctx", i);
+    for (int t : rows[i])
+      if (t < 0 || t >= c.vocab) return fail(TS_ERR_TOKEN_RANGE, "token id %d outside [0, %d)", t, c.vocab);
+    ts_status st = ensure_pages(s, s->cache_len + k);
+    if (st) return st;
+    for (int j = 0; j < k; ++j) {
+      hi[L.o_tokens + M + j] = rows[i][j];
+      hi[L.o_pos + M + j] = s->cache_len + j;
+      hi[L.o_rowseq + M + j] = i;
+    }
+    hi[L.o_len + i] = s->cache_len;
+    for (int r0 = 0; r0 < k * G; r0 += 64) {
+      hi[L.o_tile_seq + tiles] = i;
+      hi[L.o_tile_row0 + tiles] = r0;
+      ++tiles;
+    }
+    std::memcpy(hi + L.o_btab + (size_t)i * L.pages_per_seq, s->pages.data(), s->pages.size() * sizeof(int32_t));
+    M += k;
+    hi[L.o_cu + i + 1] = M;
+  }
+  m->last_B = B; m->last_M = M; m->last_tiles = tiles; m->last_flags = flags; m->have_step = true;
+  const size_t in_bytes = (size_t)(L.o_btab + (size_t)B * L.pages_per_seq) * 4;
+  CU_TRY(cudaMemcpyAsync(m->d_in(), hi, in_bytes, cudaMemcpyHostToDevice, m->st));
+  m->h2d += (int64_t)in_bytes;
+  ts_status st = run_step(m);
+  if (st) return st;
+  const size_t out_bytes = (size_t)L.out_ints * 4;
+  CU_TRY(cudaMemcpyAsync(m->h_out(), m->d_out(), out_bytes, cudaMemcpyDeviceToHost, m->st));
+  m->d2h += (int64_t)out_bytes;
+  CU_TRY(cudaStreamSynchronize(m->st));
+  const int dev_err = m->h_out()[L.o_err];
+  if (dev_err != 0) {
+    cudaMemsetAsync(m->d_out() + L.o_err, 0, 4, m->st);
+    return fail(TS_ERR_DEVICE_TIMEOUT, "a bounded device-side wait expired (code %d)", dev_err);
+  }
+  return TS_OK;
+}
+
+// y <- y (+) ids, delta per id, stop at the first finishing id.  Returns ids consumed.
+int commit_ids(ts_session *s, const int32_t *ids, int n) {
+  int used = 0;
+  for (int j = 0; j < n && !s->finished; ++j) {
+    s->y.push_back(ids[j]);
+    if (s->schema) s->fsm.step(ids[j]);
+    ++used;
+    const bool done = (s->schema && s->fsm.kind == ts::Q_DONE) ||
+                      (s->schema && ids[j] == s->schema->v.eos) ||
+                      (int)s->y.size() >= s->cfg.max_new_tokens;
+    if (done) s->finished = true;
+  }
+  return used;
+}
+
+int guess_tool(const ts_session *s) {
+  const ts_schema *sc = s->schema;
+  const ts::TrieNode &node = sc->trie[s->fsm.stage == ts::ST_NAME ? s->fsm.node : 0];
+  if (node.tools.empty()) return -1;
+  if (s->have_ranks && s->store) {
+    for (int32_t cnd : s->ranks) {
+      const int32_t t = s->store->tool_of[cnd];
+      if (t >= 0 && std::binary_search(node.tools.begin(), node.tools.end(), t)) return t;
+    }
+  }
+  int best = node.tools[0];
+  if (s->store) {
+    for (int32_t t : node.tools) {
+      const int64_t ft = t < (int32_t)s->store->freq.size() ? s->store->freq[t] : 0;
+      const int64_t fb = best < (int32_t)s->store->freq.size() ? s->store->freq[best] : 0;
+      if (ft > fb) best = t;
+    }
+  }
+  return best;
+}
+
+}  // namespace
+
+// =====================================================================================================
+extern "C" {
+
+const char *ts_last_error(void) { return g_err.c_str(); }
+
+ts_status ts_query_buffer_sizes(const ts_model_config *cfg, ts_buffer_sizes *out) {
+  if (!cfg || !out) return fail(TS_ERR_ARG, "null argument");
+  const char *why = "";
+  if (!config_ok(*cfg, &why)) return fail(TS_ERR_ARG, "bad configuration: %s", why);
+  Layout L;
+  make_layout(*cfg, &L);
+  out->weights_bytes = L.weights_bytes;
+  out->kv_pool_bytes = L.kv_bytes;
+  out->workspace_bytes = L.workspace_bytes;
+  out->host_io_bytes = L.host_io_bytes;
+  return TS_OK;
+}
+
+ts_status ts_init_model(const ts_model_config *cfg, const ts_buffers *bufs, void *stream, ts_model **out) {
+  if (!cfg || !bufs || !out) return fail(TS_ERR_ARG, "null argument");
+  const char *why = "";
+  if (!config_ok(*cfg, &why)) return fail(TS_ERR_ARG, "bad configuration: %s", why);
+  if (!bufs->weights || !bufs->kv_pool || !bufs->workspace || !bufs->host_io) return fail(TS_ERR_ARG, "null buffer");
+  if (((uintptr_t)bufs->weights | (uintptr_t)bufs->kv_pool | (uintptr_t)bufs->workspace) & 1023)
+    return fail(TS_ERR_ARG, "device buffers must be 1024-byte aligned");
+  int dev = 0;
+  CU_TRY(cudaGetDevice(&dev));
+  cudaDeviceProp prop;
+  CU_TRY(cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) return fail(TS_ERR_CUDA, "device is sm_%d%d; this library is built for sm_100a only", prop.major, prop.minor);
+  void *fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  CU_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+  if (!fn || qres != cudaDriverEntryPointSuccess) return fail(TS_ERR_CUDA, "cuTensorMapEncodeTiled not available");
+  EncodeTiledFn enc = (EncodeTiledFn)fn;
+
+  ts_model *m = new ts_model();
+  m->c = *cfg; m->b = *bufs; m->st = (cudaStream_t)stream;
+  m->planes = cfg->act_split ? 2 : 1;
+  m->n_sms = prop.multiProcessorCount;
+  make_layout(*cfg, &m->L);
+  const Layout &L = m->L;
+  const ts_model_config &c = m->c;
+  auto bail = [&](ts_status s) { delete m; return s; };
+
+  cudaError_t e = cudaMemsetAsync(bufs->workspace, 0, L.workspace_bytes, m->st);
+  if (e != cudaSuccess) return bail(fail(TS_ERR_CUDA, "cudaMemsetAsync(workspace): %s", cudaGetErrorString(e)));
+  {
+    // rotary table in double precision: (cos, sin) of pos * theta^(-2i/hd)
+    const int half = c.head_dim / 2;
+    std::vector<float2> tab((size_t)c.max_ctx * half);
+    std::vector<double> inv(half);
+    for (int i = 0; i < half; ++i) inv[i] = std::pow((double)c.rope_theta, -2.0 * i / c.head_dim);
+    for (int p = 0; p < c.max_ctx; ++p)
+      for (int i = 0; i < half; ++i) {
+        const double ang = (double)p * inv[i];
+        tab[(size_t)p * half + i] = make_float2((float)std::cos(ang), (float)std::sin(ang));
+      }
+    e = cudaMemcpyAsync(m->WS(L.rope), tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice, m->st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(m->st);
+    if (e != cudaSuccess) return bail(fail(TS_ERR_CUDA, "rotary table upload: %s", cudaGetErrorString(e)));
+  }
+  const uint64_t d = c.d_model, F = c.d_ffn, Nq = (uint64_t)c.n_q_heads * c.head_dim;
+  m->tm_qkv.resize(c.n_layers); m->tm_o.resize(c.n_layers); m->tm_gu.resize(c.n_layers); m->tm_d.resize(c.n_layers);
+  ts_status s = TS_OK;
+  for (int l = 0; l < c.n_layers && !s; ++l) {
+    s = weight_map(enc, &m->tm_qkv[l], m->W(L.wqkv[l]), L.Nqkv, d);
+    if (!s) s = weight_map(enc, &m->tm_o[l], m->W(L.wo[l]), d, Nq);
+    if (!s) s = weight_map(enc, &m->tm_gu[l], m->W(L.wgu[l]), 2 * F, d);
+    if (!s) s = weight_map(enc, &m->tm_d[l], m->W(L.wd[l]), d, F);
+  }
+  if (!s) s = weight_map(enc, &m->tm_lm, m->W(L.lm_head), c.vocab, d);
+  if (!s) s = act_maps(enc, m->tm_h, m->WS(L.h), d, L.rows_alloc, m->planes);
+  if (!s) s = act_maps(enc, m->tm_attn, m->WS(L.attn), Nq, L.rows_alloc, m->planes);
+  if (!s) s = act_maps(enc, m->tm_act, m->WS(L.act), F, L.rows_alloc, m->planes);
+  if (s) return bail(s);
+  m->free_pages.resize(c.max_pages);
+  for (int i = 0; i < c.max_pages; ++i) m->free_pages[i] = c.max_pages - 1 - i;   // hand out 0, 1, 2, ...
+  *out = m;
+  return TS_OK;
+}
+
+ts_status ts_model_destroy(ts_model *m) {
+  if (!m) return TS_OK;
+  cudaStreamSynchronize(m->st);
+  delete m;
+  return TS_OK;
+}
+
+ts_status ts_load_tensor(ts_model *m, int32_t kind, int32_t layer, const void *host, int64_t rows, int64_t cols) {
+  if (!m || !host) return fail(TS_ERR_ARG, "null argument");
+  const ts_model_config &c = m->c;
+  const Layout &L = m->L;
+  const int64_t d = c.d_model, F = c.d_ffn, hd = c.head_dim, Nq = (int64_t)c.n_q_heads * hd, Nkv = (int64_t)c.n_kv_heads * hd;
+  const bool global = kind == TS_W_EMBED || kind == TS_W_LM_HEAD || kind == TS_W_FINAL_GAIN;
+  if (!global && (layer < 0 || layer >= c.n_layers)) return fail(TS_ERR_ARG, "layer %d out of range", layer);
+  int64_t er = 0, ec = 0;
+  uint8_t *dst = nullptr;
+  size_t dpitch = 0, esz = 2;
+  switch (kind) {
+    case TS_W_EMBED: er = c.vocab; ec = d; dst = m->W(L.embed); break;
+    case TS_W_LM_HEAD: er = c.vocab; ec = d; dst = m->W(L.lm_head); break;
+    case TS_W_FINAL_GAIN: er = 1; ec = d; dst = m->W(L.gf); esz = 4; break;
+    case TS_W_GAIN1: er = 1; ec = d; dst = m->W(L.g1[layer]); esz = 4; break;
+    case TS_W_GAIN2: er = 1; ec = d; dst = m->W(L.g2[layer]); esz = 4; break;
+    case TS_W_Q: er = Nq; ec = d; dst = m->W(L.wqkv[layer]); break;
+    case TS_W_K: er = Nkv; ec = d; dst = m->W(L.wqkv[layer]) + Nq * d * 2; break;
+    case TS_W_V: er = Nkv; ec = d; dst = m->W(L.wqkv[layer]) + (Nq + Nkv) * d * 2; break;
+    case TS_W_O: er = d; ec = Nq; dst = m->W(L.wo[layer]); break;
+    case TS_W_GATE: er = F; ec = d; dst = m->W(L.wgu[layer]); dpitch = 2 * d * 2; break;           // even rows
+    case TS_W_UP: er = F; ec = d; dst = m->W(L.wgu[layer]) + d * 2; dpitch = 2 * d * 2; break;      // odd rows
+    case TS_W_DOWN: er = d; ec = F; dst = m->W(L.wd[layer]); break;
+    default: return fail(TS_ERR_ARG, "unknown tensor kind %d", kind);
+  }
+  if (rows != er || cols != ec) return fail(TS_ERR_ARG, "tensor kind %d: expected %lld x %lld, got %lld x %lld", kind,
+                                            (long long)er, (long long)ec, (long long)rows, (long long)cols);
+  const size_t row_bytes = (size_t)ec * esz;
+  if (dpitch == 0) dpitch = row_bytes;
+  CU_TRY(cudaMemcpy2DAsync(dst, dpitch, host, row_bytes, row_bytes, (size_t)er, cudaMemcpyHostToDevice, m->st));
+  CU_TRY(cudaStreamSynchronize(m->st));
+  return TS_OK;
+}
+
+// ---- schema ------------------------------------------------------------------------------------------
+ts_status ts_schema_create(const ts_vocab_layout *v, ts_schema **out) {
+  if (!v || !out) return fail(TS_ERR_ARG, "null argument");
+  const int32_t lens[5] = {v->pfx_len, v->mid_len, v->kvsep_len, v->nxt_len, v->end_len};
+  for (int i = 0; i < 5; ++i)
+    if (lens[i] < (i == 0 ? 0 : 1) || lens[i] > 8) return fail(TS_ERR_ARG, "scaffolding string length out of range");
+  ts_schema *s = new ts_schema();
+  s->v = *v;
+  s->trie.emplace_back();
+  *out = s;
+  return TS_OK;
+}
+
+ts_status ts_schema_add_tool(ts_schema *s, const int32_t *name, int32_t name_len, const int32_t *key_tokens,
+                             const int32_t *key_offsets, int32_t n_keys) {
+  if (!s || !name || !key_tokens || !key_offsets) return fail(TS_ERR_ARG, "null argument");
+  if (name_len < 1 || n_keys < 1) return fail(TS_ERR_ARG, "a tool needs a name and at least one key");
+  ts::ToolDef t;
+  t.name.assign(name, name + name_len);
+  for (int k = 0; k < n_keys; ++k) {
+    if (key_offsets[k + 1] <= key_offsets[k]) return fail(TS_ERR_ARG, "empty key");
+    t.keys.emplace_back(key_tokens + key_offsets[k], key_tokens + key_offsets[k + 1]);
+  }
+  int32_t node = 0;
+  const int32_t id = (int32_t)s->tools.size();
+  {
+    // reject duplicates
+    int32_t n = s->walk(t.name);
+    if (n >= 0 && s->trie[n].tool_exact >= 0) return fail(TS_ERR_ARG, "duplicate tool name");
+  }
+  s->trie[0].tools.push_back(id);
+  if (s->trie[0].min_tool < 0) s->trie[0].min_tool = id;
+  for (int32_t tok : t.name) {
+    int32_t nx = s->child(node, tok);
+    if (nx < 0) {
+      nx = (int32_t)s->trie.size();
+      s->trie.emplace_back();
+      auto &v = s->trie[node].next;
+      v.insert(std::lower_bound(v.begin(), v.end(), std::make_pair(tok, INT32_MIN)), {tok, nx});
+    }
+    node = nx;
+    s->trie[node].tools.push_back(id);
+    if (s->trie[node].min_tool < 0) s->trie[node].min_tool = id;
+  }
+  s->trie[node].tool_exact = id;
+  s->tools.push_back(std::move(t));
+  return TS_OK;
+}
+
+ts_status ts_schema_destroy(ts_schema *s) { delete s; return TS_OK; }
+
+// ---- datastore -----------------------------------------------------------------------------------------
+ts_status ts_datastore_create(int32_t n_tools, ts_datastore **out) {
+  if (!out || n_tools < 0) return fail(TS_ERR_ARG, "bad argument");
+  ts_datastore *d = new ts_datastore();
+  d->freq.assign(n_tools, 0);
+  *out = d;
+  return TS_OK;
+}
+
+ts_status ts_datastore_add(ts_datastore *d, const int32_t *tokens, int32_t n, int32_t tool_id) {
+  if (!d || (!tokens && n > 0) || n < 0) return fail(TS_ERR_ARG, "bad argument");
+  d->tokens.insert(d->tokens.end(), tokens, tokens + n);
+  d->offset.push_back((int64_t)d->tokens.size());
+  d->tool_of.push_back(tool_id);
+  if (tool_id >= 0 && tool_id < (int32_t)d->freq.size()) ++d->freq[tool_id];
+  return TS_OK;
+}
+
+ts_status ts_datastore_destroy(ts_datastore *d) { delete d; return TS_OK; }
+
+// ---- sessions ------------------------------------------------------------------------------------------
+ts_status ts_session_create(ts_model *model, const ts_schema *schema, const ts_datastore *store,
+                            const ts_draft_config *cfg, ts_session **out) {
+  if (!out || !cfg) return fail(TS_ERR_ARG, "null argument");
+  if (cfg->n_cap < 0 || cfg->max_new_tokens < 1) return fail(TS_ERR_ARG, "bad draft configuration");
+  ts_session *s = new ts_session();
+  s->m = model; s->schema = schema; s->store = store; s->cfg = *cfg;
+  s->fsm.s = schema;
+  *out = s;
+  return TS_OK;
+}
+
+ts_status ts_session_set_ranks(ts_session *s, const int32_t *ranks, int32_t n) {
+  if (!s || n < 0 || (n > 0 && !ranks)) return fail(TS_ERR_ARG, "bad argument");
+  if (n > 0 && !s->store) return fail(TS_ERR_STATE, "session has no datastore");
+  for (int i = 0; i < n; ++i)
+    if (ranks[i] < 0 || ranks[i] >= s->store->n_entries()) return fail(TS_ERR_ARG, "rank entry %d out of range", ranks[i]);
+  s->ranks.assign(ranks, ranks + n);
+  s->have_ranks = n > 0;
+  return TS_OK;
+}
+
+ts_status ts_session_destroy(ts_session *s) {
+  if (!s) return TS_OK;
+  if (s->m)
+    for (int32_t p : s->pages) s->m->free_pages.push_back(p);
+  delete s;
+  return TS_OK;
+}
+
+ts_status ts_prefill(ts_model *m, ts_session *s, const int32_t *tokens, int32_t n) {
+  if (!s || !tokens || n < 1) return fail(TS_ERR_ARG, "bad argument");
+  if (s->m != m) return fail(TS_ERR_ARG, "session belongs to another model");
+  if (s->cache_len >= 0) return fail(TS_ERR_STATE, "session already has a context");
+  if (s->schema)
+    for (int i = 0; i < n; ++i) s->fsm.step(tokens[i]);
+  s->cache_len = 0;
+  if (m) {
+    std::vector<std::vector<int32_t>> rows(1);
+    for (int i = 0; i < n - 1; i += m->c.k_max) {
+      const int k = std::min(m->c.k_max, n - 1 - i);
+      rows[0].assign(tokens + i, tokens + i + k);
+      ts_status st = stage_and_run(m, &s, 1, rows, TS_FLAG_SKIP_LM_HEAD);
+      if (st) { s->cache_len = -1; return st; }
+      s->cache_len += k;
+    }
+  } else {
+    s->cache_len = n - 1;
+  }
+  s->pending = tokens[n - 1];
+  return TS_OK;
+}
+
+ts_status ts_draft(ts_session *s, int32_t max_draft, int32_t *out_tokens, int32_t *out_n, int32_t *out_source) {
+  if (!s || !out_n || !out_source || (max_draft > 0 && !out_tokens)) return fail(TS_ERR_ARG, "null argument");
+  *out_n = 0; *out_source = 0;
+  if (max_draft <= 0 || s->finished) return TS_OK;
+  std::vector<int32_t> d;
+  if (s->store) {
+    const int n = std::min(s->cfg.n_cap, max_draft);
+    ts::suffix_match(s->y, *s->store, s->have_ranks ? &s->ranks : nullptr, n, &d);
+    if (!d.empty()) *out_source = 2;
+  }
+  if (d.empty() && s->schema) {
+    int guess = -1;
+    if (s->fsm.kind == ts::Q_T && s->fsm.stage != ts::ST_MID) guess = guess_tool(s);
+    s->fsm.draft(guess, &d);
+    if ((int)d.size() > max_draft) d.resize(max_draft);
+    if (!d.empty()) *out_source = 1;
+  }
+  std::memcpy(out_tokens, d.data(), d.size() * sizeof(int32_t));
+  *out_n = (int32_t)d.size();
+  return TS_OK;
+}
+
+ts_status ts_verify(ts_model *m, ts_session *const *ss, int32_t B, const int32_t *draft_tokens,
+                    const int32_t *draft_offsets, uint32_t flags, ts_verify_result *out) {
+  if (!m || !ss || !draft_offsets || !out) return fail(TS_ERR_ARG, "null argument");
+  if (B < 1 || B > m->c.max_batch) return fail(TS_ERR_ARG, "batch %d outside [1, %d]", B, m->c.max_batch);
+  std::vector<std::vector<int32_t>> rows(B);
+  for (int i = 0; i < B; ++i) {
+    ts_session *s = ss[i];
+    if (!s || s->m != m) return fail(TS_ERR_ARG, "session %d is null or belongs to another model", i);
+    if (s->cache_len < 0 || s->pending < 0) return fail(TS_ERR_STATE, "session %d has no context (call ts_prefill)", i);
+    if (s->finished) return fail(TS_ERR_STATE, "session %d is finished", i);
+    for (int j = 0; j < i; ++j)
+      if (ss[j] == s) return fail(TS_ERR_ARG, "session listed twice");
+    const int n = draft_offsets[i + 1] - draft_offsets[i];
+    if (n < 0) return fail(TS_ERR_ARG, "draft_offsets not ascending");
+    if (n > 0 && !draft_tokens) return fail(TS_ERR_ARG, "null draft_tokens");
+    rows[i].reserve(n + 1);
+    rows[i].push_back(s->pending);
+    for (int j = 0; j < n; ++j) rows[i].push_back(draft_tokens[draft_offsets[i] + j]);
+  }
+  ts_status st = stage_and_run(m, ss, B, rows, flags);
+  if (st) return st;
+  const Layout &L = m->L;
+  const int32_t *ho = m->h_out();
+  int row = 0;
+  for (int i = 0; i < B; ++i) {
+    ts_verify_result &r = out[i];
+    std::memset(&r, 0, sizeof r);
+    r.k = (int32_t)rows[i].size();
+    r.first_row = row;
+    ss[i]->last_chunk = rows[i];
+    if (!(flags & TS_FLAG_SKIP_LM_HEAD)) {
+      r.accept_len = ho[L.o_accept + i];
+      r.n_emitted = r.accept_len + 1;
+      for (int j = 0; j < r.n_emitted; ++j) r.emitted[j] = ho[L.o_emitted + i * m->c.k_max + j];
+      for (int j = 0; j < r.k; ++j) r.argmax[j] = ho[L.o_argmax + row + j];
+    }
+    row += r.k;
+  }
+  return TS_OK;
+}
+
+ts_status ts_verify_replay(ts_model *m) {
+  if (!m) return fail(TS_ERR_ARG, "null argument");
+  if (!m->have_step) return fail(TS_ERR_STATE, "no step has been staged yet");
+  return run_step(m);
+}
+
+ts_status ts_commit_forced(ts_session *s, const int32_t *emitted, int32_t n) {
+  if (!s || !emitted || n < 1) return fail(TS_ERR_ARG, "bad argument");
+  if (s->finished) return fail(TS_ERR_STATE, "session is finished");
+  if (s->cache_len < 0) return fail(TS_ERR_STATE, "session has no context");
+  const int used = commit_ids(s, emitted, n);
+  s->cache_len += used;
+  s->pending = emitted[used - 1];
+  return TS_OK;
+}
+
+ts_status ts_commit(ts_session *s, const ts_verify_result *r) {
+  if (!s || !r) return fail(TS_ERR_ARG, "null argument");
+  if (r->n_emitted < 1 || r->n_emitted > TS_K_MAX) return fail(TS_ERR_ARG, "result carries no emitted ids");
+  return ts_commit_forced(s, r->emitted, r->n_emitted);
+}
+
+ts_status ts_session_state(const ts_session *s, ts_session_info *out) {
+  if (!s || !out) return fail(TS_ERR_ARG, "null argument");
+  out->cache_len = s->cache_len; out->pending = s->pending; out->n_output = (int32_t)s->y.size();
+  out->finished = s->finished ? 1 : 0;
+  out->fsm_kind = s->fsm.kind; out->fsm_tool = s->fsm.tool; out->fsm_key = s->fsm.key;
+  out->n_pages = (int32_t)s->pages.size();
+  return TS_OK;
+}
+
+ts_status ts_session_output(const ts_session *s, int32_t *out, int32_t cap, int32_t *n) {
+  if (!s || !n || (cap > 0 && !out)) return fail(TS_ERR_ARG, "null argument");
+  *n = (int32_t)s->y.size();
+  std::memcpy(out, s->y.data(), sizeof(int32_t) * std::min<size_t>(cap, s->y.size()));
+  return TS_OK;
+}
+
+// ---- test / benchmark support -------------------------------------------------------------------------
+static ts_status kv_transfer(ts_model *m, ts_session *s, int layer, void *k, void *v, int n_tokens, bool to_device) {
+  if (!m || !s || !k || !v) return fail(TS_ERR_ARG, "null argument");
+  if (s->m != m) return fail(TS_ERR_ARG, "session belongs to another model");
+  if (layer < 0 || layer >= m->c.n_layers || n_tokens < 0) return fail(TS_ERR_ARG, "bad layer / length");
+  if (to_device) {
+    ts_status st = ensure_pages(s, n_tokens);
+    if (st) return st;
+  } else if ((n_tokens + TS_PAGE_SIZE - 1) / TS_PAGE_SIZE > (int)s->pages.size()) {
+    return fail(TS_ERR_ARG, "session holds fewer than %d tokens", n_tokens);
+  }
+  const int Hkv = m->c.n_kv_heads, hd = m->c.head_dim;
+  const size_t page_elems = (size_t)Hkv * TS_PAGE_SIZE * hd;
+  std::vector<uint16_t> stage(page_elems);
+  for (int which = 0; which < 2; ++which) {
+    uint16_t *host = (uint16_t *)(which ? v : k);
+    __nv_bfloat16 *pool = which ? m->v_pages(layer) : m->k_pages(layer);
+    for (int p = 0; p * TS_PAGE_SIZE < n_tokens; ++p) {
+      const int t0 = p * TS_PAGE_SIZE, nt = std::min(TS_PAGE_SIZE, n_tokens - t0);
+      __nv_bfloat16 *dev = pool + (size_t)s->pages[p] * page_elems;
+      if (to_device) {
+        std::fill(stage.begin(), stage.end(), 0);
+        for (int t = 0; t < nt; ++t)
+          for (int hh = 0; hh < Hkv; ++hh)
+            std::memcpy(&stage[((size_t)hh * TS_PAGE_SIZE + t) * hd], &host[((size_t)(t0 + t) * Hkv + hh) * hd], hd * 2);
+        CU_TRY(cudaMemcpyAsync(dev, stage.data(), page_elems * 2, cudaMemcpyHostToDevice, m->st));
+        CU_TRY(cudaStreamSynchronize(m->st));
+      } else {
+        CU_TRY(cudaMemcpyAsync(stage.data(), dev, page_elems * 2, cudaMemcpyDeviceToHost, m->st));
+        CU_TRY(cudaStreamSynchronize(m->st));
+        for (int t = 0; t < nt; ++t)
+          for (int hh = 0; hh < Hkv; ++hh)
+            std::memcpy(&host[((size_t)(t0 + t) * Hkv + hh) * hd], &stage[((size_t)hh * TS_PAGE_SIZE + t) * hd], hd * 2);
+      }
+    }
+  }
+  return TS_OK;
+}
+
+ts_status ts_debug_import_kv(ts_model *m, ts_session *s, int32_t layer, const void *k, const void *v, int32_t n) {
+  return kv_transfer(m, s, layer, (void *)k, (void *)v, n, true);
+}
+ts_status ts_debug_export_kv(ts_model *m, ts_session *s, int32_t layer, void *k, void *v, int32_t n) {
+  return kv_transfer(m, s, layer, k, v, n, false);
+}
+
+ts_status ts_debug_set_cache(ts_session *s, int32_t cache_len, int32_t pending) {
+  if (!s || cache_len < 0 || pending < 0) return fail(TS_ERR_ARG, "bad argument");
+  if (s->m) {
+    if (pending >= s->m->c.vocab) return fail(TS_ERR_TOKEN_RANGE, "pending id out of range");
+    ts_status st = ensure_pages(s, cache_len);
+    if (st) return st;
+  }
+  s->cache_len = cache_len;
+  s->pending = pending;
+  return TS_OK;
+}
+
+ts_status ts_read_logits(ts_model *m, int32_t row0, int32_t n_rows, float *host_out) {
+  if (!m || !host_out) return fail(TS_ERR_ARG, "null argument");
+  if (!m->have_step || (m->last_flags & TS_FLAG_SKIP_LM_HEAD)) return fail(TS_ERR_STATE, "last step produced no logits");
+  if (row0 < 0 || n_rows < 0 || row0 + n_rows > m->last_M) return fail(TS_ERR_ARG, "rows outside the last step");
+  const size_t V = m->c.vocab;
+  CU_TRY(cudaMemcpyAsync(host_out, (float *)m->WS(m->L.logits) + (size_t)row0 * V, (size_t)n_rows * V * 4,
+                         cudaMemcpyDeviceToHost, m->st));
+  CU_TRY(cudaStreamSynchronize(m->st));
+  return TS_OK;
+}
+
+ts_status ts_debug_read_buffer(ts_model *m, int32_t which, void *host_out, uint64_t bytes) {
+  if (!m || !host_out) return fail(TS_ERR_ARG, "null argument");
+  const Layout &L = m->L;
+  const uint64_t R = L.rows_alloc, P = m->planes, d = m->c.d_model, Nq = (uint64_t)m->c.n_q_heads * m->c.head_dim;
+  uint64_t off = 0, cap = 0;
+  switch (which) {
+    case 0: off = L.x; cap = R * d * 4; break;
+    case 1: off = L.h; cap = P * R * d * 2; break;
+    case 2: off = L.q; cap = R * Nq * 2; break;
+    case 3: off = L.attn; cap = P * R * Nq * 2; break;
+    case 4: off = L.act; cap = P * R * (uint64_t)m->c.d_ffn * 2; break;
+    default: return fail(TS_ERR_ARG, "unknown buffer %d", which);
+  }
+  if (bytes > cap) return fail(TS_ERR_ARG, "buffer %d holds %llu bytes", which, (unsigned long long)cap);
+  CU_TRY(cudaMemcpyAsync(host_out, m->WS(off), bytes, cudaMemcpyDeviceToHost, m->st));
+  CU_TRY(cudaStreamSynchronize(m->st));
+  return TS_OK;
+}
+
+ts_status ts_model_counters(const ts_model *m, int64_t *launches, int64_t *h2d, int64_t *d2h) {
+  if (!m) return fail(TS_ERR_ARG, "null argument");
+  if (launches) *launches = m->launches;
+  if (h2d) *h2d = m->h2d;
+  if (d2h) *d2h = m->d2h;
+  return TS_OK;
+}
+
+}  // extern "C"

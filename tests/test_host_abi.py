@@ -1,0 +1,149 @@
+"""CPU-only checks of the boundary: the library loads, exports every declared symbol, validates
+arguments, and its host C++ drafter (FSM, datastore index, commit) is bit-exact with the oracle."""
+import ctypes as C
+import os
+import random
+import re
+
+import pytest
+
+import oracle
+import synth
+import paper_2604_13519_b200 as ts
+from paper_2604_13519_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2604_13519_b200 import build
+    build.build()
+
+
+def test_exports_every_declared_symbol():
+    hdr = open(os.path.join(ROOT, "include", "toolspec.h")).read()
+    declared = set(re.findall(r"^(?:ts_status|const char \*)\s*(ts_[a-z_0-9]+)\s*\(", hdr, re.M))
+    assert {"ts_init_model", "ts_draft", "ts_verify", "ts_commit"} <= declared
+    L = B.lib()
+    for name in declared:
+        assert hasattr(L, name), name
+    assert declared == set(B.EXPORTED)
+
+
+def test_buffer_sizes_and_argument_errors():
+    c = B.ts_model_config()
+    s = synth.SHAPES["8b"]
+    for n in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab", "rope_theta", "rms_eps"):
+        setattr(c, n, getattr(s, n))
+    c.max_pages, c.max_batch, c.k_max, c.max_rows, c.max_ctx, c.act_split = 1024, 1, 32, 32, 16384, 1
+    out = B.ts_buffer_sizes()
+    assert B.lib().ts_query_buffer_sizes(C.byref(c), C.byref(out)) == 0
+    w_expect = 2 * (s.n_params_matmul() + s.vocab * s.d_model)
+    assert w_expect <= out.weights_bytes < w_expect * 1.001 + (1 << 20)
+    assert out.kv_pool_bytes == 1024 * 16 * s.n_kv_heads * s.head_dim * 2 * 2 * s.n_layers
+    c.head_dim = 96
+    assert B.lib().ts_query_buffer_sizes(C.byref(c), C.byref(out)) == -1
+    assert b"head_dim" in B.lib().ts_last_error()
+    c.head_dim, c.k_max = 128, 65
+    assert B.lib().ts_query_buffer_sizes(C.byref(c), C.byref(out)) == -1
+    assert B.lib().ts_query_buffer_sizes(None, C.byref(out)) == -1
+    # no device here (or no model): the verify entry point must fail, never fall back
+    assert B.lib().ts_verify(None, None, 1, None, None, 0, None) == -1
+    assert B.lib().ts_verify_replay(None) == -1
+
+
+def _pair(schema, inv, n_cap=32, ranks=None, max_new=10 ** 6):
+    st_o = oracle.Datastore(len(schema.tools))
+    st_c = ts.Datastore(len(schema.tools))
+    for tid, toks in inv:
+        st_o.add(toks, tid)
+        st_c.add(toks, tid)
+    sc = ts.Schema(schema.vocab, schema.tools)
+    d = oracle.Drafter(schema, st_o, n_cap=n_cap, ranks=ranks)
+    s = ts.Session(None, sc, st_c, n_cap=n_cap, max_new_tokens=max_new)
+    if ranks is not None:
+        s.set_ranks(ranks)
+    return d, s
+
+
+KIND = {oracle.Q_O: 0, oracle.Q_T: 1, oracle.Q_P: 2, oracle.Q_V: 3, oracle.Q_DONE: 4}
+
+
+@pytest.mark.parametrize("seed,n_tools,n_inv,ranks", [(1, 8, 64, None), (2, 32, 300, None), (3, 16, 100, [7, 3, 50, 9])])
+def test_draft_and_commit_bit_exact_with_oracle(seed, n_tools, n_inv, ranks):
+    schema = synth.make_schema(4096, n_tools, seed=seed)
+    inv = synth.make_datastore(schema, n_inv, seed=seed)
+    rnd = random.Random(seed)
+    v = schema.vocab
+    for trial in range(40):
+        d, s = _pair(schema, inv, ranks=ranks, max_new=200)
+        prompt = [rnd.randrange(64, 4096) for _ in range(5)] + [v.tool_call]
+        d.feed_prompt(prompt)
+        ts.ts_prefill(None, s, prompt)
+        # script: a historical invocation, perturbed in places so that both drafters see misses,
+        # off-schema ids and early stops
+        tid, script = inv[rnd.randrange(len(inv))]
+        script = list(script)
+        for _ in range(rnd.randrange(0, 3)):
+            script[rnd.randrange(len(script))] = rnd.randrange(64, 4096)
+        script += [rnd.randrange(64, 4096) for _ in range(10)] + [v.eos]
+        pos = 0
+        while pos < len(script):
+            md = rnd.choice([0, 1, 5, 31, 63])
+            want, src = d.draft(md)
+            got, gsrc = ts.ts_draft(s, md)
+            assert (got, gsrc) == (want, src), (trial, pos)
+            n = rnd.randrange(1, 8)
+            span = script[pos:pos + n]
+            used, fin = d.commit(span, v.eos, 200)
+            ts.ts_commit_forced(s, span)
+            info = s.state()
+            assert info.n_output == len(d.y) and bool(info.finished) == fin
+            assert info.fsm_kind == KIND[d.fsm.kind]
+            if d.fsm.kind in (oracle.Q_P, oracle.Q_V):
+                assert (info.fsm_tool, info.fsm_key) == (d.fsm.tool, d.fsm.key)
+            assert info.cache_len == len(prompt) - 1 + len(d.y)
+            pos += used
+            if fin:
+                break
+        assert s.output() == d.y
+
+
+def test_large_store_whole_index_search():
+    schema = synth.make_schema(8192, 64, seed=9)
+    inv = synth.make_datastore(schema, 3000, seed=9, total_len=(20, 120))
+    d, s = _pair(schema, inv, n_cap=64)
+    rnd = random.Random(9)
+    hits = 0
+    for trial in range(60):
+        tid, toks = inv[rnd.randrange(len(inv))]
+        cut = rnd.randrange(5, len(toks))
+        d.y = list(toks[:cut]) if trial % 3 else [rnd.randrange(64, 8192) for _ in range(9)]
+        # mirror y into the C session through forced commits on a fresh session
+        s = ts.Session(None, s.schema, s.store, n_cap=64)
+        ts.ts_prefill(None, s, [77])
+        ts.ts_commit_forced(s, d.y)
+        want, _ = oracle.suffix_match(d.y, d.store, None, 64, 63)
+        got, src = ts.ts_draft(s, 63)
+        if want:
+            hits += 1
+            assert src == 2 and got == want
+        else:
+            assert src != 2
+    assert hits > 20
+
+
+def test_session_errors():
+    schema = synth.make_schema(4096, 4, seed=1)
+    sc = ts.Schema(schema.vocab, schema.tools)
+    s = ts.Session(None, sc, None)
+    with pytest.raises(ts.TsError) as e:
+        ts.ts_commit_forced(s, [5])
+    assert e.value.code == -2          # no context yet
+    ts.ts_prefill(None, s, [9, 3])
+    with pytest.raises(ts.TsError):
+        ts.ts_prefill(None, s, [9, 3])   # twice
+    assert ts.ts_draft(s, 0) == ([], 0)
+    with pytest.raises(ts.TsError):
+        s.set_ranks([0])                 # no datastore
