@@ -60,7 +60,7 @@ typedef struct ts_session ts_session;
 typedef struct {
   int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
   float rope_theta, rms_eps;
-  int32_t max_pages;   /* KV pages in the pool (each TS_PAGE_SIZE tokens, all layers) */
+  int32_t max_pages;   /* KV pages in the pool (each TS_PAGE_SIZE tokens, all layers; fp16 elements) */
   int32_t max_batch;   /* most sequences per ts_verify call */
   int32_t k_max;       /* most rows per sequence per call, <= TS_K_MAX */
   int32_t max_rows;    /* most rows per call summed over the batch */
@@ -202,19 +202,21 @@ ts_status ts_session_state(const ts_session *s, ts_session_info *out);
 ts_status ts_session_output(const ts_session *s, int32_t *out, int32_t cap, int32_t *n);
 
 /* ---- test / benchmark support ------------------------------------------------------------------- */
-/* Overwrite the session's cache for one layer with n_tokens rows of host bf16 K and V
- * ([n_tokens][n_kv_heads][head_dim]).  After all layers were imported with the same n_tokens call
+/* Overwrite the session's cache for one layer with n_tokens rows of host float32 K and V
+ * ([n_tokens][n_kv_heads][head_dim]); values are rounded to the cache's storage type (fp16,
+ * saturating).  After all layers were imported with the same n_tokens call
  * ts_debug_set_cache(s, n_tokens, pending) to make them the session's context. */
-ts_status ts_debug_import_kv(ts_model *m, ts_session *s, int32_t layer, const void *k_bf16,
-                             const void *v_bf16, int32_t n_tokens);
-ts_status ts_debug_export_kv(ts_model *m, ts_session *s, int32_t layer, void *k_bf16, void *v_bf16,
+ts_status ts_debug_import_kv(ts_model *m, ts_session *s, int32_t layer, const float *k,
+                             const float *v, int32_t n_tokens);
+/* Read the first n_tokens cached rows of one layer back as float32. */
+ts_status ts_debug_export_kv(ts_model *m, ts_session *s, int32_t layer, float *k, float *v,
                              int32_t n_tokens);
 ts_status ts_debug_set_cache(ts_session *s, int32_t cache_len, int32_t pending);
 /* Copy rows [row0, row0+n_rows) of the last step's float32 logits [rows][vocab] to host memory. */
 ts_status ts_read_logits(ts_model *m, int32_t row0, int32_t n_rows, float *host_out);
 /* Copy the first `bytes` bytes of an internal activation buffer of the last step to host memory:
  * 0 residual stream x (float32 [rows_alloc][d_model]); 1 normed activations (bf16
- * [planes][rows_alloc][d_model]); 2 rotated queries (bf16 [rows_alloc][n_q_heads*head_dim]);
+ * [planes][rows_alloc][d_model]); 2 rotated queries (fp16 [rows_alloc][n_q_heads*head_dim]);
  * 3 attention output (bf16 [planes][rows_alloc][n_q_heads*head_dim]); 4 SwiGLU output (bf16
  * [planes][rows_alloc][d_ffn]).  rows_alloc = max_rows rounded up to 128; planes = 1 + act_split. */
 ts_status ts_debug_read_buffer(ts_model *m, int32_t which, void *host_out, uint64_t bytes);

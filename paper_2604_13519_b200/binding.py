@@ -211,11 +211,11 @@ class Model:
         _check(lib().ts_init_model(C.byref(c), C.byref(b), _P(sp), C.byref(self.h)))
 
     def kv_pool_tensor(self):
-        """The caller-owned KV pool viewed as a bf16 tensor (e.g. to fill it with synthetic data)."""
+        """The caller-owned KV pool viewed as an fp16 tensor (e.g. to fill it with synthetic data)."""
         torch = self.torch
         off = self.kv_pool_ptr - self._raw[1].data_ptr()
         n = int(self.sizes.kv_pool_bytes)
-        return self._raw[1][off:off + n].view(torch.bfloat16)
+        return self._raw[1][off:off + n].view(torch.float16)
 
     def load_tensor(self, kind: int, layer: int, t):
         t = t.contiguous()
@@ -247,7 +247,7 @@ class Model:
         P = 1 + self.cfg.act_split
         Nq = s.n_q_heads * s.head_dim
         shape, dt = {0: ((R, s.d_model), torch.float32), 1: ((P, R, s.d_model), torch.bfloat16),
-                     2: ((R, Nq), torch.bfloat16), 3: ((P, R, Nq), torch.bfloat16),
+                     2: ((R, Nq), torch.float16), 3: ((P, R, Nq), torch.bfloat16),
                      4: ((P, R, s.d_ffn), torch.bfloat16)}[which]
         out = torch.empty(shape, dtype=dt)
         _check(lib().ts_debug_read_buffer(self.h, which, _P(out.data_ptr()), out.numel() * out.element_size()))
@@ -298,15 +298,15 @@ class Session:
         _check(lib().ts_debug_set_cache(self.h, cache_len, pending))
 
     def import_kv(self, layer: int, k, v):
-        """k, v: CPU bf16 tensors [n_tokens][n_kv_heads][head_dim]."""
-        k, v = k.contiguous(), v.contiguous()
+        """k, v: CPU tensors [n_tokens][n_kv_heads][head_dim] (any float dtype; sent as float32)."""
+        k, v = k.float().contiguous(), v.float().contiguous()
         _check(lib().ts_debug_import_kv(self.model.h, self.h, layer, _P(k.data_ptr()), _P(v.data_ptr()),
                                         k.shape[0]))
 
     def export_kv(self, layer: int, n_tokens: int):
         torch = self.model.torch
         s = self.model.shape
-        k = torch.empty(n_tokens, s.n_kv_heads, s.head_dim, dtype=torch.bfloat16)
+        k = torch.empty(n_tokens, s.n_kv_heads, s.head_dim, dtype=torch.float32)
         v = torch.empty_like(k)
         _check(lib().ts_debug_export_kv(self.model.h, self.h, layer, _P(k.data_ptr()), _P(v.data_ptr()),
                                         n_tokens))

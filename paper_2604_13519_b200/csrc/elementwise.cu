@@ -89,11 +89,14 @@ cudaError_t launch_add_norm(int M, int d, const float *part, int n_splits, int p
                     planes);
 }
 
+__device__ __forceinline__ __half to_half_sat(float x) {
+  return __float2half_rn(fminf(fmaxf(x, -65504.f), 65504.f));
+}
+
 // grid = (M, Hq + 2*Hkv); one CTA of hd/2 threads per (row, head).  Thread i handles the rotary pair
 // (i, i + hd/2) of q or k heads, or elements (i, i + hd/2) of a v head.
 __global__ void rope_kv_kernel(StepIn in, const float *part, int n_splits, int part_rows, int Hq, int Hkv, int hd,
-                               const float2 *rope_tab, __nv_bfloat16 *q_out, __nv_bfloat16 *k_pages,
-                               __nv_bfloat16 *v_pages) {
+                               const float2 *rope_tab, __half *q_out, __half *k_pages, __half *v_pages) {
   pdl_wait();
   const int m = blockIdx.x, head = blockIdx.y, i = threadIdx.x, half = hd >> 1;
   const int N = (Hq + 2 * Hkv) * hd;
@@ -113,23 +116,23 @@ __global__ void rope_kv_kernel(StepIn in, const float *part, int n_splits, int p
     a = ra; b = rb;
   }
   if (head < Hq) {
-    __nv_bfloat16 *q = q_out + ((size_t)m * Hq + head) * hd;
-    q[i] = __float2bfloat16_rn(a);
-    q[i + half] = __float2bfloat16_rn(b);
+    __half *q = q_out + ((size_t)m * Hq + head) * hd;
+    q[i] = to_half_sat(a);
+    q[i + half] = to_half_sat(b);
   } else {
     const int seq = in.row_seq[m];
     const int page = in.block_tab[(size_t)seq * in.pages_per_seq + (pos >> 4)];
     const bool is_k = head < Hq + Hkv;
     const int kh = is_k ? head - Hq : head - Hq - Hkv;
-    __nv_bfloat16 *dst = (is_k ? k_pages : v_pages) + (((size_t)page * Hkv + kh) * 16 + (pos & 15)) * hd;
-    dst[i] = __float2bfloat16_rn(a);
-    dst[i + half] = __float2bfloat16_rn(b);
+    __half *dst = (is_k ? k_pages : v_pages) + (((size_t)page * Hkv + kh) * 16 + (pos & 15)) * hd;
+    dst[i] = to_half_sat(a);
+    dst[i + half] = to_half_sat(b);
   }
 }
 
 cudaError_t launch_rope_kv(const StepIn &in, const float *part, int n_splits, int part_rows, int Hq, int Hkv,
-                           int hd, const float2 *rope_tab, __nv_bfloat16 *q_out, __nv_bfloat16 *k_pages,
-                           __nv_bfloat16 *v_pages, cudaStream_t st) {
+                           int hd, const float2 *rope_tab, __half *q_out, __half *k_pages, __half *v_pages,
+                           cudaStream_t st) {
   return launch_pdl(rope_kv_kernel, dim3(in.M, Hq + 2 * Hkv), dim3(hd / 2), 0, st, in, part, n_splits,
                     part_rows, Hq, Hkv, hd, rope_tab, q_out, k_pages, v_pages);
 }

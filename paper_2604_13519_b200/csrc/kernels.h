@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda.h>          // CUtensorMap (types only; the driver entry point is resolved at run time)
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -49,16 +50,16 @@ cudaError_t launch_embed_norm(const StepIn &in, const __nv_bfloat16 *embed, cons
 // x[m] += sum_s part[s][m]; h = rmsnorm(x) * gain -> bf16 (hi[, lo])
 cudaError_t launch_add_norm(int M, int d, const float *part, int n_splits, int part_rows, const float *gain,
                             float eps, float *x, __nv_bfloat16 *h, int h_rows, int planes, cudaStream_t st);
-// qkv = sum of split-K partials; rotary on q and k; q -> bf16 [M][Hq][hd]; k, v -> pages
+// qkv = sum of split-K partials; rotary on q and k; q -> fp16 [M][Hq][hd]; k, v -> fp16 pages
 cudaError_t launch_rope_kv(const StepIn &in, const float *part, int n_splits, int part_rows, int Hq, int Hkv,
-                           int hd, const float2 *rope_tab, __nv_bfloat16 *q_out, __nv_bfloat16 *k_pages,
-                           __nv_bfloat16 *v_pages, cudaStream_t st);
+                           int hd, const float2 *rope_tab, __half *q_out, __half *k_pages, __half *v_pages,
+                           cudaStream_t st);
 
 struct AttnArgs {
   StepIn in;
-  const __nv_bfloat16 *q;        // [M][Hq][hd]
-  const __nv_bfloat16 *k_pages;  // [page][Hkv][16][hd]
-  const __nv_bfloat16 *v_pages;
+  const __half *q;               // [M][Hq][hd] rotated queries, fp16
+  const __half *k_pages;         // [page][Hkv][16][hd], fp16
+  const __half *v_pages;
   int Hq, Hkv, hd;
   int n_splits;                  // KV splits per (sequence, kv head, row tile)
   int n_row_tiles_total;         // sum over sequences of row tiles

@@ -45,7 +45,7 @@ struct Layout {
   std::vector<uint64_t> wqkv, wo, wgu, wd, g1, g2;
   uint64_t weights_bytes;
   // kv pool
-  uint64_t kv_layer_stride, kv_v_offset, kv_bytes;   // in bf16 elements / bytes
+  uint64_t kv_layer_stride, kv_v_offset, kv_bytes;   // in fp16 elements / bytes
   // workspace (byte offsets)
   uint64_t x, h, part, q, attn_o, attn_ml, attn, act, logits, amax, rope, d_in, d_out, workspace_bytes;
   // step io (int32 offsets inside d_in / h_in)
@@ -151,6 +151,7 @@ struct ts_model {
   std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_d;
   CUtensorMap tm_lm{}, tm_h[4]{}, tm_attn[4]{}, tm_act[4]{};
   std::vector<int32_t> free_pages;
+  std::vector<ts_session *> sessions;   // live sessions over this model (detached on destroy)
   // last staged step
   int last_B = 0, last_M = 0, last_tiles = 0;
   uint32_t last_flags = 0;
@@ -164,8 +165,8 @@ struct ts_model {
   int32_t *h_out() const { return (int32_t *)b.host_io + L.in_ints; }
   int32_t *d_in() const { return (int32_t *)WS(L.d_in); }
   int32_t *d_out() const { return (int32_t *)WS(L.d_out); }
-  __nv_bfloat16 *k_pages(int l) const { return (__nv_bfloat16 *)b.kv_pool + (uint64_t)l * L.kv_layer_stride; }
-  __nv_bfloat16 *v_pages(int l) const { return k_pages(l) + L.kv_v_offset; }
+  __half *k_pages(int l) const { return (__half *)b.kv_pool + (uint64_t)l * L.kv_layer_stride; }
+  __half *v_pages(int l) const { return k_pages(l) + L.kv_v_offset; }
 };
 
 struct ts_session {
@@ -262,7 +263,7 @@ ts_status run_step(ts_model *m) {
   float *x = (float *)m->WS(L.x);
   __nv_bfloat16 *h = (__nv_bfloat16 *)m->WS(L.h);
   float *part = (float *)m->WS(L.part);
-  __nv_bfloat16 *q = (__nv_bfloat16 *)m->WS(L.q);
+  __half *q = (__half *)m->WS(L.q);
   __nv_bfloat16 *attn = (__nv_bfloat16 *)m->WS(L.attn);
   __nv_bfloat16 *act = (__nv_bfloat16 *)m->WS(L.act);
   const float2 *rope = (const float2 *)m->WS(L.rope);
@@ -518,6 +519,10 @@ ts_status ts_init_model(const ts_model_config *cfg, const ts_buffers *bufs, void
 ts_status ts_model_destroy(ts_model *m) {
   if (!m) return TS_OK;
   cudaStreamSynchronize(m->st);
+  for (ts_session *s : m->sessions) {   // sessions outlive the model as host-only sessions
+    s->m = nullptr;
+    s->pages.clear();
+  }
   delete m;
   return TS_OK;
 }
@@ -635,6 +640,7 @@ ts_status ts_session_create(ts_model *model, const ts_schema *schema, const ts_d
   ts_session *s = new ts_session();
   s->m = model; s->schema = schema; s->store = store; s->cfg = *cfg;
   s->fsm.s = schema;
+  if (model) model->sessions.push_back(s);
   *out = s;
   return TS_OK;
 }
@@ -651,8 +657,11 @@ ts_status ts_session_set_ranks(ts_session *s, const int32_t *ranks, int32_t n) {
 
 ts_status ts_session_destroy(ts_session *s) {
   if (!s) return TS_OK;
-  if (s->m)
+  if (s->m) {
     for (int32_t p : s->pages) s->m->free_pages.push_back(p);
+    auto &v = s->m->sessions;
+    v.erase(std::remove(v.begin(), v.end(), s), v.end());
+  }
   delete s;
   return TS_OK;
 }
@@ -783,7 +792,7 @@ ts_status ts_session_output(const ts_session *s, int32_t *out, int32_t cap, int3
 
 // ---- test / benchmark support -------------------------------------------------------------------------
 static ts_status kv_transfer(ts_model *m, ts_session *s, int layer, void *k, void *v, int n_tokens, bool to_device) {
-  if (!m || !s || !k || !v) return fail(TS_ERR_ARG, "null argument");
+  if (!m || !s || (n_tokens > 0 && (!k || !v))) return fail(TS_ERR_ARG, "null argument");
   if (s->m != m) return fail(TS_ERR_ARG, "session belongs to another model");
   if (layer < 0 || layer >= m->c.n_layers || n_tokens < 0) return fail(TS_ERR_ARG, "bad layer / length");
   if (to_device) {
@@ -794,18 +803,21 @@ static ts_status kv_transfer(ts_model *m, ts_session *s, int layer, void *k, voi
   }
   const int Hkv = m->c.n_kv_heads, hd = m->c.head_dim;
   const size_t page_elems = (size_t)Hkv * TS_PAGE_SIZE * hd;
-  std::vector<uint16_t> stage(page_elems);
+  std::vector<__half> stage(page_elems);
   for (int which = 0; which < 2; ++which) {
-    uint16_t *host = (uint16_t *)(which ? v : k);
-    __nv_bfloat16 *pool = which ? m->v_pages(layer) : m->k_pages(layer);
+    float *host = (float *)(which ? v : k);
+    __half *pool = which ? m->v_pages(layer) : m->k_pages(layer);
     for (int p = 0; p * TS_PAGE_SIZE < n_tokens; ++p) {
       const int t0 = p * TS_PAGE_SIZE, nt = std::min(TS_PAGE_SIZE, n_tokens - t0);
-      __nv_bfloat16 *dev = pool + (size_t)s->pages[p] * page_elems;
+      __half *dev = pool + (size_t)s->pages[p] * page_elems;
       if (to_device) {
-        std::fill(stage.begin(), stage.end(), 0);
+        std::fill(stage.begin(), stage.end(), __float2half(0.f));
         for (int t = 0; t < nt; ++t)
           for (int hh = 0; hh < Hkv; ++hh)
-            std::memcpy(&stage[((size_t)hh * TS_PAGE_SIZE + t) * hd], &host[((size_t)(t0 + t) * Hkv + hh) * hd], hd * 2);
+            for (int e = 0; e < hd; ++e) {
+              const float x = host[((size_t)(t0 + t) * Hkv + hh) * hd + e];
+              stage[((size_t)hh * TS_PAGE_SIZE + t) * hd + e] = __float2half_rn(std::min(std::max(x, -65504.f), 65504.f));
+            }
         CU_TRY(cudaMemcpyAsync(dev, stage.data(), page_elems * 2, cudaMemcpyHostToDevice, m->st));
         CU_TRY(cudaStreamSynchronize(m->st));
       } else {
@@ -813,17 +825,18 @@ static ts_status kv_transfer(ts_model *m, ts_session *s, int layer, void *k, voi
         CU_TRY(cudaStreamSynchronize(m->st));
         for (int t = 0; t < nt; ++t)
           for (int hh = 0; hh < Hkv; ++hh)
-            std::memcpy(&host[((size_t)(t0 + t) * Hkv + hh) * hd], &stage[((size_t)hh * TS_PAGE_SIZE + t) * hd], hd * 2);
+            for (int e = 0; e < hd; ++e)
+              host[((size_t)(t0 + t) * Hkv + hh) * hd + e] = __half2float(stage[((size_t)hh * TS_PAGE_SIZE + t) * hd + e]);
       }
     }
   }
   return TS_OK;
 }
 
-ts_status ts_debug_import_kv(ts_model *m, ts_session *s, int32_t layer, const void *k, const void *v, int32_t n) {
+ts_status ts_debug_import_kv(ts_model *m, ts_session *s, int32_t layer, const float *k, const float *v, int32_t n) {
   return kv_transfer(m, s, layer, (void *)k, (void *)v, n, true);
 }
-ts_status ts_debug_export_kv(ts_model *m, ts_session *s, int32_t layer, void *k, void *v, int32_t n) {
+ts_status ts_debug_export_kv(ts_model *m, ts_session *s, int32_t layer, float *k, float *v, int32_t n) {
   return kv_transfer(m, s, layer, k, v, n, false);
 }
 
