@@ -94,9 +94,10 @@ ts_status ts_init_model(const ts_model_config *cfg, const ts_buffers *bufs, void
 enum { TS_W_EMBED = 0, TS_W_LM_HEAD = 1, TS_W_FINAL_GAIN = 2, TS_W_Q = 3, TS_W_K = 4, TS_W_V = 5,
        TS_W_O = 6, TS_W_GATE = 7, TS_W_UP = 8, TS_W_DOWN = 9, TS_W_GAIN1 = 10, TS_W_GAIN2 = 11 };
 
-/* Upload one tensor.  Matrices are host bf16, row-major [out_features][in_features]; gains are
- * host float32 [d_model].  `layer` is ignored for the three global tensors.  The library lays the
- * matrix out for its kernels (Q,K,V rows concatenated; gate and up rows interleaved).  Synchronous.
+/* Upload one tensor.  Matrices are bf16, row-major [out_features][in_features]; gains are
+ * float32 [d_model]; the source may be host or device memory (the copy direction is inferred).
+ * `layer` is ignored for the three global tensors.  The library lays the matrix out for its
+ * kernels (Q,K,V rows concatenated; gate and up rows interleaved).  Synchronous.
  * Errors: TS_ERR_ARG on a shape that does not match the configuration. */
 ts_status ts_load_tensor(ts_model *m, int32_t kind, int32_t layer, const void *host_data,
                          int64_t rows, int64_t cols);
@@ -181,6 +182,13 @@ ts_status ts_verify(ts_model *m, ts_session *const *sessions, int32_t B,
  * in device memory; no host<->device copy, no synchronisation.  The step is idempotent because
  * sessions advance only in ts_commit.  For timing the kernels alone. */
 ts_status ts_verify_replay(ts_model *m);
+
+/* Run the last step once more with an event after every kernel launch (no overlap between
+ * kernels) and return, per kernel class, the summed milliseconds and the launch count:
+ * 0 projection GEMM, 1 attention, 2 attention merge, 3 norm / residual, 4 rotary + KV append,
+ * 5 acceptance.  n_classes >= 6.  Synchronises the stream.  For the benchmark's roofline line. */
+ts_status ts_profile_step(ts_model *m, float *ms_by_class, int32_t *launches_by_class,
+                          int32_t n_classes);
 
 /* ts_commit — y <- y (+) emitted, q <- delta(q, .) applied id by id (bonus token included), cache
  * length and pending token advanced; stops at the first id that finishes the generation (call

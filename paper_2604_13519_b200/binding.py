@@ -87,6 +87,7 @@ _SIGNATURES = {
     "ts_draft": [_P, C.c_int32, _I32P, _I32P, _I32P],
     "ts_verify": [_P, C.POINTER(_P), C.c_int32, _I32P, _I32P, C.c_uint32, C.POINTER(ts_verify_result)],
     "ts_verify_replay": [_P],
+    "ts_profile_step": [_P, C.POINTER(C.c_float), _I32P, C.c_int32],
     "ts_commit": [_P, C.POINTER(ts_verify_result)],
     "ts_commit_forced": [_P, _I32P, C.c_int32],
     "ts_session_state": [_P, C.POINTER(ts_session_info)],
@@ -351,6 +352,17 @@ def ts_verify(model: Model, sessions: Sequence[Session], drafts: Sequence[Sequen
 
 def ts_verify_replay(model: Model):
     _check(lib().ts_verify_replay(model.h))
+
+
+KERNEL_CLASSES = ("gemm", "attention", "attention_merge", "norm", "rope_kv", "accept")
+
+
+def ts_profile_step(model: Model):
+    """dict class -> (total ms, launches) for one replay of the last step, kernels serialised."""
+    ms = (C.c_float * 8)()
+    n = (C.c_int32 * 8)()
+    _check(lib().ts_profile_step(model.h, ms, n, 8))
+    return {k: (ms[i], n[i]) for i, k in enumerate(KERNEL_CLASSES)}
 
 
 def ts_commit(session: Session, result: ts_verify_result):

@@ -279,7 +279,7 @@ static cudaError_t launch_attn_pdl(K kernel, dim3 grid, dim3 block, size_t smem,
   return cudaLaunchKernelEx(&cfg, kernel, a);
 }
 
-cudaError_t launch_attention(const AttnArgs &a, cudaStream_t st) {
+cudaError_t launch_attention_split(const AttnArgs &a, cudaStream_t st) {
   static bool attr_done = false;
   if (!attr_done) {
     cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -292,9 +292,11 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t st) {
   }
   const dim3 grid(a.n_splits, a.Hkv, a.n_row_tiles_total);
   const size_t smem = (size_t)5 * kBlk * a.hd * 2;
-  cudaError_t e = (a.hd == 128) ? launch_attn_pdl(attn_split_kernel<128>, grid, dim3(128), smem, st, a)
-                                : launch_attn_pdl(attn_split_kernel<64>, grid, dim3(128), smem, st, a);
-  if (e != cudaSuccess) return e;
+  return (a.hd == 128) ? launch_attn_pdl(attn_split_kernel<128>, grid, dim3(128), smem, st, a)
+                       : launch_attn_pdl(attn_split_kernel<64>, grid, dim3(128), smem, st, a);
+}
+
+cudaError_t launch_attention_combine(const AttnArgs &a, cudaStream_t st) {
   return launch_attn_pdl(attn_combine_kernel, dim3(a.in.M, a.Hq), dim3(a.hd), 0, st, a);
 }
 

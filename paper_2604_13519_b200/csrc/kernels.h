@@ -70,7 +70,8 @@ struct AttnArgs {
   __nv_bfloat16 *out;            // [planes][out_rows][Hq*hd]
   int out_rows, planes;
 };
-cudaError_t launch_attention(const AttnArgs &a, cudaStream_t st);
+cudaError_t launch_attention_split(const AttnArgs &a, cudaStream_t st);
+cudaError_t launch_attention_combine(const AttnArgs &a, cudaStream_t st);
 
 // per-row argmax over the LM-head tiles, longest accepted prefix per sequence, new lengths
 struct AcceptArgs {

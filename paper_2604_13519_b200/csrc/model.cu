@@ -158,6 +158,21 @@ struct ts_model {
   bool have_step = false;
   int64_t launches = 0, h2d = 0, d2h = 0;
   bool use_pdl = true;
+  // per-kernel timing pass (ts_profile_step): one event after every launch
+  bool profiling = false;
+  std::vector<cudaEvent_t> prof_ev;
+  std::vector<int> prof_cls;
+  void launched(int cls) {
+    ++launches;
+    if (profiling) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) == cudaSuccess) {
+        cudaEventRecord(e, st);
+        prof_ev.push_back(e);
+        prof_cls.push_back(cls);
+      }
+    }
+  }
 
   uint8_t *W(uint64_t off) const { return (uint8_t *)b.weights + off; }
   uint8_t *WS(uint64_t off) const { return (uint8_t *)b.workspace + off; }
@@ -245,8 +260,8 @@ ts_status run_gemm(ts_model *m, int epi, const CUtensorMap &tw, const CUtensorMa
   g.amax = amax;
   g.err = m->d_out() + m->L.o_err;
   if (plan) { plan->splits = splits; plan->kb_per_split = g.kb_per_split; }
-  CU_TRY(ts::launch_gemm(epi, tw, ta4[mi], g, splits, m->gemm_smem_budget, m->st, m->use_pdl));
-  ++m->launches;
+  CU_TRY(ts::launch_gemm(epi, tw, ta4[mi], g, splits, m->gemm_smem_budget, m->st, m->use_pdl && !m->profiling));
+  m->launched(0);
   return TS_OK;
 }
 
@@ -288,27 +303,29 @@ ts_status run_step(ts_model *m) {
 
   CU_TRY(ts::launch_embed_norm(in, (const __nv_bfloat16 *)m->W(L.embed), (const float *)m->W(L.g1[0]), c.rms_eps,
                                d, x, h, R, m->planes, m->st));
-  ++m->launches;
+  m->launched(3);
   GemmPlan plan{};
   for (int l = 0; l < c.n_layers; ++l) {
     if (l > 0) {
       CU_TRY(ts::launch_add_norm(M, d, part, plan.splits, R, (const float *)m->W(L.g1[l]), c.rms_eps, x, h, R,
                                  m->planes, m->st));
-      ++m->launches;
+      m->launched(3);
     }
     ts_status s = run_gemm(m, ts::EPI_PARTIAL, m->tm_qkv[l], m->tm_h, L.Nqkv, d, M, part, nullptr, nullptr, &plan);
     if (s) return s;
     CU_TRY(ts::launch_rope_kv(in, part, plan.splits, R, c.n_q_heads, c.n_kv_heads, c.head_dim, rope, q,
                               m->k_pages(l), m->v_pages(l), m->st));
-    ++m->launches;
+    m->launched(4);
     aa.k_pages = m->k_pages(l); aa.v_pages = m->v_pages(l);
-    CU_TRY(ts::launch_attention(aa, m->st));
-    m->launches += 2;
+    CU_TRY(ts::launch_attention_split(aa, m->st));
+    m->launched(1);
+    CU_TRY(ts::launch_attention_combine(aa, m->st));
+    m->launched(2);
     s = run_gemm(m, ts::EPI_PARTIAL, m->tm_o[l], m->tm_attn, d, Nq, M, part, nullptr, nullptr, &plan);
     if (s) return s;
     CU_TRY(ts::launch_add_norm(M, d, part, plan.splits, R, (const float *)m->W(L.g2[l]), c.rms_eps, x, h, R,
                                m->planes, m->st));
-    ++m->launches;
+    m->launched(3);
     s = run_gemm(m, ts::EPI_SWIGLU, m->tm_gu[l], m->tm_h, 2 * F, d, M, nullptr, act, nullptr, nullptr);
     if (s) return s;
     s = run_gemm(m, ts::EPI_PARTIAL, m->tm_d[l], m->tm_act, d, F, M, part, nullptr, nullptr, &plan);
@@ -317,7 +334,7 @@ ts_status run_step(ts_model *m) {
   if (m->last_flags & TS_FLAG_SKIP_LM_HEAD) return TS_OK;
   CU_TRY(ts::launch_add_norm(M, d, part, plan.splits, R, (const float *)m->W(L.gf), c.rms_eps, x, h, R, m->planes,
                              m->st));
-  ++m->launches;
+  m->launched(3);
   float2 *amax = (float2 *)m->WS(L.amax);
   ts_status s = run_gemm(m, ts::EPI_LOGITS, m->tm_lm, m->tm_h, c.vocab, d, M, (float *)m->WS(L.logits), nullptr,
                          amax, nullptr);
@@ -328,7 +345,7 @@ ts_status run_step(ts_model *m) {
   ac.argmax = dout + L.o_argmax; ac.accept_len = dout + L.o_accept; ac.emitted = dout + L.o_emitted;
   ac.new_len = dout + L.o_newlen; ac.new_pending = dout + L.o_newpend; ac.k_max = c.k_max;
   CU_TRY(ts::launch_accept(ac, m->st));
-  ++m->launches;
+  m->launched(5);
   return TS_OK;
 }
 
@@ -556,7 +573,7 @@ ts_status ts_load_tensor(ts_model *m, int32_t kind, int32_t layer, const void *h
                                             (long long)er, (long long)ec, (long long)rows, (long long)cols);
   const size_t row_bytes = (size_t)ec * esz;
   if (dpitch == 0) dpitch = row_bytes;
-  CU_TRY(cudaMemcpy2DAsync(dst, dpitch, host, row_bytes, row_bytes, (size_t)er, cudaMemcpyHostToDevice, m->st));
+  CU_TRY(cudaMemcpy2DAsync(dst, dpitch, host, row_bytes, row_bytes, (size_t)er, cudaMemcpyDefault, m->st));
   CU_TRY(cudaStreamSynchronize(m->st));
   return TS_OK;
 }
@@ -756,6 +773,35 @@ ts_status ts_verify_replay(ts_model *m) {
   if (!m) return fail(TS_ERR_ARG, "null argument");
   if (!m->have_step) return fail(TS_ERR_STATE, "no step has been staged yet");
   return run_step(m);
+}
+
+ts_status ts_profile_step(ts_model *m, float *ms_by_class, int32_t *launches_by_class, int32_t n_classes) {
+  if (!m || !ms_by_class || !launches_by_class || n_classes < 6) return fail(TS_ERR_ARG, "bad argument");
+  if (!m->have_step) return fail(TS_ERR_STATE, "no step has been staged yet");
+  for (int i = 0; i < n_classes; ++i) { ms_by_class[i] = 0.f; launches_by_class[i] = 0; }
+  cudaEvent_t start;
+  CU_TRY(cudaEventCreate(&start));
+  CU_TRY(cudaEventRecord(start, m->st));
+  m->profiling = true;
+  ts_status st = run_step(m);
+  m->profiling = false;
+  cudaError_t e = cudaStreamSynchronize(m->st);
+  cudaEvent_t prev = start;
+  for (size_t i = 0; i < m->prof_ev.size(); ++i) {
+    float ms = 0.f;
+    if (e == cudaSuccess && cudaEventElapsedTime(&ms, prev, m->prof_ev[i]) == cudaSuccess) {
+      ms_by_class[m->prof_cls[i]] += ms;
+      ++launches_by_class[m->prof_cls[i]];
+    }
+    prev = m->prof_ev[i];
+  }
+  cudaEventDestroy(start);
+  for (cudaEvent_t ev : m->prof_ev) cudaEventDestroy(ev);
+  m->prof_ev.clear();
+  m->prof_cls.clear();
+  if (st) return st;
+  if (e != cudaSuccess) return fail(TS_ERR_CUDA, "profile step: %s", cudaGetErrorString(e));
+  return TS_OK;
 }
 
 ts_status ts_commit_forced(ts_session *s, const int32_t *emitted, int32_t n) {
