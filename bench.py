@@ -35,6 +35,8 @@ WORKLOADS = {
     "c3_8b_ctx8192_k16": ("8b", [8192], [16]),
     "c3_8b_ctx8192_k32": ("8b", [8192], [32]),
     "c5_8b_b4_ctx8192_k64": ("8b", [8192] * 4, [64] * 4),
+    # reduced-depth case for profiler captures (same per-layer kernels and grids as c3)
+    "prof_8b4l_ctx8192_k32": ("8b-4l", [8192], [32]),
 }
 DEFAULT_WORKLOAD = "c3_8b_ctx8192_k32"
 METRIC = "verified_tokens_per_s"

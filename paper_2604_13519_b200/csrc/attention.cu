@@ -235,29 +235,43 @@ attn_split_kernel(const AttnArgs a) {
   }
 }
 
-// grid = (M, Hq), hd threads: merge the splits of one (row, query head).
+// grid = (M, Hq), hd threads: merge the splits of one (row, query head).  The first warp turns the
+// splits' (max, sum) pairs into normalised weights in shared memory; every thread then sums its
+// output element over the splits with independent loads.
 __global__ void attn_combine_kernel(const AttnArgs a) {
+  __shared__ float w_s[64];
   pdl_wait();
   const int m = blockIdx.x, h = blockIdx.y, d = threadIdx.x;
   const size_t base = ((size_t)m * a.Hq + h) * a.n_splits;
-  float mx = -INFINITY;
-  for (int s = 0; s < a.n_splits; ++s) {
-    const float2 ml = a.part_ml[base + s];
-    if (ml.y > 0.f) mx = fmaxf(mx, ml.x);
-  }
-  float num = 0.f, den = 0.f;
-  for (int s = 0; s < a.n_splits; ++s) {
-    const float2 ml = a.part_ml[base + s];
-    if (ml.y > 0.f) {
-      const float w = exp2f(ml.x - mx);
-      den += w * ml.y;
-      num += w * a.part_o[(base + s) * a.hd + d];
+  if (threadIdx.x < 32) {
+    float mx = -INFINITY;
+    for (int s = threadIdx.x; s < a.n_splits; s += 32) {
+      const float2 ml = a.part_ml[base + s];
+      if (ml.y > 0.f) mx = fmaxf(mx, ml.x);
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float den = 0.f;
+    for (int s = threadIdx.x; s < a.n_splits; s += 32) {
+      const float2 ml = a.part_ml[base + s];
+      const float w = ml.y > 0.f ? exp2f(ml.x - mx) : 0.f;
+      w_s[s] = w;
+      den += w * ml.y;
+    }
+    den = warp_sum(den);
+    const float inv = 1.f / den;
+    for (int s = threadIdx.x; s < a.n_splits; s += 32) w_s[s] *= inv;
   }
+  __syncthreads();
   pdl_launch_dependents();
-  const float v = num / den;
+  float num = 0.f;
+#pragma unroll 8
+  for (int s = 0; s < a.n_splits; ++s) {
+    const float w = w_s[s];
+    if (w != 0.f) num += w * a.part_o[(base + s) * a.hd + d];
+  }
   __nv_bfloat16 hi, lo;
-  split_bf16(v, hi, lo);
+  split_bf16(num, hi, lo);
   const size_t col = (size_t)h * a.hd + d;
   const size_t ld = (size_t)a.Hq * a.hd;
   a.out[(size_t)m * ld + col] = hi;

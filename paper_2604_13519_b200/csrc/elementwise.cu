@@ -1,34 +1,41 @@
 // Memory-light kernels of the verify step: embedding gather + RMSNorm, residual add + RMSNorm (which
 // also folds the split-K partial sums of the preceding projection), rotary embedding + paged KV
 // append, and the acceptance kernel (per-row argmax, longest accepted draft prefix, new lengths).
+#include <algorithm>
+
 #include "kernels.h"
 
 namespace ts {
 
-static constexpr int kNormThreads = 256;
+static constexpr int kNormMaxThreads = 1024;
+static constexpr int kNormMaxSplits = 12;   // split-K slabs folded in one pass (the GEMM launcher's cap)
 
 __device__ __forceinline__ float block_sum(float v, float *red) {
   v = warp_sum(v);
   const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
   if (l == 0) red[w] = v;
   __syncthreads();
-  float t = (l < (int)(blockDim.x >> 5)) ? red[l] : 0.f;
+  float t = (l < (int)((blockDim.x + 31) >> 5)) ? red[l] : 0.f;
   t = warp_sum(t);
   __syncthreads();
   return t;
 }
 
-// One CTA per row.  MODE 0: x = embedding row.  MODE 1: x += sum of partial slabs.
+// One CTA per row, one float4 of the row per thread and pass (d/4 threads, at most 1024), so that the
+// loads of all split-K slabs are in flight together.  MODE 0: x = embedding row (and the row's argmax
+// slot is cleared for the LM-head epilogue).  MODE 1: x += sum of partial slabs.
 template <int MODE>
-__global__ void __launch_bounds__(kNormThreads)
+__global__ void __launch_bounds__(kNormMaxThreads)
 norm_kernel(const int32_t *tokens, const __nv_bfloat16 *embed, const float *part, int n_splits, int part_rows,
-            const float *gain, float eps, int d, float *x, __nv_bfloat16 *h, int h_rows, int planes) {
+            const float *gain, float eps, int d, float *x, __nv_bfloat16 *h, int h_rows, int planes,
+            unsigned long long *amax) {
   __shared__ float red[32];
   pdl_wait();
   const int m = blockIdx.x;
   float *xr = x + (size_t)m * d;
   float ss = 0.f;
-  for (int c = threadIdx.x * 4; c < d; c += kNormThreads * 4) {
+  if (MODE == 0 && threadIdx.x == 0) amax[m] = 0ull;
+  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
     float4 v;
     if (MODE == 0) {
       const __nv_bfloat16 *e = embed + (size_t)tokens[m] * d + c;
@@ -38,9 +45,16 @@ norm_kernel(const int32_t *tokens, const __nv_bfloat16 *embed, const float *part
       v = make_float4(__low2float(a), __high2float(a), __low2float(b), __high2float(b));
     } else {
       v = *reinterpret_cast<const float4 *>(xr + c);
-      for (int s = 0; s < n_splits; ++s) {
-        const float4 p = *reinterpret_cast<const float4 *>(part + ((size_t)s * part_rows + m) * d + c);
-        v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+      // two batches of six independent loads (a 1024-thread CTA has 64 registers per thread)
+#pragma unroll
+      for (int s0 = 0; s0 < kNormMaxSplits; s0 += 6) {
+        float4 p[6];
+#pragma unroll
+        for (int s = 0; s < 6; ++s)
+          if (s0 + s < n_splits) p[s] = *reinterpret_cast<const float4 *>(part + ((size_t)(s0 + s) * part_rows + m) * d + c);
+#pragma unroll
+        for (int s = 0; s < 6; ++s)
+          if (s0 + s < n_splits) { v.x += p[s].x; v.y += p[s].y; v.z += p[s].z; v.w += p[s].w; }
       }
     }
     *reinterpret_cast<float4 *>(xr + c) = v;
@@ -49,7 +63,7 @@ norm_kernel(const int32_t *tokens, const __nv_bfloat16 *embed, const float *part
   const float tot = block_sum(ss, red);
   const float r = rsqrtf(tot / (float)d + eps);
   pdl_launch_dependents();
-  for (int c = threadIdx.x * 4; c < d; c += kNormThreads * 4) {
+  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
     const float4 v = *reinterpret_cast<const float4 *>(xr + c);
     const float4 gn = *reinterpret_cast<const float4 *>(gain + c);
     const float o[4] = {v.x * r * gn.x, v.y * r * gn.y, v.z * r * gn.z, v.w * r * gn.w};
@@ -76,17 +90,21 @@ static cudaError_t launch_pdl(K kernel, dim3 grid, dim3 block, size_t smem, cuda
   return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
+static int norm_threads(int d) { return std::min(kNormMaxThreads, (d / 4 + 31) / 32 * 32); }
+
 cudaError_t launch_embed_norm(const StepIn &in, const __nv_bfloat16 *embed, const float *gain, float eps,
-                              int d, float *x, __nv_bfloat16 *h, int h_rows, int planes, cudaStream_t st) {
-  return launch_pdl(norm_kernel<0>, dim3(in.M), dim3(kNormThreads), 0, st, in.tokens, embed,
-                    (const float *)nullptr, 0, 0, gain, eps, d, x, h, h_rows, planes);
+                              int d, float *x, __nv_bfloat16 *h, int h_rows, int planes,
+                              unsigned long long *amax, cudaStream_t st) {
+  return launch_pdl(norm_kernel<0>, dim3(in.M), dim3(norm_threads(d)), 0, st, in.tokens, embed,
+                    (const float *)nullptr, 0, 0, gain, eps, d, x, h, h_rows, planes, amax);
 }
 
 cudaError_t launch_add_norm(int M, int d, const float *part, int n_splits, int part_rows, const float *gain,
                             float eps, float *x, __nv_bfloat16 *h, int h_rows, int planes, cudaStream_t st) {
-  return launch_pdl(norm_kernel<1>, dim3(M), dim3(kNormThreads), 0, st, (const int32_t *)nullptr,
+  if (n_splits > kNormMaxSplits) return cudaErrorInvalidValue;
+  return launch_pdl(norm_kernel<1>, dim3(M), dim3(norm_threads(d)), 0, st, (const int32_t *)nullptr,
                     (const __nv_bfloat16 *)nullptr, part, n_splits, part_rows, gain, eps, d, x, h, h_rows,
-                    planes);
+                    planes, (unsigned long long *)nullptr);
 }
 
 __device__ __forceinline__ __half to_half_sat(float x) {
@@ -137,32 +155,17 @@ cudaError_t launch_rope_kv(const StepIn &in, const float *part, int n_splits, in
                     part_rows, Hq, Hkv, hd, rope_tab, q_out, k_pages, v_pages);
 }
 
-// One CTA per sequence.  Step 1: every warp reduces the per-tile maxima of some rows to the row's
-// argmax (lowest id among equal maxima).  Step 2: thread 0 walks the draft: row j predicted the
-// token that row j+1 was fed; the accepted length is the number of leading agreements.
-__global__ void __launch_bounds__(256)
+// One CTA per sequence.  Each row's argmax was reduced by the LM-head epilogue into a packed
+// (ordered value bits, ~token id) word, so the largest word is the largest logit with the lowest id.
+// Thread 0 then walks the draft: row j predicted the token that row j+1 was fed; the accepted length
+// is the number of leading agreements.
+__global__ void __launch_bounds__(64)
 accept_kernel(AcceptArgs a) {
   pdl_wait();
   const int seq = blockIdx.x;
   const int r0 = a.in.cu_rows[seq], r1 = a.in.cu_rows[seq + 1];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int r = r0 + warp; r < r1; r += 8) {
-    float bv = -INFINITY;
-    int bi = 0x7fffffff;
-    const float2 *p = a.amax + (size_t)r * a.n_part;
-    for (int t = lane; t < a.n_part; t += 32) {
-      const float2 e = p[t];
-      const int idx = __float_as_int(e.y);
-      if (e.x > bv || (e.x == bv && idx < bi)) { bv = e.x; bi = idx; }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-    }
-    if (lane == 0) a.argmax[r] = bi;
-  }
+  for (int r = r0 + threadIdx.x; r < r1; r += blockDim.x)
+    a.argmax[r] = (int32_t)(0xFFFFFFFFu - (uint32_t)(a.amax[r] & 0xFFFFFFFFull));
   __syncthreads();
   if (threadIdx.x == 0) {
     const int k = r1 - r0;
@@ -178,7 +181,7 @@ accept_kernel(AcceptArgs a) {
 }
 
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t st) {
-  return launch_pdl(accept_kernel, dim3(a.in.B), dim3(256), 0, st, a);
+  return launch_pdl(accept_kernel, dim3(a.in.B), dim3(64), 0, st, a);
 }
 
 }  // namespace ts

@@ -178,8 +178,12 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
               int oi = __shfl_xor_sync(0xffffffffu, bi, o);
               if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
             }
-            if (lane == 0 && m < g.M)
-              g.amax[(size_t)m * (gridDim.x * 4) + blockIdx.x * 4 + q] = make_float2(bv, __int_as_float(bi));
+            if (lane == 0 && m < g.M) {
+              // order-preserving map of the float to an unsigned word; ties resolve to the lowest id
+              uint32_t u = __float_as_uint(bv);
+              u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+              atomicMax(g.amax + m, ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)bi));
+            }
           }
         } else {  // EPI_SWIGLU: even feature row = gate_f, odd = up_f, f = n / 2
           const int f = n >> 1;

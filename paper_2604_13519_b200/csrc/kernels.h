@@ -24,7 +24,7 @@ struct GemmArgs {
   __nv_bfloat16 *act_out;  // EPI_SWIGLU: [out_planes][act_rows][N/2]
   int act_rows;
   int out_planes;
-  float2 *amax;         // EPI_LOGITS: [M][tiles*4] (max value, index bits)
+  unsigned long long *amax;  // EPI_LOGITS: [M] packed (ordered logit bits << 32 | ~token id), atomicMax
   int *err;             // device status word
 };
 
@@ -46,7 +46,8 @@ struct StepIn {
 
 // x[m] = E[tokens[m]]; h = rmsnorm(x) * gain -> bf16 (hi[, lo])
 cudaError_t launch_embed_norm(const StepIn &in, const __nv_bfloat16 *embed, const float *gain, float eps,
-                              int d, float *x, __nv_bfloat16 *h, int h_rows, int planes, cudaStream_t st);
+                              int d, float *x, __nv_bfloat16 *h, int h_rows, int planes,
+                              unsigned long long *amax, cudaStream_t st);
 // x[m] += sum_s part[s][m]; h = rmsnorm(x) * gain -> bf16 (hi[, lo])
 cudaError_t launch_add_norm(int M, int d, const float *part, int n_splits, int part_rows, const float *gain,
                             float eps, float *x, __nv_bfloat16 *h, int h_rows, int planes, cudaStream_t st);
@@ -76,8 +77,7 @@ cudaError_t launch_attention_combine(const AttnArgs &a, cudaStream_t st);
 // per-row argmax over the LM-head tiles, longest accepted prefix per sequence, new lengths
 struct AcceptArgs {
   StepIn in;
-  const float2 *amax;      // [M][n_part]
-  int n_part;
+  const unsigned long long *amax;   // [M] packed per-row maxima written by the LM-head epilogue
   int32_t *argmax;         // [M]
   int32_t *accept_len;     // [B]
   int32_t *emitted;        // [B][k_max]

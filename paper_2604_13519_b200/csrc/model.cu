@@ -115,7 +115,7 @@ void make_layout(const ts_model_config &c, Layout *L) {
   L->attn = take(planes * R * Nq * 2);
   L->act = take(planes * R * F * 2);
   L->logits = take(R * V * 4);
-  L->amax = take(R * (uint64_t)L->n_vocab_tiles * 4 * 8);
+  L->amax = take(R * 8);
   L->rope = take((uint64_t)c.max_ctx * (hd / 2) * 8);
   int io = 0;
   auto itake = [&](int n) { int r = io; io += (n + 3) / 4 * 4; return r; };
@@ -246,7 +246,7 @@ int pick_splits(const ts_model *m, int n_tiles, int m_chunks, int n_kblocks, boo
 struct GemmPlan { int splits, kb_per_split; };
 
 ts_status run_gemm(ts_model *m, int epi, const CUtensorMap &tw, const CUtensorMap *ta4, int N, int K, int M,
-                   float *out, __nv_bfloat16 *act_out, float2 *amax, GemmPlan *plan) {
+                   float *out, __nv_bfloat16 *act_out, unsigned long long *amax, GemmPlan *plan) {
   const int mi = pick_mc_index(M);
   ts::GemmArgs g{};
   g.N = N; g.K = K; g.M = M; g.Mc = kMcOptions[mi]; g.planes = m->planes;
@@ -302,7 +302,7 @@ ts_status run_step(ts_model *m) {
   }
 
   CU_TRY(ts::launch_embed_norm(in, (const __nv_bfloat16 *)m->W(L.embed), (const float *)m->W(L.g1[0]), c.rms_eps,
-                               d, x, h, R, m->planes, m->st));
+                               d, x, h, R, m->planes, (unsigned long long *)m->WS(L.amax), m->st));
   m->launched(3);
   GemmPlan plan{};
   for (int l = 0; l < c.n_layers; ++l) {
@@ -335,13 +335,13 @@ ts_status run_step(ts_model *m) {
   CU_TRY(ts::launch_add_norm(M, d, part, plan.splits, R, (const float *)m->W(L.gf), c.rms_eps, x, h, R, m->planes,
                              m->st));
   m->launched(3);
-  float2 *amax = (float2 *)m->WS(L.amax);
+  unsigned long long *amax = (unsigned long long *)m->WS(L.amax);
   ts_status s = run_gemm(m, ts::EPI_LOGITS, m->tm_lm, m->tm_h, c.vocab, d, M, (float *)m->WS(L.logits), nullptr,
                          amax, nullptr);
   if (s) return s;
   ts::AcceptArgs ac{};
   int32_t *dout = m->d_out();
-  ac.in = in; ac.amax = amax; ac.n_part = L.n_vocab_tiles * 4;
+  ac.in = in; ac.amax = amax;
   ac.argmax = dout + L.o_argmax; ac.accept_len = dout + L.o_accept; ac.emitted = dout + L.o_emitted;
   ac.new_len = dout + L.o_newlen; ac.new_pending = dout + L.o_newpend; ac.k_max = c.k_max;
   CU_TRY(ts::launch_accept(ac, m->st));

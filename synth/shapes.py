@@ -38,4 +38,6 @@ SHAPES = {
     # smaller vocabulary, so that a CPU check of a whole forward finishes in seconds
     "1b-2l": ModelShape("1b-2l", 2, 2048, 32, 8, 64, 8192, 8192, 500000.0, 1e-5),
     "8b-2l": ModelShape("8b-2l", 2, 4096, 32, 8, 128, 12288, 8192, 1000000.0, 1e-6),
+    # the 8B layer at four layers and a 32k vocabulary: a few GB on the device, for profiler captures
+    "8b-4l": ModelShape("8b-4l", 4, 4096, 32, 8, 128, 12288, 32768, 1000000.0, 1e-6),
 }
