@@ -233,6 +233,55 @@ ts_status ts_debug_read_buffer(ts_model *m, int32_t which, void *host_out, uint6
 ts_status ts_model_counters(const ts_model *m, int64_t *launches, int64_t *h2d_bytes,
                             int64_t *d2h_bytes);
 
+/* ---- attention without device allocation -------------------------------------------------------- */
+/* The paper has no counterpart to this call; it exists for deployment reasons only.
+ *
+ * Some hosts of this library are not allowed to obtain device memory themselves: a plugin inside
+ * a serving process whose memory pool is owned (and fully reserved) by the host application, a
+ * callback that runs where cudaMalloc is forbidden, or a process working under a fixed memory
+ * budget.  Such a caller cannot size and allocate the workspace that ts_init_model needs.
+ * ts_attention_static runs the attention stage of the verify step (rows of the chunk against the
+ * paged cache plus the chunk itself, causal inside the chunk; the same two kernels ts_verify uses)
+ * with all of its scratch memory (per-split partial outputs, their running max / sum, the
+ * row-tile table) in a fixed array of TS_STATIC_ATTN_SCRATCH_MIB MiB (plus about 0.5 MiB of
+ * bookkeeping) that is part of the library image.  Every GPU on which the library is loaded
+ * holds that array until the process exits.  The call itself allocates nothing, on the host
+ * heap or on the device.
+ *
+ * Arguments: the *_host arrays are read on the host during the call; everything else is device
+ * memory owned by the caller and must stay valid until the stream has run the work.
+ *   q            fp16 [rows][n_q_heads][head_dim], rotary already applied, rows = cu_rows[batch]
+ *   k_pages,
+ *   v_pages      fp16 [page][n_kv_heads][TS_PAGE_SIZE][head_dim]; must already hold the chunk rows
+ *   block_table  int32 [batch][pages_per_seq]: page ids of each sequence, in position order
+ *   cu_rows      int32 [batch+1] row offsets (cu_rows[0] = 0), on the device and on the host
+ *   seq_len      int32 [batch] tokens in the cache before the chunk, on the device and on the host
+ *   out          bf16 [planes][out_rows][n_q_heads*head_dim]: plane 0 the rounded result, plane 1
+ *                (planes = 2) the rounding remainder, as the output projection consumes them
+ * Limits: head_dim 64 or 128; at most TS_K_MAX rows per sequence; rows * n_q_heads * head_dim * 4
+ * bytes must fit the scratch array (the number of KV splits is lowered to fit before that);
+ * at most 512 row tiles of 64 packed rows.  Beyond them the call fails with TS_ERR_K_TOO_LARGE
+ * and a message naming the limit; nothing is launched.
+ * First use: the first call on each device looks up the array's device address (that device
+ * must be current) and keeps it; make that first call outside any stream capture.
+ * Sharing: every call on a device uses the same array, which keeps whatever the previous call
+ * left there.  No part of it has to start at zero: each call writes every word it later reads.
+ * Two calls whose kernels overlap on the GPU (different streams, no ordering between them) race
+ * on the array and both results are undefined; order them on one stream or with events.
+ * Asynchronous: work is enqueued on `stream` (a cudaStream_t, 0 = default); errors found later
+ * surface through the stream as usual.  Errors: TS_ERR_ARG, TS_ERR_K_TOO_LARGE, TS_ERR_CUDA. */
+#define TS_STATIC_ATTN_SCRATCH_MIB 16
+typedef struct {
+  int32_t n_q_heads, n_kv_heads, head_dim;
+  int32_t batch, pages_per_seq;
+  int32_t out_rows, planes;
+  const int32_t *cu_rows_host, *seq_len_host;        /* host */
+  const int32_t *cu_rows, *seq_len, *block_table;    /* device */
+  const void *q, *k_pages, *v_pages;                 /* device */
+  void *out;                                         /* device */
+} ts_attention_args;
+ts_status ts_attention_static(const ts_attention_args *a, void *stream);
+
 const char *ts_last_error(void);
 
 #ifdef __cplusplus

@@ -69,6 +69,15 @@ class ts_session_info(C.Structure):
 
 _P = C.c_void_p
 _I32P = C.POINTER(C.c_int32)
+
+
+class ts_attention_args(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_q_heads", "n_kv_heads", "head_dim", "batch", "pages_per_seq",
+                                         "out_rows", "planes")] + \
+               [("cu_rows_host", _I32P), ("seq_len_host", _I32P)] + \
+               [(n, _P) for n in ("cu_rows", "seq_len", "block_table", "q", "k_pages", "v_pages", "out")]
+
+
 _SIGNATURES = {
     "ts_query_buffer_sizes": [C.POINTER(ts_model_config), C.POINTER(ts_buffer_sizes)],
     "ts_init_model": [C.POINTER(ts_model_config), C.POINTER(ts_buffers), _P, C.POINTER(_P)],
@@ -98,6 +107,7 @@ _SIGNATURES = {
     "ts_read_logits": [_P, C.c_int32, C.c_int32, C.POINTER(C.c_float)],
     "ts_debug_read_buffer": [_P, C.c_int32, _P, C.c_uint64],
     "ts_model_counters": [_P, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64)],
+    "ts_attention_static": [C.POINTER(ts_attention_args), _P],
 }
 EXPORTED = sorted(list(_SIGNATURES) + ["ts_last_error"])
 
@@ -371,3 +381,26 @@ def ts_commit(session: Session, result: ts_verify_result):
 
 def ts_commit_forced(session: Session, emitted: Sequence[int]):
     _check(lib().ts_commit_forced(session.h, _i32(emitted), len(emitted)))
+
+
+def ts_attention_static(q, k_pages, v_pages, block_table, cu_rows: Sequence[int], seq_len: Sequence[int],
+                        n_q_heads: int, n_kv_heads: int, head_dim: int, out, stream=None):
+    """Attention stage of the verify step with library-resident scratch (no device allocation in the
+    call).  q, k_pages, v_pages: CUDA fp16 tensors; block_table: CUDA int32 [batch][pages_per_seq];
+    cu_rows / seq_len: Python ints (uploaded here as the device copies the call also needs);
+    out: CUDA bf16 tensor [planes][out_rows][n_q_heads*head_dim], written in place."""
+    import torch
+    B = len(seq_len)
+    a = ts_attention_args()
+    a.n_q_heads, a.n_kv_heads, a.head_dim = n_q_heads, n_kv_heads, head_dim
+    a.batch, a.pages_per_seq = B, block_table.shape[1]
+    a.planes, a.out_rows = out.shape[0], out.shape[1]
+    h_cu, h_len = _i32(cu_rows), _i32(seq_len)
+    d_cu = torch.tensor(list(cu_rows), dtype=torch.int32, device=q.device)
+    d_len = torch.tensor(list(seq_len), dtype=torch.int32, device=q.device)
+    a.cu_rows_host, a.seq_len_host = h_cu, h_len
+    a.cu_rows, a.seq_len, a.block_table = d_cu.data_ptr(), d_len.data_ptr(), block_table.data_ptr()
+    a.q, a.k_pages, a.v_pages, a.out = q.data_ptr(), k_pages.data_ptr(), v_pages.data_ptr(), out.data_ptr()
+    sp = stream.cuda_stream if stream is not None else torch.cuda.current_stream().cuda_stream
+    _check(lib().ts_attention_static(C.byref(a), _P(sp)))
+    return d_cu, d_len      # keep the device copies alive until the caller has synchronised

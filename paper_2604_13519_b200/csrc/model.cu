@@ -141,6 +141,19 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 
 }  // namespace
 
+namespace ts {
+// records the thread's last error text for entry points that live in other translation units
+ts_status set_error(ts_status code, const char *fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  g_err = buf;
+  return code;
+}
+}  // namespace ts
+
 struct ts_model {
   ts_model_config c{};
   ts_buffers b{};
