@@ -44,6 +44,8 @@ UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the projection GEMM, from the ncu
 # capture summarised under profiles/ (None until a capture exists)
 GEMM_TRAFFIC_BYTES_PER_LAUNCH = None
+# the same for one launch of the persistent kernel on the default workload
+FUSED_TRAFFIC_BYTES_PER_LAUNCH = None
 
 
 def c4_workload():
@@ -161,7 +163,7 @@ def max_over_ranks(value_ms: float, world: int, backend_device=None) -> float:
     return float(t[0])
 
 
-def build_gpu_model(shape, lens, ks, act_split=True):
+def build_gpu_model(shape, lens, ks, act_split=True, path=0):
     """Random-init weights generated on the device (N(0, 0.02) rounded to bf16, gains one) and a KV
     pool filled with N(0,1) fp16 values; sessions placed at their context lengths."""
     import torch
@@ -171,7 +173,7 @@ def build_gpu_model(shape, lens, ks, act_split=True):
     max_ctx = max(lens) + 2 * k_max
     pages = sum((n + 2 * k_max + 15) // 16 for n in lens) + 8
     m = ts.Model(shape, max_pages=pages, max_batch=B_, k_max=k_max, max_rows=max(sum(ks), k_max),
-                 max_ctx=max_ctx, act_split=act_split)
+                 max_ctx=max_ctx, act_split=act_split, path=path)
     g = torch.Generator(device="cuda").manual_seed(260413519)
     s = shape
 
@@ -271,6 +273,7 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the latency-vs-k sweep")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-act-split", action="store_true")
+    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 one kernel per stage, 2 single persistent kernel")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -292,7 +295,7 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     ts.binding.lib()
     planes = 1 if args.no_act_split else 2
-    model, sessions = build_gpu_model(shape, lens, ks, act_split=not args.no_act_split)
+    model, sessions = build_gpu_model(shape, lens, ks, act_split=not args.no_act_split, path=args.path)
     M = sum(ks)
     drafts = [[64 + (7 * j + i) % (shape.vocab - 64) for j in range(k - 1)] for i, k in enumerate(ks)]
     stream = torch.cuda.current_stream()
@@ -352,16 +355,27 @@ def main():
     peaks = measured_peaks()
     ab = algorithmic_bytes(shape, lens, ks)
     fl = algorithmic_flops(shape, lens, ks)
-    gemm_bytes, gemm_launches = gemm_bytes_per_step(shape, M, planes)
-    gemm_ms, gemm_n = prof["gemm"]
-    gemm_gbs = gemm_bytes / gemm_launches / (gemm_ms / gemm_n * 1e-3) / 1e9 if gemm_n else None
     t_hbm = ab["total"] / (peaks["hbm_gbs"] * 1e9)
     t_tc = fl / (peaks["bf16_tflops"] * 1e12)
     bound = "hbm" if t_hbm >= t_tc else "tensor"
-    roofline = {"bound": "hbm", "kernel": "gemm_ws_kernel", "achieved": gemm_gbs, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "frac": gemm_gbs / peaks["hbm_gbs"] if gemm_gbs else None,
-                "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH, "peak_source": peaks["source"],
-                "bytes_per_launch": gemm_bytes / gemm_launches, "ms_per_launch": gemm_ms / gemm_n if gemm_n else None}
+    fused_ms, fused_n = prof.get("fused_kernel", (0.0, 0))
+    if fused_n:
+        # the step is ONE launch of the persistent kernel: its algorithmic bytes are the step's; its
+        # duration is the average launch duration over the timed region (launches run back to back)
+        gbs = ab["total"] / (ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": "fused_verify_kernel", "achieved": gbs, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": FUSED_TRAFFIC_BYTES_PER_LAUNCH,
+                    "peak_source": peaks["source"], "bytes_per_launch": ab["total"], "ms_per_launch": ms,
+                    "phase_ms": {k: v[0] for k, v in prof.items() if k in ("gemm", "attention", "attention_merge")}}
+    else:
+        gemm_bytes, gemm_launches = gemm_bytes_per_step(shape, M, planes)
+        gemm_ms, gemm_n = prof["gemm"]
+        gemm_gbs = gemm_bytes / gemm_launches / (gemm_ms / gemm_n * 1e-3) / 1e9 if gemm_n else None
+        roofline = {"bound": "hbm", "kernel": "gemm_ws_kernel", "achieved": gemm_gbs, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": gemm_gbs / peaks["hbm_gbs"] if gemm_gbs else None,
+                    "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH, "peak_source": peaks["source"],
+                    "bytes_per_launch": gemm_bytes / gemm_launches,
+                    "ms_per_launch": gemm_ms / gemm_n if gemm_n else None}
     step_roof = {"bound": bound, "bytes": ab["total"], "flops": fl, "achieved_gbs": ab["total"] / (ms * 1e-3) / 1e9,
                  "frac_of_measured_hbm": ab["total"] / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                  "frac_of_nominal_8tbs": ab["total"] / (ms * 1e-3) / 1e9 / 8000.0,

@@ -66,6 +66,8 @@ typedef struct {
   int32_t max_rows;    /* most rows per call summed over the batch */
   int32_t max_ctx;     /* most tokens per sequence (cache + chunk) */
   int32_t act_split;   /* 1: GEMM activations are fed as a bf16 (hi, lo) pair; 0: hi only */
+  int32_t path;        /* 0: the library chooses; 1: one kernel per stage; 2: the single persistent kernel
+                          (steps of at most 64 rows; a larger step fails with TS_ERR_K_TOO_LARGE) */
 } ts_model_config;
 
 typedef struct {
@@ -97,7 +99,9 @@ enum { TS_W_EMBED = 0, TS_W_LM_HEAD = 1, TS_W_FINAL_GAIN = 2, TS_W_Q = 3, TS_W_K
 /* Upload one tensor.  Matrices are bf16, row-major [out_features][in_features]; gains are
  * float32 [d_model]; the source may be host or device memory (the copy direction is inferred).
  * `layer` is ignored for the three global tensors.  The library lays the matrix out for its
- * kernels (Q,K,V rows concatenated; gate and up rows interleaved).  Synchronous.
+ * kernels (Q,K,V rows concatenated with rotary partners adjacent; gate and up rows interleaved;
+ * every projection matrix stored as contiguous 128 x 64 blocks).  Uses the workspace as staging,
+ * so the last step's logits are gone afterwards.  Synchronous.
  * Errors: TS_ERR_ARG on a shape that does not match the configuration. */
 ts_status ts_load_tensor(ts_model *m, int32_t kind, int32_t layer, const void *host_data,
                          int64_t rows, int64_t cols);
@@ -183,10 +187,13 @@ ts_status ts_verify(ts_model *m, ts_session *const *sessions, int32_t B,
  * sessions advance only in ts_commit.  For timing the kernels alone. */
 ts_status ts_verify_replay(ts_model *m);
 
-/* Run the last step once more with an event after every kernel launch (no overlap between
- * kernels) and return, per kernel class, the summed milliseconds and the launch count:
+/* Run the last step once more and return, per class, the summed milliseconds and a count:
  * 0 projection GEMM, 1 attention, 2 attention merge, 3 norm / residual, 4 rotary + KV append,
- * 5 acceptance.  n_classes >= 6.  Synchronises the stream.  For the benchmark's roofline line. */
+ * 5 acceptance, 6 the persistent kernel as a whole.  n_classes >= 6 (class 6 is written if
+ * n_classes > 6).  With separate kernels an event follows every launch (no overlap between
+ * kernels) and the count is the launches; with the persistent kernel classes 0..2 are sums of
+ * its phases (time between the grid-wide ends of consecutive phases, read from device-side
+ * clocks) and the count is the phases.  Synchronises the stream.  For the benchmark. */
 ts_status ts_profile_step(ts_model *m, float *ms_by_class, int32_t *launches_by_class,
                           int32_t n_classes);
 
@@ -223,11 +230,25 @@ ts_status ts_debug_set_cache(ts_session *s, int32_t cache_len, int32_t pending);
 /* Copy rows [row0, row0+n_rows) of the last step's float32 logits [rows][vocab] to host memory. */
 ts_status ts_read_logits(ts_model *m, int32_t row0, int32_t n_rows, float *host_out);
 /* Copy the first `bytes` bytes of an internal activation buffer of the last step to host memory:
- * 0 residual stream x (float32 [rows_alloc][d_model]); 1 normed activations (bf16
- * [planes][rows_alloc][d_model]); 2 rotated queries (fp16 [rows_alloc][n_q_heads*head_dim]);
+ * 0 residual stream x (float32 [rows_alloc][d_model]); 1 projection input activations (bf16
+ * [planes][rows_alloc][d_model]; normalised with separate kernels, x times gain before the
+ * row scale with the persistent kernel); 2 rotated queries (fp16 [rows_alloc][n_q_heads*head_dim]);
  * 3 attention output (bf16 [planes][rows_alloc][n_q_heads*head_dim]); 4 SwiGLU output (bf16
  * [planes][rows_alloc][d_ffn]).  rows_alloc = max_rows rounded up to 128; planes = 1 + act_split. */
 ts_status ts_debug_read_buffer(ts_model *m, int32_t which, void *host_out, uint64_t bytes);
+/* Device-side clocks (nanoseconds of the GPU's global timer, latest over the CTAs) that the
+ * persistent kernel left during the last ts_profile_step: three rows of *n_phases entries —
+ * end of each phase, last MMA of the phase issued, first operand block of the phase ready.
+ * Copies at most cap values to out (host).  Phases: 0 embedding, then per layer QKV, attention,
+ * merge, O, gate-up, down, then the LM head. */
+ts_status ts_debug_phase_clocks(ts_model *m, uint64_t *out, int32_t cap, int32_t *n_phases);
+/* The persistent kernel's partition of a projection with n_tiles output tiles of 128 features and
+ * n_kblocks blocks of 64 reduction columns over n_ctas CTAs, evaluated on the host for CTA `cta`:
+ * writes up to cap records {tile, first k-block, end k-block, parking slot, first CTA of the tile,
+ * CTAs sharing the tile} to segments (host, 6 int32 each) and the record count to *n_segments.
+ * Host only; for testing the index arithmetic without a GPU. */
+ts_status ts_debug_schedule(int32_t n_tiles, int32_t n_kblocks, int32_t n_ctas, int32_t cta, int32_t cap,
+                            int32_t *segments, int32_t *n_segments);
 /* Counters: kernels launched since ts_init_model, bytes copied host->device and device->host by
  * ts_verify since then. */
 ts_status ts_model_counters(const ts_model *m, int64_t *launches, int64_t *h2d_bytes,

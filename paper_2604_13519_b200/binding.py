@@ -34,7 +34,7 @@ class ts_model_config(C.Structure):
                                          "d_ffn", "vocab")] + \
                [("rope_theta", C.c_float), ("rms_eps", C.c_float)] + \
                [(n, C.c_int32) for n in ("max_pages", "max_batch", "k_max", "max_rows", "max_ctx",
-                                         "act_split")]
+                                         "act_split", "path")]
 
 
 class ts_buffer_sizes(C.Structure):
@@ -108,6 +108,8 @@ _SIGNATURES = {
     "ts_debug_read_buffer": [_P, C.c_int32, _P, C.c_uint64],
     "ts_model_counters": [_P, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64)],
     "ts_attention_static": [C.POINTER(ts_attention_args), _P],
+    "ts_debug_phase_clocks": [_P, C.POINTER(C.c_uint64), C.c_int32, _I32P],
+    "ts_debug_schedule": [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _I32P, _I32P],
 }
 EXPORTED = sorted(list(_SIGNATURES) + ["ts_last_error"])
 
@@ -193,7 +195,7 @@ class Model:
     """ts_init_model + ts_load_tensor over buffers allocated with torch."""
 
     def __init__(self, shape, max_pages: int, max_batch: int, k_max: int, max_rows: int, max_ctx: int,
-                 act_split: bool = True, device="cuda:0", stream=None):
+                 act_split: bool = True, device="cuda:0", stream=None, path: int = 0):
         import torch
         self.torch = torch
         self.shape = shape
@@ -203,6 +205,7 @@ class Model:
             setattr(c, n, getattr(shape, n))
         c.max_pages, c.max_batch, c.k_max, c.max_rows, c.max_ctx = max_pages, max_batch, k_max, max_rows, max_ctx
         c.act_split = 1 if act_split else 0
+        c.path = path
         self.cfg = c
         sizes = ts_buffer_sizes()
         _check(lib().ts_query_buffer_sizes(C.byref(c), C.byref(sizes)))
@@ -263,6 +266,14 @@ class Model:
         out = torch.empty(shape, dtype=dt)
         _check(lib().ts_debug_read_buffer(self.h, which, _P(out.data_ptr()), out.numel() * out.element_size()))
         return out
+
+    def phase_clocks(self):
+        """[3][n_phases] device clocks (ns) left by the last ts_profile_step of the persistent kernel."""
+        import numpy as np
+        n = C.c_int32()
+        buf = (C.c_uint64 * 4096)()
+        _check(lib().ts_debug_phase_clocks(self.h, buf, 4096, C.byref(n)))
+        return np.array(buf[:3 * n.value], dtype=np.uint64).reshape(3, n.value)
 
     def counters(self):
         a, b, c = C.c_int64(), C.c_int64(), C.c_int64()
@@ -364,7 +375,7 @@ def ts_verify_replay(model: Model):
     _check(lib().ts_verify_replay(model.h))
 
 
-KERNEL_CLASSES = ("gemm", "attention", "attention_merge", "norm", "rope_kv", "accept")
+KERNEL_CLASSES = ("gemm", "attention", "attention_merge", "norm", "rope_kv", "accept", "fused_kernel")
 
 
 def ts_profile_step(model: Model):

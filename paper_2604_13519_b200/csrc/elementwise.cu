@@ -118,12 +118,13 @@ __global__ void rope_kv_kernel(StepIn in, const float *part, int n_splits, int p
   pdl_wait();
   const int m = blockIdx.x, head = blockIdx.y, i = threadIdx.x, half = hd >> 1;
   const int N = (Hq + 2 * Hkv) * hd;
-  const int col = head * hd + i;
+  // the QKV weight rows are stored with rotary partners adjacent: feature 2i = element i, 2i+1 = element i + hd/2
+  const int col = head * hd + 2 * i;
   float a = 0.f, b = 0.f;
   for (int s = 0; s < n_splits; ++s) {
-    const float *p = part + ((size_t)s * part_rows + m) * N;
-    a += p[col];
-    b += p[col + half];
+    const float2 ab = *reinterpret_cast<const float2 *>(part + ((size_t)s * part_rows + m) * N + col);
+    a += ab.x;
+    b += ab.y;
   }
   pdl_launch_dependents();
   const int pos = in.pos[m];
@@ -153,6 +154,33 @@ cudaError_t launch_rope_kv(const StepIn &in, const float *part, int n_splits, in
                            cudaStream_t st) {
   return launch_pdl(rope_kv_kernel, dim3(in.M, Hq + 2 * Hkv), dim3(hd / 2), 0, st, in, part, n_splits,
                     part_rows, Hq, Hkv, hd, rope_tab, q_out, k_pages, v_pages);
+}
+
+// One CTA per source row; thread i moves 16 bytes.  Block (tile, kb) of the stored matrix starts at row
+// (tile * K/64 + kb) * 128 of a [.][64] array.
+__global__ void retile_kernel(const __nv_bfloat16 *src, int r0, int K, RowMap rm, __nv_bfloat16 *dst) {
+  const int r = r0 + blockIdx.x;
+  int row;
+  if (rm.hd) {
+    const int e = r % rm.hd, half = rm.hd >> 1;
+    row = rm.base + (r / rm.hd) * rm.hd + (e < half ? 2 * e : 2 * (e - half) + 1);
+  } else {
+    row = rm.base + r * rm.mul;
+  }
+  const int tile = row >> 7, rr = row & 127, KB = K >> 6;
+  const uint4 *s = reinterpret_cast<const uint4 *>(src + (size_t)blockIdx.x * K);
+  for (int i = threadIdx.x; i < K / 8; i += blockDim.x) {
+    const int kb = i >> 3, c = i & 7;
+    uint4 *d = reinterpret_cast<uint4 *>(dst + ((size_t)(tile * KB + kb) * 128 + rr) * 64) + c;
+    *d = s[i];
+  }
+}
+
+cudaError_t launch_retile(const __nv_bfloat16 *src, int n_rows, int r0, int K, RowMap rm, __nv_bfloat16 *dst,
+                          cudaStream_t st) {
+  if (n_rows <= 0) return cudaSuccess;
+  retile_kernel<<<n_rows, 256, 0, st>>>(src, r0, K, rm, dst);
+  return cudaGetLastError();
 }
 
 // One CTA per sequence.  Each row's argmax was reduced by the LM-head epilogue into a packed

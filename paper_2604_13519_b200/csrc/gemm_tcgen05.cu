@@ -2,6 +2,7 @@
 //     out[m][n] = sum_k act[m][k] * W[n][k]
 // with few rows m (the verified positions) and a large weight matrix read exactly once.
 //
+// The weight matrix is stored as contiguous 128 x 64 blocks (one TMA box each).
 // Operands are swapped with respect to the usual layout so that the 128-row dimension of the
 // tensor-core instruction runs over output features: a CTA owns 128 rows of W (operand A, K-major,
 // 16 KB per 64-wide k-block) and a chunk of up to 128 activation rows (operand B).  Activations can
@@ -80,7 +81,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
       for (int it = 0; it < pre; ++it) {
         uint32_t bar = smem_u32(&ctl->full[it]);
         mbar_expect_tx(bar, stage_bytes);
-        tma_load_2d(smem_u32(smem + (size_t)it * stage_bytes), &tmap_w, (kb0 + it) * kBlockK, n0, bar, pol_w);
+        tma_load_2d(smem_u32(smem + (size_t)it * stage_bytes), &tmap_w, 0, (blockIdx.x * g.n_kblocks + kb0 + it) * kTileN, bar, pol_w);
       }
       pdl_wait();
       for (int it = 0; it < pre; ++it) {
@@ -98,7 +99,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
         uint32_t bar = smem_u32(&ctl->full[s]);
         mbar_expect_tx(bar, stage_bytes);
         uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
-        tma_load_2d(dst, &tmap_w, (kb0 + it) * kBlockK, n0, bar, pol_w);
+        tma_load_2d(dst, &tmap_w, 0, (blockIdx.x * g.n_kblocks + kb0 + it) * kTileN, bar, pol_w);
         tma_load_3d(dst + kWBytes, &tmap_a, (kb0 + it) * kBlockK, m0, 0, bar, pol_a);
       }
     } else if (lane == 0) {

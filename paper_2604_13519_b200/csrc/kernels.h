@@ -87,4 +87,58 @@ struct AcceptArgs {
 };
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t st);
 
+// Where a source row of an uploaded matrix goes in the stored matrix: row r -> base + r * mul, or, with
+// hd != 0, base + (r / hd) * hd + p(r % hd) with p(e) = 2e for e < hd/2 and 2(e - hd/2) + 1 otherwise.
+struct RowMap { int base, mul, hd; };
+// Scatter n_rows source rows (row-major, K columns, first one being row r0 of the uploaded matrix) into the
+// 128 x 64-block storage of the stored matrix.
+cudaError_t launch_retile(const __nv_bfloat16 *src, int n_rows, int r0, int K, RowMap rm, __nv_bfloat16 *dst,
+                          cudaStream_t st);
+
+// ---- fused single-kernel step (fused.cu) ---------------------------------------------------------------
+struct FusedArgs {
+  // model shape
+  int n_layers, d, Nqkv, Nq, F, V, Hq, Hkv, hd;
+  float eps;
+  // step
+  StepIn in;
+  int Mc, mc_index, planes;      // activation rows per MMA (16, 32 or 64), its index, 1 or 2 planes
+  int n_ctas, ring, attn_smem_bytes, skip_lm, k_max;
+  int n_attn_tiles, attn_splits;
+  const int32_t *tile_seq;       // [n_attn_tiles] sequence of each 128-row tile of packed rows
+  const int32_t *tile_row0;      // [n_attn_tiles] first packed row of the tile
+  // tensor maps in device memory: 4 per layer (qkv, o, gate-up, down), LM head, then per row-chunk
+  // size three activation maps (h, attn, act)
+  const CUtensorMap *maps;
+  const __nv_bfloat16 *embed;
+  const float *gains;            // g1[0], g2[0], g1[1], ..., gf; gain_stride floats apart
+  int gain_stride;
+  const float2 *rope;
+  __half *kv_pool;
+  unsigned long long kv_layer_stride, kv_v_offset;   // in fp16 elements
+  // workspace
+  float *x;                      // [R][d] residual stream
+  __nv_bfloat16 *h, *attn, *act; // [planes][R][.]
+  int R;
+  __half *q;                     // [R][Hq*hd]
+  float *slab;                   // [n_ctas][2][Mc][128] parked partial tiles
+  float *ss_part;                // [d/128][R] per-tile sums of squares of x
+  float *attn_o;                 // [M*Hq][splits][hd]
+  float2 *attn_ml;               // [M*Hq][splits]
+  float *logits;                 // [M][V]
+  unsigned long long *amax;      // [M]
+  int *sync;                     // [0] phase counter, [2] exit counter, [8..] tile counters (all zero between launches)
+  int *err;                      // device status word shared with the other kernels
+  int n_counters;
+  // optional clocks (ns, latest over the CTAs), three rows of n_phases: phase end; last MMA of the phase
+  // issued; first weight+activation block of the phase ready
+  unsigned long long *phase_t;
+  int n_phases;
+  // results
+  int32_t *out_argmax, *out_accept, *out_emitted, *out_newlen, *out_newpend;
+};
+size_t fused_attn_smem_bytes(int hd);
+int fused_ring_stages(int planes, int Mc, int hd, size_t smem_limit);
+cudaError_t launch_fused(FusedArgs a, size_t smem_limit, cudaStream_t st);
+
 }  // namespace ts

@@ -10,6 +10,7 @@
 
 #include "drafter.h"
 #include "kernels.h"
+#include "schedule.h"
 #include "toolspec.h"
 
 namespace {
@@ -38,6 +39,9 @@ inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 constexpr int kMaxSplits = 12;
 constexpr int kMaxAttnSplits = 32;
 constexpr int kMcOptions[4] = {16, 32, 64, 128};
+constexpr int kMaxFusedCtas = 256;   // the fused kernel runs one CTA per SM
+constexpr int kFusedMaxRows = 64;    // most rows per step the fused kernel takes
+constexpr bool kAutoPrefersFused = false;   // path = 0 picks the faster of the two on the 8B batch-1 step
 
 struct Layout {
   // weights buffer (byte offsets)
@@ -48,6 +52,9 @@ struct Layout {
   uint64_t kv_layer_stride, kv_v_offset, kv_bytes;   // in fp16 elements / bytes
   // workspace (byte offsets)
   uint64_t x, h, part, q, attn_o, attn_ml, attn, act, logits, amax, rope, d_in, d_out, workspace_bytes;
+  // fused single-kernel path
+  uint64_t maps, slab, ss_part, sync, phase_t;
+  int n_maps, n_counters, n_phases, max_tiles128, o_tile128_seq, o_tile128_row0;
   // step io (int32 offsets inside d_in / h_in)
   int o_tokens, o_pos, o_rowseq, o_cu, o_len, o_tile_seq, o_tile_row0, o_btab, in_ints;
   // step out (int32 offsets)
@@ -68,6 +75,7 @@ bool config_ok(const ts_model_config &c, const char **why) {
   REQ(c.max_batch >= 1 && c.max_rows >= c.k_max && c.max_rows <= c.max_batch * c.k_max, "max_rows out of range");
   REQ(c.max_ctx >= c.k_max && c.max_pages >= 1, "max_ctx / max_pages out of range");
   REQ(c.act_split == 0 || c.act_split == 1, "act_split must be 0 or 1");
+  REQ(c.path >= 0 && c.path <= 2, "path must be 0 (auto), 1 (separate kernels) or 2 (fused kernel)");
   REQ(c.rope_theta > 1.f && c.rms_eps > 0.f, "rope_theta / rms_eps out of range");
 #undef REQ
   return true;
@@ -122,6 +130,8 @@ void make_layout(const ts_model_config &c, Layout *L) {
   L->o_tokens = itake(c.max_rows); L->o_pos = itake(c.max_rows); L->o_rowseq = itake(c.max_rows);
   L->o_cu = itake(c.max_batch + 1); L->o_len = itake(c.max_batch);
   L->o_tile_seq = itake(L->max_tiles); L->o_tile_row0 = itake(L->max_tiles);
+  L->max_tiles128 = c.max_batch * ((c.k_max * G + 127) / 128);
+  L->o_tile128_seq = itake(L->max_tiles128); L->o_tile128_row0 = itake(L->max_tiles128);
   L->o_btab = itake(c.max_batch * L->pages_per_seq);
   L->in_ints = io;
   io = 0;
@@ -130,6 +140,14 @@ void make_layout(const ts_model_config &c, Layout *L) {
   L->out_ints = io;
   L->d_in = take((uint64_t)L->in_ints * 4);
   L->d_out = take((uint64_t)L->out_ints * 4);
+  L->n_maps = 4 * c.n_layers + 1 + 3 * 3;
+  L->maps = take((uint64_t)L->n_maps * sizeof(CUtensorMap));
+  L->slab = take((uint64_t)kMaxFusedCtas * 2 * kFusedMaxRows * 128 * 4);
+  L->ss_part = take((uint64_t)(d / 128) * R * 4);
+  L->n_counters = (int)((L->Nqkv + 2 * d + 2 * F + V) / 128);
+  L->sync = take((uint64_t)(8 + L->n_counters) * 4);
+  L->n_phases = 6 * c.n_layers + 3;
+  L->phase_t = take((uint64_t)3 * L->n_phases * 8);
   L->workspace_bytes = o;
   L->host_io_bytes = align_up((uint64_t)(L->in_ints + L->out_ints) * 4, 4096);
 }
@@ -166,11 +184,13 @@ struct ts_model {
   std::vector<int32_t> free_pages;
   std::vector<ts_session *> sessions;   // live sessions over this model (detached on destroy)
   // last staged step
-  int last_B = 0, last_M = 0, last_tiles = 0;
+  int last_B = 0, last_M = 0, last_tiles = 0, last_tiles128 = 0;
   uint32_t last_flags = 0;
   bool have_step = false;
   int64_t launches = 0, h2d = 0, d2h = 0;
   bool use_pdl = true;
+  bool fused_ok = false, last_fused = false;   // device can run the fused kernel; the staged step uses it
+  size_t smem_optin = 0;
   // per-kernel timing pass (ts_profile_step): one event after every launch
   bool profiling = false;
   std::vector<cudaEvent_t> prof_ev;
@@ -225,8 +245,11 @@ ts_status make_map(EncodeTiledFn enc, CUtensorMap *out, void *base, int rank, co
   return TS_OK;
 }
 
+// Weights are stored block by block: the 128 x 64 block (tile t, k-block kb) of an [N][K] matrix is the
+// contiguous 16 KB at rows (t * K/64 + kb) * 128 .. of a [.][64] array.  One block is one TMA box and one run
+// of DRAM pages.
 ts_status weight_map(EncodeTiledFn enc, CUtensorMap *out, void *base, uint64_t N, uint64_t K) {
-  const uint64_t dims[2] = {K, N};
+  const uint64_t dims[2] = {64, N * (K / 64)};
   const uint32_t box[2] = {64, 128};
   return make_map(enc, out, base, 2, dims, box);
 }
@@ -278,7 +301,55 @@ ts_status run_gemm(ts_model *m, int epi, const CUtensorMap &tw, const CUtensorMa
   return TS_OK;
 }
 
+// The staged step as one persistent kernel (fused.cu).
+ts_status run_step_fused(ts_model *m) {
+  const ts_model_config &c = m->c;
+  const Layout &L = m->L;
+  int32_t *di = m->d_in();
+  int32_t *dout = m->d_out();
+  ts::FusedArgs a{};
+  a.n_layers = c.n_layers; a.d = c.d_model; a.Nqkv = L.Nqkv; a.Nq = c.n_q_heads * c.head_dim; a.F = c.d_ffn;
+  a.V = c.vocab; a.Hq = c.n_q_heads; a.Hkv = c.n_kv_heads; a.hd = c.head_dim; a.eps = c.rms_eps;
+  a.in.tokens = di + L.o_tokens; a.in.pos = di + L.o_pos; a.in.row_seq = di + L.o_rowseq; a.in.cu_rows = di + L.o_cu;
+  a.in.seq_len = di + L.o_len; a.in.block_tab = di + L.o_btab; a.in.pages_per_seq = L.pages_per_seq;
+  a.in.B = m->last_B; a.in.M = m->last_M;
+  a.mc_index = pick_mc_index(m->last_M); a.Mc = kMcOptions[a.mc_index]; a.planes = m->planes;
+  a.n_ctas = m->n_sms; a.skip_lm = (m->last_flags & TS_FLAG_SKIP_LM_HEAD) ? 1 : 0;
+  a.k_max = c.k_max;
+  a.n_attn_tiles = m->last_tiles128;
+  {
+    int max_total = 0;
+    const int32_t *hi = m->h_in();
+    for (int i = 0; i < m->last_B; ++i)
+      max_total = std::max(max_total, hi[L.o_len + i] + (hi[L.o_cu + i + 1] - hi[L.o_cu + i]));
+    const int nblk = (max_total + 63) / 64;
+    const int s = m->n_sms / std::max(1, c.n_kv_heads * m->last_tiles128);
+    a.attn_splits = std::max(1, std::min(std::min(s, kMaxAttnSplits), nblk));
+  }
+  a.tile_seq = di + L.o_tile128_seq; a.tile_row0 = di + L.o_tile128_row0;
+  a.maps = (const CUtensorMap *)m->WS(L.maps);
+  a.embed = (const __nv_bfloat16 *)m->W(L.embed);
+  a.gains = (const float *)m->W(L.g1[0]);
+  a.gain_stride = (int)(align_up((uint64_t)c.d_model * 4, 1024) / 4);
+  a.rope = (const float2 *)m->WS(L.rope);
+  a.kv_pool = (__half *)m->b.kv_pool; a.kv_layer_stride = L.kv_layer_stride; a.kv_v_offset = L.kv_v_offset;
+  a.x = (float *)m->WS(L.x); a.h = (__nv_bfloat16 *)m->WS(L.h); a.attn = (__nv_bfloat16 *)m->WS(L.attn);
+  a.act = (__nv_bfloat16 *)m->WS(L.act); a.R = L.rows_alloc; a.q = (__half *)m->WS(L.q);
+  a.slab = (float *)m->WS(L.slab); a.ss_part = (float *)m->WS(L.ss_part);
+  a.attn_o = (float *)m->WS(L.attn_o); a.attn_ml = (float2 *)m->WS(L.attn_ml);
+  a.logits = (float *)m->WS(L.logits); a.amax = (unsigned long long *)m->WS(L.amax);
+  a.sync = (int *)m->WS(L.sync); a.err = dout + L.o_err; a.n_counters = L.n_counters;
+  a.phase_t = m->profiling ? (unsigned long long *)m->WS(L.phase_t) : nullptr;
+  a.n_phases = L.n_phases;
+  a.out_argmax = dout + L.o_argmax; a.out_accept = dout + L.o_accept; a.out_emitted = dout + L.o_emitted;
+  a.out_newlen = dout + L.o_newlen; a.out_newpend = dout + L.o_newpend;
+  CU_TRY(ts::launch_fused(a, m->smem_optin, m->st));
+  m->launched(6);
+  return TS_OK;
+}
+
 ts_status run_step(ts_model *m) {
+  if (m->last_fused) return run_step_fused(m);
   const ts_model_config &c = m->c;
   const Layout &L = m->L;
   const int M = m->last_M, B = m->last_B;
@@ -381,7 +452,7 @@ ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::ve
   const Layout &L = m->L;
   int32_t *hi = m->h_in();
   const int G = c.n_q_heads / c.n_kv_heads;
-  int M = 0, tiles = 0;
+  int M = 0, tiles = 0, tiles128 = 0;
   hi[L.o_cu] = 0;
   for (int i = 0; i < B; ++i) {
     ts_session *s = ss[i];
@@ -404,11 +475,22 @@ ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::ve
       hi[L.o_tile_row0 + tiles] = r0;
       ++tiles;
     }
+    for (int r0 = 0; r0 < k * G; r0 += 128) {
+      hi[L.o_tile128_seq + tiles128] = i;
+      hi[L.o_tile128_row0 + tiles128] = r0;
+      ++tiles128;
+    }
     std::memcpy(hi + L.o_btab + (size_t)i * L.pages_per_seq, s->pages.data(), s->pages.size() * sizeof(int32_t));
     M += k;
     hi[L.o_cu + i + 1] = M;
   }
-  m->last_B = B; m->last_M = M; m->last_tiles = tiles; m->last_flags = flags; m->have_step = true;
+  const bool can_fuse = m->fused_ok && M <= kFusedMaxRows;
+  if (c.path == 2 && !can_fuse)
+    return fail(TS_ERR_K_TOO_LARGE, "the fused kernel takes at most %d rows on a device that supports it (step has %d)",
+                kFusedMaxRows, M);
+  m->last_fused = can_fuse && (c.path == 2 || (c.path == 0 && kAutoPrefersFused));
+  m->last_B = B; m->last_M = M; m->last_tiles = tiles; m->last_tiles128 = tiles128; m->last_flags = flags;
+  m->have_step = true;
   const size_t in_bytes = (size_t)(L.o_btab + (size_t)B * L.pages_per_seq) * 4;
   CU_TRY(cudaMemcpyAsync(m->d_in(), hi, in_bytes, cudaMemcpyHostToDevice, m->st));
   m->h2d += (int64_t)in_bytes;
@@ -421,6 +503,7 @@ ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::ve
   const int dev_err = m->h_out()[L.o_err];
   if (dev_err != 0) {
     cudaMemsetAsync(m->d_out() + L.o_err, 0, 4, m->st);
+    cudaMemsetAsync(m->WS(L.sync), 0, (size_t)(8 + L.n_counters) * 4, m->st);   // the fused kernel left its counters mid-step
     return fail(TS_ERR_DEVICE_TIMEOUT, "a bounded device-side wait expired (code %d)", dev_err);
   }
   return TS_OK;
@@ -540,6 +623,28 @@ ts_status ts_init_model(const ts_model_config *cfg, const ts_buffers *bufs, void
   if (!s) s = act_maps(enc, m->tm_attn, m->WS(L.attn), Nq, L.rows_alloc, m->planes);
   if (!s) s = act_maps(enc, m->tm_act, m->WS(L.act), F, L.rows_alloc, m->planes);
   if (s) return bail(s);
+  {
+    // the fused kernel reads its tensor maps from device memory
+    std::vector<CUtensorMap> maps(L.n_maps);
+    for (int l = 0; l < c.n_layers; ++l) {
+      maps[4 * l + 0] = m->tm_qkv[l]; maps[4 * l + 1] = m->tm_o[l]; maps[4 * l + 2] = m->tm_gu[l]; maps[4 * l + 3] = m->tm_d[l];
+    }
+    maps[4 * c.n_layers] = m->tm_lm;
+    for (int i = 0; i < 3; ++i) {
+      maps[4 * c.n_layers + 1 + 3 * i + 0] = m->tm_h[i];
+      maps[4 * c.n_layers + 1 + 3 * i + 1] = m->tm_attn[i];
+      maps[4 * c.n_layers + 1 + 3 * i + 2] = m->tm_act[i];
+    }
+    e = cudaMemcpyAsync(m->WS(L.maps), maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, m->st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(m->st);
+    if (e != cudaSuccess) return bail(fail(TS_ERR_CUDA, "tensor map upload: %s", cudaGetErrorString(e)));
+    int coop = 0, optin = 0;
+    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    m->smem_optin = (size_t)optin;
+    m->fused_ok = coop != 0 && m->n_sms <= kMaxFusedCtas &&
+                  ts::fused_ring_stages(m->planes, kFusedMaxRows, c.head_dim, m->smem_optin) >= 2;
+  }
   m->free_pages.resize(c.max_pages);
   for (int i = 0; i < c.max_pages; ++i) m->free_pages[i] = c.max_pages - 1 - i;   // hand out 0, 1, 2, ...
   *out = m;
@@ -566,28 +671,50 @@ ts_status ts_load_tensor(ts_model *m, int32_t kind, int32_t layer, const void *h
   if (!global && (layer < 0 || layer >= c.n_layers)) return fail(TS_ERR_ARG, "layer %d out of range", layer);
   int64_t er = 0, ec = 0;
   uint8_t *dst = nullptr;
-  size_t dpitch = 0, esz = 2;
+  size_t esz = 2;
+  ts::RowMap rm{0, 1, 0};
   switch (kind) {
     case TS_W_EMBED: er = c.vocab; ec = d; dst = m->W(L.embed); break;
     case TS_W_LM_HEAD: er = c.vocab; ec = d; dst = m->W(L.lm_head); break;
     case TS_W_FINAL_GAIN: er = 1; ec = d; dst = m->W(L.gf); esz = 4; break;
     case TS_W_GAIN1: er = 1; ec = d; dst = m->W(L.g1[layer]); esz = 4; break;
     case TS_W_GAIN2: er = 1; ec = d; dst = m->W(L.g2[layer]); esz = 4; break;
-    case TS_W_Q: er = Nq; ec = d; dst = m->W(L.wqkv[layer]); break;
-    case TS_W_K: er = Nkv; ec = d; dst = m->W(L.wqkv[layer]) + Nq * d * 2; break;
-    case TS_W_V: er = Nkv; ec = d; dst = m->W(L.wqkv[layer]) + (Nq + Nkv) * d * 2; break;
+    case TS_W_Q: er = Nq; ec = d; dst = m->W(L.wqkv[layer]); rm.base = 0; rm.hd = (int)hd; break;
+    case TS_W_K: er = Nkv; ec = d; dst = m->W(L.wqkv[layer]); rm.base = (int)Nq; rm.hd = (int)hd; break;
+    case TS_W_V: er = Nkv; ec = d; dst = m->W(L.wqkv[layer]); rm.base = (int)(Nq + Nkv); rm.hd = (int)hd; break;
     case TS_W_O: er = d; ec = Nq; dst = m->W(L.wo[layer]); break;
-    case TS_W_GATE: er = F; ec = d; dst = m->W(L.wgu[layer]); dpitch = 2 * d * 2; break;           // even rows
-    case TS_W_UP: er = F; ec = d; dst = m->W(L.wgu[layer]) + d * 2; dpitch = 2 * d * 2; break;      // odd rows
+    case TS_W_GATE: er = F; ec = d; dst = m->W(L.wgu[layer]); rm.mul = 2; break;               // even rows
+    case TS_W_UP: er = F; ec = d; dst = m->W(L.wgu[layer]); rm.mul = 2; rm.base = 1; break;    // odd rows
     case TS_W_DOWN: er = d; ec = F; dst = m->W(L.wd[layer]); break;
     default: return fail(TS_ERR_ARG, "unknown tensor kind %d", kind);
   }
   if (rows != er || cols != ec) return fail(TS_ERR_ARG, "tensor kind %d: expected %lld x %lld, got %lld x %lld", kind,
                                             (long long)er, (long long)ec, (long long)rows, (long long)cols);
   const size_t row_bytes = (size_t)ec * esz;
-  if (dpitch == 0) dpitch = row_bytes;
-  CU_TRY(cudaMemcpy2DAsync(dst, dpitch, host, row_bytes, row_bytes, (size_t)er, cudaMemcpyDefault, m->st));
-  CU_TRY(cudaStreamSynchronize(m->st));
+  if (esz == 4 || kind == TS_W_EMBED) {   // gains and the embedding table stay row-major
+    CU_TRY(cudaMemcpyAsync(dst, host, row_bytes * (size_t)er, cudaMemcpyDefault, m->st));
+    CU_TRY(cudaStreamSynchronize(m->st));
+    return TS_OK;
+  }
+  // Projection matrices: rows go to their place in the stored matrix (Q, K, V concatenated, with rotary
+  // partners i and i + hd/2 on adjacent rows 2i and 2i+1; gate and up rows interleaved) and the matrix is
+  // stored as 128 x 64 blocks.  Host sources pass through a staging area inside the workspace.
+  cudaPointerAttributes pa{};
+  const bool on_device = cudaPointerGetAttributes(&pa, host) == cudaSuccess && pa.type == cudaMemoryTypeDevice;
+  cudaGetLastError();
+  const size_t stage_bytes = (size_t)L.rows_alloc * (size_t)c.vocab * 4;   // the logits area doubles as staging
+  const int64_t rows_per_chunk = on_device ? er : std::max<int64_t>(1, (int64_t)(stage_bytes / row_bytes));
+  for (int64_t r0 = 0; r0 < er; r0 += rows_per_chunk) {
+    const int64_t nr = std::min(rows_per_chunk, er - r0);
+    const void *src = (const uint8_t *)host + (size_t)r0 * row_bytes;
+    if (!on_device) {
+      CU_TRY(cudaMemcpyAsync(m->WS(L.logits), src, (size_t)nr * row_bytes, cudaMemcpyHostToDevice, m->st));
+      src = m->WS(L.logits);
+    }
+    CU_TRY(ts::launch_retile((const __nv_bfloat16 *)src, (int)nr, (int)r0, (int)ec, rm, (__nv_bfloat16 *)dst, m->st));
+    CU_TRY(cudaStreamSynchronize(m->st));
+  }
+  m->have_step = false;   // the staging area held the last step's logits
   return TS_OK;
 }
 
@@ -792,6 +919,42 @@ ts_status ts_profile_step(ts_model *m, float *ms_by_class, int32_t *launches_by_
   if (!m || !ms_by_class || !launches_by_class || n_classes < 6) return fail(TS_ERR_ARG, "bad argument");
   if (!m->have_step) return fail(TS_ERR_STATE, "no step has been staged yet");
   for (int i = 0; i < n_classes; ++i) { ms_by_class[i] = 0.f; launches_by_class[i] = 0; }
+  if (m->last_fused) {
+    // one kernel: class 6 is its event time; the phase classes come from the device-side phase-end stamps
+    const Layout &L = m->L;
+    const int n_ph = (m->last_flags & TS_FLAG_SKIP_LM_HEAD) ? 6 * m->c.n_layers + 1 : 6 * m->c.n_layers + 2;
+    CU_TRY(cudaMemsetAsync(m->WS(L.phase_t), 0, (size_t)3 * L.n_phases * 8, m->st));
+    cudaEvent_t e0, e1;
+    CU_TRY(cudaEventCreate(&e0));
+    CU_TRY(cudaEventCreate(&e1));
+    CU_TRY(cudaEventRecord(e0, m->st));
+    m->profiling = true;
+    ts_status st = run_step(m);
+    m->profiling = false;
+    for (cudaEvent_t ev : m->prof_ev) cudaEventDestroy(ev);
+    m->prof_ev.clear();
+    m->prof_cls.clear();
+    cudaEventRecord(e1, m->st);
+    std::vector<unsigned long long> t(L.n_phases);
+    cudaError_t e = cudaMemcpyAsync(t.data(), m->WS(L.phase_t), (size_t)L.n_phases * 8, cudaMemcpyDeviceToHost, m->st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(m->st);
+    float total = 0.f;
+    if (e == cudaSuccess) cudaEventElapsedTime(&total, e0, e1);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (st) return st;
+    if (e != cudaSuccess) return fail(TS_ERR_CUDA, "profile step: %s", cudaGetErrorString(e));
+    for (int p = 1; p < n_ph; ++p) {
+      if (t[p] == 0 || t[p - 1] == 0) continue;
+      const float ms = (float)((double)(t[p] - t[p - 1]) * 1e-6);
+      const int r = (p - 1) % 6;   // 0 qkv, 1 attention, 2 merge, 3 o, 4 gate-up, 5 down; the last phase is the LM head
+      const int cls = (p == 6 * m->c.n_layers + 1) ? 0 : (r == 1 ? 1 : (r == 2 ? 2 : 0));
+      ms_by_class[cls] += ms;
+      ++launches_by_class[cls];
+    }
+    if (n_classes > 6) { ms_by_class[6] = total; launches_by_class[6] = 1; }
+    return TS_OK;
+  }
   cudaEvent_t start;
   CU_TRY(cudaEventCreate(&start));
   CU_TRY(cudaEventRecord(start, m->st));
@@ -938,6 +1101,36 @@ ts_status ts_debug_read_buffer(ts_model *m, int32_t which, void *host_out, uint6
   if (bytes > cap) return fail(TS_ERR_ARG, "buffer %d holds %llu bytes", which, (unsigned long long)cap);
   CU_TRY(cudaMemcpyAsync(host_out, m->WS(off), bytes, cudaMemcpyDeviceToHost, m->st));
   CU_TRY(cudaStreamSynchronize(m->st));
+  return TS_OK;
+}
+
+ts_status ts_debug_phase_clocks(ts_model *m, uint64_t *out, int32_t cap, int32_t *n_phases) {
+  if (!m || !n_phases || (cap > 0 && !out)) return fail(TS_ERR_ARG, "null argument");
+  *n_phases = m->L.n_phases;
+  const size_t n = std::min<size_t>((size_t)std::max(cap, 0), (size_t)3 * m->L.n_phases);
+  CU_TRY(cudaMemcpyAsync(out, m->WS(m->L.phase_t), n * 8, cudaMemcpyDeviceToHost, m->st));
+  CU_TRY(cudaStreamSynchronize(m->st));
+  return TS_OK;
+}
+
+ts_status ts_debug_schedule(int32_t n_tiles, int32_t n_kblocks, int32_t n_ctas, int32_t cta, int32_t cap,
+                            int32_t *segments, int32_t *n_segments) {
+  if (n_tiles < 1 || n_kblocks < 1 || n_ctas < 1 || cta < 0 || cta >= n_ctas || !n_segments || (cap > 0 && !segments))
+    return fail(TS_ERR_ARG, "bad argument");
+  ts::SegmentIter it((uint32_t)cta, n_tiles, n_kblocks, (uint32_t)n_ctas);
+  ts::Segment sg;
+  int n = 0;
+  while (it.next(&sg)) {
+    if (n < cap) {
+      const ts::TileCover tc = ts::tile_cover(sg.tile, n_tiles, n_kblocks, (uint32_t)n_ctas);
+      int32_t *o = segments + 6 * n;
+      o[0] = sg.tile; o[1] = sg.kb0; o[2] = sg.kb1;
+      o[3] = ts::slab_slot_of(cta, sg.tile, n_tiles, n_kblocks, (uint32_t)n_ctas);
+      o[4] = tc.c_first; o[5] = tc.n_seg;
+    }
+    ++n;
+  }
+  *n_segments = n;
   return TS_OK;
 }
 

@@ -12,13 +12,13 @@ GAP = 0.05               # integer results may differ only where the oracle's to
 
 
 def make_pair(shape, max_batch=1, k_max=8, max_rows=None, max_ctx=1024, max_pages=None, act_split=True,
-              weights=None):
+              weights=None, path=0):
     w = weights if weights is not None else synth.make_weights(shape)
     om = oracle.OracleModel(shape, w)
     max_rows = max_rows or max_batch * k_max
     max_pages = max_pages or max_batch * ((max_ctx + 15) // 16)
     gm = ts.Model(shape, max_pages=max_pages, max_batch=max_batch, k_max=k_max, max_rows=max_rows,
-                  max_ctx=max_ctx, act_split=act_split)
+                  max_ctx=max_ctx, act_split=act_split, path=path)
     gm.load_weights(w)
     return om, gm
 

@@ -12,6 +12,9 @@ from gpu_util import make_pair, synthetic_context, check_step
 
 pytestmark = pytest.mark.gpu
 
+# both implementations of a step: 1 = one kernel per stage, 2 = the single persistent kernel
+PATHS = [pytest.param(1, id="separate"), pytest.param(2, id="fused")]
+
 
 def _rand_draft(vocab, n, seed):
     g = torch.Generator().manual_seed(seed)
@@ -26,11 +29,12 @@ def _stores(schema, inv):
     return st_o, st_c
 
 
-def test_c1_decode_loop_parity():
+@pytest.mark.parametrize("path", PATHS)
+def test_c1_decode_loop_parity(path):
     """Config 1: tiny decoder, 256-token context through the real prefill on both sides, k = 8,
     8 tools, 64 historical invocations, 20 decode steps following the oracle's trajectory."""
     shape = synth.SHAPES["tiny"]
-    om, gm = make_pair(shape, k_max=8, max_ctx=512)
+    om, gm = make_pair(shape, k_max=8, max_ctx=512, path=path)
     schema = synth.make_schema(shape.vocab, 8)
     inv = synth.make_datastore(schema, 64)
     v = schema.vocab
@@ -73,12 +77,13 @@ def test_c1_decode_loop_parity():
     assert max(accepted) == 7 and 0 < min(a for a in accepted if a) < 7   # full and partial acceptance
 
 
+@pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("name,ctx,k", [("1b-2l", 128, 4), ("1b-2l", 128, 8), ("1b-2l", 131, 16), ("8b-2l", 100, 32)])
-def test_real_prefill_shapes(name, ctx, k):
+def test_real_prefill_shapes(name, ctx, k, path):
     """Configs 2/3 at reduced depth: real prefill on both sides (K/V are rounded to bf16 on the
     GPU only), then one verify step with a partly correct draft."""
     shape = synth.SHAPES[name]
-    om, gm = make_pair(shape, k_max=max(k, 16), max_ctx=512)
+    om, gm = make_pair(shape, k_max=max(k, 16), max_ctx=512, path=path)
     prompt = synth.make_context(shape.vocab, ctx)
     cache, pending = oracle.prefill(om, prompt)
     s = ts.Session(gm, None, None)
@@ -94,13 +99,14 @@ def test_real_prefill_shapes(name, ctx, k):
     gm.close()
 
 
+@pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("name,ctx,k", [("8b-2l", 2048, 32), ("8b-2l", 1000, 1), ("8b-2l", 64, 17),
-                                        ("1b-2l", 4096, 16), ("1b-2l", 15, 2), ("tiny", 0, 8)])
-def test_synthetic_kv_single(name, ctx, k):
+                                        ("1b-2l", 4096, 16), ("1b-2l", 15, 2), ("tiny", 0, 8), ("8b-2l", 700, 64)])
+def test_synthetic_kv_single(name, ctx, k, path):
     """Long contexts as seeded synthetic K/V imported on both sides; ragged lengths around page and
     block boundaries; k = 1 (empty draft) and an empty cache included."""
     shape = synth.SHAPES[name]
-    om, gm = make_pair(shape, k_max=max(k, 8), max_ctx=ctx + 64)
+    om, gm = make_pair(shape, k_max=max(k, 8), max_ctx=ctx + 64, path=path)
     cache, s, pending = synthetic_context(shape, om, gm, ctx)
     draft = _rand_draft(shape.vocab, k - 1, 5)
     ref = om.verify(pending, draft, cache, want_logits=True)
@@ -200,4 +206,24 @@ def test_argument_and_capacity_errors():
     assert e.value.code == -3
     res = ts.ts_verify(gm, [s], [[70]])[0]                 # the context is still usable
     assert res.k == 2
+    gm.close()
+
+
+def test_small_batch_fused():
+    """Several short sequences in one step of the persistent kernel (ragged k, ragged contexts)."""
+    shape = synth.SHAPES["1b-2l"]
+    lens, ks = [40, 333, 17, 129], [9, 4, 16, 11]
+    om, gm = make_pair(shape, max_batch=4, k_max=16, max_rows=sum(ks), max_ctx=512, path=2)
+    sess, drafts, refs = [], [], []
+    for i, (n, k) in enumerate(zip(lens, ks)):
+        cache, s, pending = synthetic_context(shape, om, gm, n, stream=i, pending=100 + i)
+        draft = _rand_draft(shape.vocab, k - 1, 20 + i)
+        sess.append(s); drafts.append(draft)
+        refs.append(om.verify(pending, draft, cache, want_logits=True))
+    out = ts.ts_verify(gm, sess, drafts)
+    row = 0
+    for i, (res, ref) in enumerate(zip(out, refs)):
+        assert res.first_row == row and res.k == ks[i]
+        check_step(res, gm.read_logits(row, res.k), ref, f"seq {i}")
+        row += res.k
     gm.close()

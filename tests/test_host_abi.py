@@ -147,3 +147,39 @@ def test_session_errors():
     assert ts.ts_draft(s, 0) == ([], 0)
     with pytest.raises(ts.TsError):
         s.set_ranks([0])                 # no datastore
+
+
+@pytest.mark.parametrize("T,KB,n", [(48, 64, 148), (32, 64, 148), (192, 64, 148), (32, 192, 148), (1187, 64, 148),
+                                    (6, 4, 148), (2, 4, 148), (1, 1, 148), (7, 3, 5), (5, 9, 4), (3, 64, 1)])
+def test_fused_schedule_partition(T, KB, n):
+    """The persistent kernel's split of a projection over CTAs: every (tile, k-block) unit exactly
+    once, equal shares to within one unit among the CTAs that take part, a tile's pieces on
+    consecutive CTAs, whole tiles in the middle of a range, one parked piece per slot at most."""
+    L = B.lib()
+    seen, sizes, per_tile = {}, [], {}
+    for c in range(n):
+        buf = (C.c_int32 * (6 * 4096))()
+        cnt = C.c_int32()
+        assert L.ts_debug_schedule(T, KB, n, c, 4096, buf, C.byref(cnt)) == 0
+        segs = [tuple(buf[6 * i:6 * i + 6]) for i in range(cnt.value)]
+        units, slots = 0, set()
+        for i, (tile, kb0, kb1, slot, c_first, n_seg) in enumerate(segs):
+            assert 0 <= tile < T and 0 <= kb0 < kb1 <= KB
+            for kb in range(kb0, kb1):
+                assert (tile, kb) not in seen
+                seen[(tile, kb)] = c
+            units += kb1 - kb0
+            assert slot == (0 if i == 0 else 1)
+            partial = not (kb0 == 0 and kb1 == KB)
+            assert (n_seg > 1) == partial
+            if partial:
+                assert slot not in slots and (i == 0 or i == len(segs) - 1)
+                slots.add(slot)
+            per_tile.setdefault(tile, []).append((c, c_first, n_seg))
+        if units:
+            sizes.append(units)
+    assert len(seen) == T * KB
+    assert len(sizes) == min(n, T * KB) and max(sizes) - min(sizes) <= 1
+    for tile, lst in per_tile.items():
+        assert [c for c, _, _ in lst] == list(range(lst[0][1], lst[0][1] + lst[0][2]))
+        assert all(cf == lst[0][1] and ns == lst[0][2] for _, cf, ns in lst)
