@@ -86,7 +86,8 @@ typedef struct {
 ts_status ts_query_buffer_sizes(const ts_model_config *cfg, ts_buffer_sizes *out);
 
 /* ts_init_model — create the target model M of Algorithm 1 ("Require: target model M") over
- * caller-owned buffers.  Zeroes the workspace, builds the TMA descriptors and the rotary table.
+ * caller-owned buffers.  Zeroes the workspace and the KV pool (cache positions that were never
+ * written must read as finite numbers), builds the TMA descriptors and the rotary table.
  * Weights are loaded afterwards with ts_load_tensor.  `stream` is a cudaStream_t (0 = default).
  * Errors: TS_ERR_ARG (bad shape: head_dim not 64/128, dims not multiples of 128, ...),
  * TS_ERR_CUDA. */

@@ -12,8 +12,8 @@
 //                      once the phase that writes them has completed on every CTA.
 //              warp 2  tcgen05.mma issue (weights = operand A, 128 rows; activations = operand B),
 //                      fp32 accumulators in tensor memory, four buffers.
-//              warps 3..10  workers: epilogues out of tensor memory, tile fix-up, attention
-//                      (mma.sync on fp16 K/V staged with cp.async), merge, acceptance.
+//              warps 3..10  workers: epilogues out of tensor memory, tile fix-up, the softmax of attention
+//                      (both attention products run on tcgen05 as well, see below), merge, acceptance.
 //
 // Projections are cut stream-K style (schedule.h): every CTA owns an equal run of (tile, k-block)
 // units; a tile shared by several CTAs is finished by the last one to arrive, which adds the parked
@@ -55,6 +55,10 @@ struct __align__(16) FusedCtl {
   uint32_t tmem_base;
   int flag;
   int attn_epoch;            // attention phases this CTA has finished (ring slots under the staging area are free)
+  // attention pipeline: K/V stages (TMA -> MMA), Q tile, score / probability / output-block buffers
+  uint64_t kv_full[2], kv_empty[2], q_full;
+  uint64_t s_full[2], s_empty[2], p_full[2], o_full[2], o_empty[2];
+  float l_half[kAttnRows];
   int row_pos[kMaxMc];       // absolute position of each row
   int row_page[kMaxMc];      // KV page holding that position
   float r_s[kMaxMc];
@@ -266,210 +270,174 @@ __device__ __forceinline__ void compute_row_scale(const FusedArgs &a, FusedCtl *
   worker_sync();
 }
 
-// ---- attention (workers) --------------------------------------------------------------------------------
+// ---- attention ----------------------------------------------------------------------------------------------
+// One unit = (128-row tile of packed (position, query head) rows, kv head, split of the KV positions).
+// Both products run on tcgen05:  S = Q K^T  (A = Q tile, B = K block, both K-major fp16 in shared memory,
+// D = 128 x 64 fp32 in tensor memory), then the worker threads (one row each) take the running max, write
+// P = exp2(S - max) back to tensor memory as fp16, and  O_blk = P V  (A = P from tensor memory, B = the V block
+// read MN-major from the same [position][64 elements] image K uses).  The workers add O_blk into registers
+// with the usual running-softmax rescale.  K/V blocks of 64 positions arrive by TMA straight from the pages.
+struct AttnUnit {
+  int tile, kh, split;
+  int seq, row0, rows_here, r_beg, len, G;
+  int pos_beg, pos_end, nblk;
+};
+
+__device__ __forceinline__ AttnUnit attn_unit_info(const FusedArgs &a, int u) {
+  AttnUnit t;
+  t.split = u % a.attn_splits;
+  t.kh = (u / a.attn_splits) % a.Hkv;
+  t.tile = u / (a.attn_splits * a.Hkv);
+  t.G = a.Hq / a.Hkv;
+  t.seq = a.tile_seq[t.tile];
+  t.row0 = a.tile_row0[t.tile];
+  t.r_beg = a.in.cu_rows[t.seq];
+  const int k_i = a.in.cu_rows[t.seq + 1] - t.r_beg;
+  t.len = a.in.seq_len[t.seq];
+  t.rows_here = min(kAttnRows, k_i * t.G - t.row0);
+  const int total = t.len + k_i;
+  const int j_max = (t.row0 + t.rows_here - 1) / t.G;
+  int p0, p1;
+  split_pages((total + 15) >> 4, a.attn_splits, t.split, &p0, &p1);
+  t.pos_beg = p0 << 4;
+  t.pos_end = min(min(p1 << 4, total), t.len + j_max + 1);   // nothing beyond the last row's own position is visible
+  t.nblk = t.pos_end > t.pos_beg ? (t.pos_end - t.pos_beg + kAttnBlk - 1) / kAttnBlk : 0;
+  return t;
+}
+
+// tensor-memory columns of the attention phase (they lie over the projection accumulators, which are idle then)
+static constexpr int kColS = 0;      // two score buffers of 64 columns
+static constexpr int kColP = 128;    // two probability buffers of 32 columns (fp16 pairs)
+static constexpr int kColO = 192;    // two output-block buffers of head_dim columns
+
 __device__ __forceinline__ void cp_async16z(uint32_t dst, const void *src, bool valid) {
   const int sz = valid ? 16 : 0;
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
 }
-__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void ldsm4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-               : "r"(addr));
-}
-__device__ __forceinline__ void ldsm4t(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-               : "r"(addr));
-}
-__device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
-      "{%0, %1, %2, %3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+__device__ __forceinline__ void cp_commit_wait_all() {
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
 }
 __device__ __forceinline__ uint32_t pack_h2(float x, float y) {
   __half2 v = __floats2half2_rn(x, y);
   return *reinterpret_cast<uint32_t *>(&v);
 }
-template <int HD>
-__device__ __forceinline__ uint32_t swz(int r, int c) {
-  return (uint32_t)(r * (HD * 2) + ((c ^ (r & 7)) << 4));
-}
 
-// One unit: (row tile, kv head, split).  256 worker threads; warp w owns packed rows 16w .. 16w+15.
-// K/V blocks of 64 positions are double buffered; scores are taken 32 positions at a time, each with its
-// own running-softmax update, which halves the score registers.
+// Worker side of one unit.  Thread <-> row (tensor-memory lane q*32 + lane); the two warps that share a lane
+// quarter split the exponentials (32 positions each) and the output columns (head_dim / 2 each).
+// `blk` counts K/V blocks over all units of this CTA (buffer index and barrier parity come from it).
 template <int HD>
-__device__ __noinline__ void attn_unit(const FusedArgs &a, int layer, uint8_t *sm, int tile, int kh, int split, int widx,
-                                       int lane, int wtid) {
-  constexpr int CH = HD / 8;
-  constexpr int QB = kAttnRows * HD * 2;
-  constexpr int TB = kAttnBlk * HD * 2;
-  uint8_t *sQ = sm, *sK = sm + QB, *sV = sm + QB + 2 * TB;
-  const int G = a.Hq / a.Hkv;
-  const int seq = a.tile_seq[tile], row0 = a.tile_row0[tile];
-  const int r_beg = a.in.cu_rows[seq];
-  const int k_i = a.in.cu_rows[seq + 1] - r_beg;
-  const int len = a.in.seq_len[seq];
-  const int R = k_i * G;
-  const int rows_here = min(kAttnRows, R - row0);
-  const int total = len + k_i;
-  const int j_max = (row0 + rows_here - 1) / G;
-  int p0, p1;
-  split_pages((total + 15) >> 4, a.attn_splits, split, &p0, &p1);
-  const int pos_beg = p0 << 4;
-  const int pos_end = min(min(p1 << 4, total), len + j_max + 1);
-  const int32_t *btab = a.in.block_tab + (size_t)seq * a.in.pages_per_seq;
-  const __half *kp = a.kv_pool + (size_t)layer * a.kv_layer_stride;
-  const __half *vp = kp + a.kv_v_offset;
-
-  const int rl = widx * 16 + (lane >> 2), rh = rl + 8;
-  const int prl = row0 + rl, prh = row0 + rh;
-  const bool vl = rl < rows_here, vh = rh < rows_here;
-  const int lim_l = min(len + (vl ? prl / G : 0), pos_end - 1), lim_h = min(len + (vh ? prh / G : 0), pos_end - 1);
-  auto out_base = [&](int pr) -> size_t {
-    const int j = pr / G, gq = pr % G;
-    return ((size_t)(r_beg + j) * a.Hq + kh * G + gq) * a.attn_splits + split;
-  };
-  if (pos_beg >= pos_end) {   // nothing visible in this split: mark it empty
-    if ((lane & 3) == 0) {
-      if (vl) a.attn_ml[out_base(prl)] = make_float2(-INFINITY, 0.f);
-      if (vh) a.attn_ml[out_base(prh)] = make_float2(-INFINITY, 0.f);
-    }
-    return;
+__device__ __noinline__ bool attn_unit_workers(const FusedArgs &a, FusedCtl *ctl, const AttnUnit &t, uint8_t *sQ, uint32_t tmem_base,
+                                               int q, int half, int lane, int wtid, uint32_t &blk, uint32_t unit_no,
+                                               const int *err) {
+  constexpr int CH = HD / 8;          // 16-byte chunks per row
+  constexpr int OC = HD / 2;          // output columns per thread
+  const int row = q * 32 + lane;      // row of the tile
+  const int pr = t.row0 + row;        // packed row of the sequence
+  const bool valid = row < t.rows_here;
+  const int j = valid ? pr / t.G : 0, gq = valid ? pr % t.G : 0;
+  const size_t ob = ((size_t)(t.r_beg + j) * a.Hq + t.kh * t.G + gq) * a.attn_splits + t.split;
+  if (t.nblk == 0) {   // nothing visible in this split: mark it empty
+    if (valid && half == 0) a.attn_ml[ob] = make_float2(-INFINITY, 0.f);
+    return true;
   }
-  const int nblk = (pos_end - pos_beg + kAttnBlk - 1) / kAttnBlk;
-
-  worker_sync();   // the previous unit's readers are done with the staging buffers
+  // ---- stage Q: [128 rows][64 elements] images with the 128-byte swizzle, one per 64-element half ----------
   for (int idx = wtid; idx < kAttnRows * CH; idx += kWorkers) {
     const int r = idx / CH, c = idx % CH;
-    const int pr = row0 + r;
-    const bool valid = r < rows_here;
-    const int j = valid ? pr / G : 0, gq = valid ? pr % G : 0;
-    const __half *src = a.q + ((size_t)(r_beg + j) * a.Hq + kh * G + gq) * HD + c * 8;
-    cp_async16z(smem_u32(sQ) + swz<HD>(r, c), src, valid);
+    const int prr = t.row0 + r;
+    const bool v = r < t.rows_here;
+    const int jj = v ? prr / t.G : 0, gg = v ? prr % t.G : 0;
+    const __half *src = a.q + ((size_t)(t.r_beg + jj) * a.Hq + t.kh * t.G + gg) * HD + c * 8;
+    const uint32_t dst = smem_u32(sQ) + (c >> 3) * (kAttnRows * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+    cp_async16z(dst, src, v);
   }
-  auto load_block = [&](int b, int stage) {
-    const uint32_t dK = smem_u32(sK) + stage * TB, dV = smem_u32(sV) + stage * TB;
-    for (int idx = wtid; idx < kAttnBlk * CH; idx += kWorkers) {
-      const int r = idx / CH, c = idx % CH;
-      const int pos = pos_beg + b * kAttnBlk + r;
-      const bool valid = pos < pos_end;
-      const int page = valid ? btab[pos >> 4] : 0;
-      const size_t off = (((size_t)page * a.Hkv + kh) * 16 + (pos & 15)) * HD + c * 8;
-      cp_async16z(dK + swz<HD>(r, c), kp + off, valid);
-      cp_async16z(dV + swz<HD>(r, c), vp + off, valid);
-    }
-  };
-  load_block(0, 0);
-  cp_commit();
+  cp_commit_wait_all();
+  fence_proxy_async_all();   // generic-proxy writes -> tcgen05 (async proxy) reads
+  worker_sync();
+  if (wtid == 0) mbar_arrive(smem_u32(&ctl->q_full));
 
-  float o[HD / 8][4];
-#pragma unroll
-  for (int t = 0; t < HD / 8; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
-  float m_l = -INFINITY, m_h = -INFINITY, l_l = 0.f, l_h = 0.f;
+  const uint32_t tq = tmem_base + ((uint32_t)(q * 32) << 16);
+  const int lim = min(t.len + j, t.pos_end - 1);   // last visible position of this row
   const float scale = rsqrtf((float)HD) * 1.4426950408889634f;
-  const bool warp_active = widx * 16 < rows_here;
+  float acc[OC];
+#pragma unroll
+  for (int i = 0; i < OC; ++i) acc[i] = 0.f;
+  float m_run = -INFINITY, l_run = 0.f, f_pending = 0.f;
+  bool ok = true;
 
-  for (int b = 0; b < nblk; ++b) {
-    const int stage = b & 1;
-    if (b + 1 < nblk) load_block(b + 1, stage ^ 1);
-    cp_commit();
-    cp_wait<1>();
-    worker_sync();
-    if (warp_active) {
-      const uint32_t bK = smem_u32(sK) + stage * TB, bV = smem_u32(sV) + stage * TB;
-      const int mat = lane >> 3;
-#pragma unroll 1
-      for (int sb = 0; sb < 2; ++sb) {
-        float s[4][4];
+  auto consume_o = [&](uint32_t bi, float f) {   // acc = acc * f + O_blk
+    const uint32_t buf = bi & 1;
+    if (ok && !mbar_wait_err(smem_u32(&ctl->o_full[buf]), (bi >> 1) & 1, err)) { ok = false; atomicCAS((int *)err, 0, DEV_TIMEOUT_TMEM); }
+    tc_fence_after();
 #pragma unroll
-        for (int t = 0; t < 4; ++t) s[t][0] = s[t][1] = s[t][2] = s[t][3] = 0.f;
+    for (int i = 0; i < OC / 16; ++i) {
+      uint32_t r[16];
+      tmem_ld16(tq + kColO + buf * HD + half * OC + i * 16, r);
+      tmem_wait_ld();
 #pragma unroll
-        for (int ks = 0; ks < HD / 16; ++ks) {
-          uint32_t qa[4];   // Q fragment of this k-slice, re-read from shared memory to keep registers free
-          ldsm4(smem_u32(sQ) + swz<HD>(widx * 16 + (lane & 7) + 8 * (mat & 1), ks * 2 + (mat >> 1)), qa[0], qa[1], qa[2], qa[3]);
+      for (int e = 0; e < 16; ++e) acc[i * 16 + e] = acc[i * 16 + e] * f + __uint_as_float(r[e]);
+    }
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&ctl->o_empty[buf]));
+  };
+
+  for (int b = 0; b < t.nblk; ++b, ++blk) {
+    const uint32_t buf = blk & 1;
+    if (ok && !mbar_wait_err(smem_u32(&ctl->s_full[buf]), (blk >> 1) & 1, err)) { ok = false; atomicCAS((int *)err, 0, DEV_TIMEOUT_TMEM); }
+    tc_fence_after();
+    const int p_base = t.pos_beg + b * kAttnBlk;
+    float mine[32];
+    float mx = -INFINITY;
 #pragma unroll
-          for (int n2 = 0; n2 < 2; ++n2) {
-            uint32_t k0, k1, k2, k3;
-            ldsm4(bK + swz<HD>(sb * 32 + n2 * 16 + (lane & 7) + 8 * (mat >> 1), ks * 2 + (mat & 1)), k0, k1, k2, k3);
-            mma16816(s[2 * n2], qa, k0, k1);
-            mma16816(s[2 * n2 + 1], qa, k2, k3);
-          }
-        }
-        const int pbase = pos_beg + b * kAttnBlk + sb * 32 + (lane & 3) * 2;
-        float mx_l = -INFINITY, mx_h = -INFINITY;
+    for (int i = 0; i < 4; ++i) {
+      uint32_t r[16];
+      tmem_ld16(tq + kColS + buf * 64 + i * 16, r);
+      tmem_wait_ld();
 #pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          const int q0 = pbase + t * 8;
-          s[t][0] = (q0 <= lim_l) ? s[t][0] * scale : -INFINITY;
-          s[t][1] = (q0 + 1 <= lim_l) ? s[t][1] * scale : -INFINITY;
-          s[t][2] = (q0 <= lim_h) ? s[t][2] * scale : -INFINITY;
-          s[t][3] = (q0 + 1 <= lim_h) ? s[t][3] * scale : -INFINITY;
-          mx_l = fmaxf(mx_l, fmaxf(s[t][0], s[t][1]));
-          mx_h = fmaxf(mx_h, fmaxf(s[t][2], s[t][3]));
-        }
-        mx_l = fmaxf(mx_l, __shfl_xor_sync(0xffffffffu, mx_l, 1));
-        mx_l = fmaxf(mx_l, __shfl_xor_sync(0xffffffffu, mx_l, 2));
-        mx_h = fmaxf(mx_h, __shfl_xor_sync(0xffffffffu, mx_h, 1));
-        mx_h = fmaxf(mx_h, __shfl_xor_sync(0xffffffffu, mx_h, 2));
-        const float mn_l = fmaxf(m_l, mx_l), mn_h = fmaxf(m_h, mx_h);
-        const float ref_l = (mn_l == -INFINITY) ? 0.f : mn_l, ref_h = (mn_h == -INFINITY) ? 0.f : mn_h;
-        const float f_l = exp2f(m_l - ref_l), f_h = exp2f(m_h - ref_h);   // exp2(-inf) = 0 on the first block
-        m_l = mn_l; m_h = mn_h;
-        l_l *= f_l; l_h *= f_h;
-#pragma unroll
-        for (int t = 0; t < HD / 8; ++t) { o[t][0] *= f_l; o[t][1] *= f_l; o[t][2] *= f_h; o[t][3] *= f_h; }
-        uint32_t pa[2][4];
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          const float e0 = exp2f(s[t][0] - ref_l), e1 = exp2f(s[t][1] - ref_l);
-          const float e2 = exp2f(s[t][2] - ref_h), e3 = exp2f(s[t][3] - ref_h);
-          l_l += e0 + e1;
-          l_h += e2 + e3;
-          pa[t >> 1][(t & 1) * 2 + 0] = pack_h2(e0, e1);
-          pa[t >> 1][(t & 1) * 2 + 1] = pack_h2(e2, e3);
-        }
-#pragma unroll
-        for (int kt = 0; kt < 2; ++kt) {
-#pragma unroll
-          for (int d2 = 0; d2 < HD / 16; ++d2) {
-            uint32_t v0, v1, v2, v3;
-            ldsm4t(bV + swz<HD>(sb * 32 + kt * 16 + (lane & 7) + 8 * (mat & 1), d2 * 2 + (mat >> 1)), v0, v1, v2, v3);
-            mma16816(o[2 * d2], pa[kt], v0, v1);
-            mma16816(o[2 * d2 + 1], pa[kt], v2, v3);
-          }
-        }
+      for (int e = 0; e < 16; ++e) {
+        const float sv = (p_base + i * 16 + e <= lim) ? __uint_as_float(r[e]) * scale : -INFINITY;
+        mx = fmaxf(mx, sv);
+        if ((i >> 1) == half) mine[(i & 1) * 16 + e] = sv;
       }
     }
-    worker_sync();
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&ctl->s_empty[buf]));
+    const float m_new = fmaxf(m_run, mx);
+    const float ref = (m_new == -INFINITY) ? 0.f : m_new;
+    const float f = exp2f(m_run - ref);   // exp2(-inf) = 0 on the first block
+    m_run = m_new;
+    uint32_t pk[16];
+    float sum = 0.f;
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      const float e0 = exp2f(mine[2 * e] - ref), e1 = exp2f(mine[2 * e + 1] - ref);
+      sum += e0 + e1;
+      pk[e] = pack_h2(e0, e1);
+    }
+    l_run = l_run * f + sum;
+    // the P buffer is free: the product that read it two blocks ago was seen complete when its O_blk was taken
+    tmem_st16(tq + kColP + buf * 32 + half * 16, pk);
+    tmem_wait_st();
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&ctl->p_full[buf]));
+    if (b > 0) consume_o(blk - 1, f_pending);
+    f_pending = f;
   }
-  cp_wait<0>();
+  consume_o(blk - 1, f_pending);
+  if (!worker_all(ok)) return false;
 
-  l_l += __shfl_xor_sync(0xffffffffu, l_l, 1);
-  l_l += __shfl_xor_sync(0xffffffffu, l_l, 2);
-  l_h += __shfl_xor_sync(0xffffffffu, l_h, 1);
-  l_h += __shfl_xor_sync(0xffffffffu, l_h, 2);
-  if (vl) {
-    const size_t ob = out_base(prl);
-    if ((lane & 3) == 0) a.attn_ml[ob] = make_float2(m_l, l_l);
-    float *dst = a.attn_o + ob * HD + (lane & 3) * 2;
+  // ---- partial result of this split: un-normalised output, running max (log2 domain), sum -----------------
+  if (half == 1) ctl->l_half[row] = l_run;
+  worker_sync();
+  if (valid) {
+    if (half == 0) a.attn_ml[ob] = make_float2(m_run, l_run + ctl->l_half[row]);
+    float4 *dst = reinterpret_cast<float4 *>(a.attn_o + ob * HD + half * OC);
 #pragma unroll
-    for (int t = 0; t < HD / 8; ++t) *reinterpret_cast<float2 *>(dst + t * 8) = make_float2(o[t][0], o[t][1]);
+    for (int i = 0; i < OC / 4; ++i) dst[i] = make_float4(acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3]);
   }
-  if (vh) {
-    const size_t ob = out_base(prh);
-    if ((lane & 3) == 0) a.attn_ml[ob] = make_float2(m_h, l_h);
-    float *dst = a.attn_o + ob * HD + (lane & 3) * 2;
-#pragma unroll
-    for (int t = 0; t < HD / 8; ++t) *reinterpret_cast<float2 *>(dst + t * 8) = make_float2(o[t][2], o[t][3]);
-  }
+  return true;
 }
 
 // Merge the splits of one (row, query head): one warp per pair, lane <-> split for the weights.
@@ -534,8 +502,9 @@ __global__ void __launch_bounds__(kThreads, 1) fused_verify_kernel(const __grid_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t c = blockIdx.x, n = gridDim.x;
   const int ncols = a.planes * a.Mc;        // accumulator columns of one buffer
-  uint32_t alloc_cols = 32;
-  while (alloc_cols < (uint32_t)(kAccBufs * ncols)) alloc_cols <<= 1;
+  // all of tensor memory: the projection accumulators (kAccBufs * ncols columns) and, over them, the
+  // attention buffers (kColO + 2 * head_dim columns)
+  const uint32_t alloc_cols = 512;
   int *ctr = a.sync, *err = a.err;
   const int n_gemms = 4 * a.n_layers + (a.skip_lm ? 0 : 1);
 
@@ -548,6 +517,16 @@ __global__ void __launch_bounds__(kThreads, 1) fused_verify_kernel(const __grid_
       mbar_init(smem_u32(&ctl->tmem_full[b]), 1);
       mbar_init(smem_u32(&ctl->tmem_empty[b]), 8);   // one arrival per worker warp
     }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&ctl->kv_full[b]), 1);    // producer's expect_tx arrival
+      mbar_init(smem_u32(&ctl->kv_empty[b]), 1);   // tcgen05.commit after P V
+      mbar_init(smem_u32(&ctl->s_full[b]), 1);
+      mbar_init(smem_u32(&ctl->s_empty[b]), 8);
+      mbar_init(smem_u32(&ctl->p_full[b]), 8);
+      mbar_init(smem_u32(&ctl->o_full[b]), 1);
+      mbar_init(smem_u32(&ctl->o_empty[b]), 8);
+    }
+    mbar_init(smem_u32(&ctl->q_full), 1);
     ctl->flag = 0;
     ctl->attn_epoch = 0;
     fence_barrier_init();
@@ -618,8 +597,40 @@ __global__ void __launch_bounds__(kThreads, 1) fused_verify_kernel(const __grid_
       uint32_t round_par = 0;
       int slot = 0;
       bool ok = true;
+      uint32_t blk = 0;
       for (int g = 0; g < n_gemms && ok; ++g) {
         const OpInfo o = gemm_op(a, g);
+        if (o.op == OP_O) {
+          // ---- attention of this layer: stream the K/V blocks of this CTA's units ---------------------
+          ok = grid_wait(ctr, (o.phase - 2) * (int)n, err);   // the QKV phase (rotary, KV append) is complete everywhere
+          if (!ok) { atomicCAS(err, 0, DEV_TIMEOUT_GRID); break; }
+          fence_proxy_async_all();
+          const int n_units = a.n_attn_tiles * a.Hkv * a.attn_splits;
+          const int halves = a.hd / 64;
+          const uint32_t kv_bytes = 2u * kAttnBlk * a.hd * 2;
+          for (int u = (int)c; u < n_units && ok; u += (int)n) {
+            const AttnUnit t = attn_unit_info(a, u);
+            const int32_t *btab = a.in.block_tab + (size_t)t.seq * a.in.pages_per_seq;
+            for (int b = 0; b < t.nblk; ++b, ++blk) {
+              const uint32_t st = blk & 1;
+              if (!mbar_wait_err(smem_u32(&ctl->kv_empty[st]), ((blk >> 1) & 1) ^ 1, err)) { ok = false; atomicCAS(err, 0, DEV_TIMEOUT_EMPTY); break; }
+              const uint32_t bar = smem_u32(&ctl->kv_full[st]);
+              mbar_expect_tx(bar, kv_bytes);
+              uint8_t *sK = attn_sm + kAttnRows * a.hd * 2 + st * kv_bytes, *sV = sK + kAttnBlk * a.hd * 2;
+              for (int pg = 0; pg < kAttnBlk / 16; ++pg) {
+                // a page past the split's end is never visible; load the last visible page again instead
+                const int pos = min(t.pos_beg + b * kAttnBlk + pg * 16, t.pos_end - 1);
+                const int page = btab[pos >> 4];
+                for (int hh = 0; hh < halves; ++hh) {
+                  const uint32_t off = hh * (kAttnBlk * 128) + pg * 2048;
+                  tma_load_5d(smem_u32(sK + off), &a.maps[a.map_kv], hh * 64, 0, t.kh, page, 2 * o.layer, bar, pol_a);
+                  tma_load_5d(smem_u32(sV + off), &a.maps[a.map_kv], hh * 64, 0, t.kh, page, 2 * o.layer + 1, bar, pol_a);
+                }
+              }
+            }
+          }
+          if (!ok) break;
+        }
         SegmentIter sit(c, o.T, o.KB, n);
         Segment sg;
         bool first = true;
@@ -654,8 +665,55 @@ __global__ void __launch_bounds__(kThreads, 1) fused_verify_kernel(const __grid_
       uint32_t seg = 0, round_par = 0;
       int slot = 0;
       bool ok = true;
+      uint32_t blk = 0, unit_no = 0;
+      const uint32_t idesc_qk = umma_idesc_f16(kAttnRows, kAttnBlk, 0);
+      const uint32_t idesc_pv = umma_idesc_f16(kAttnRows, (uint32_t)a.hd, 1);
       for (int g = 0; g < n_gemms && ok; ++g) {
         const OpInfo o = gemm_op(a, g);
+        if (o.op == OP_O) {
+          // ---- attention of this layer --------------------------------------------------------------
+          const int n_units = a.n_attn_tiles * a.Hkv * a.attn_splits;
+          const int halves = a.hd / 64;
+          const uint32_t kv_bytes = 2u * kAttnBlk * a.hd * 2;
+          const uint32_t sQ = smem_u32(attn_sm);
+          auto issue_pv = [&](uint32_t bi) -> bool {   // O_blk = P V for block number bi
+            const uint32_t pb = bi & 1;
+            if (!mbar_wait_err(smem_u32(&ctl->p_full[pb]), (bi >> 1) & 1, err)) return false;
+            if (!mbar_wait_err(smem_u32(&ctl->o_empty[pb]), ((bi >> 1) & 1) ^ 1, err)) return false;
+            tc_fence_after();
+            const uint32_t sV = sQ + kAttnRows * a.hd * 2 + pb * kv_bytes + kAttnBlk * a.hd * 2;
+#pragma unroll
+            for (int ks = 0; ks < kAttnBlk / 16; ++ks)   // 16 positions per instruction
+              umma_f16_ts(tmem_base + kColO + pb * a.hd, tmem_base + kColP + pb * 32 + ks * 8,
+                          umma_desc_sw128_mn(sV + ks * 2048, kAttnBlk * 128), idesc_pv, ks > 0 ? 1u : 0u);
+            umma_commit(smem_u32(&ctl->o_full[pb]));
+            umma_commit(smem_u32(&ctl->kv_empty[pb]));
+            return true;
+          };
+          for (int u = (int)c; u < n_units && ok; u += (int)n) {
+            const AttnUnit t = attn_unit_info(a, u);
+            if (t.nblk == 0) continue;
+            if (!mbar_wait_err(smem_u32(&ctl->q_full), unit_no & 1, err)) { ok = false; break; }
+            ++unit_no;
+            for (int b = 0; b < t.nblk && ok; ++b, ++blk) {
+              const uint32_t st = blk & 1;
+              if (!mbar_wait_err(smem_u32(&ctl->kv_full[st]), (blk >> 1) & 1, err)) { ok = false; break; }
+              if (!mbar_wait_err(smem_u32(&ctl->s_empty[st]), ((blk >> 1) & 1) ^ 1, err)) { ok = false; break; }
+              tc_fence_after();
+              const uint32_t sK = sQ + kAttnRows * a.hd * 2 + st * kv_bytes;
+              for (int hh = 0; hh < halves; ++hh) {
+                const uint64_t dq = umma_desc_sw128(sQ + hh * (kAttnRows * 128)), dk = umma_desc_sw128(sK + hh * (kAttnBlk * 128));
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                  umma_bf16(tmem_base + kColS + st * 64, dq + 2 * kk, dk + 2 * kk, idesc_qk, (hh | kk) != 0 ? 1u : 0u);
+              }
+              umma_commit(smem_u32(&ctl->s_full[st]));
+              if (b > 0) ok = issue_pv(blk - 1);
+            }
+            if (ok) ok = issue_pv(blk - 1);
+          }
+          if (!ok) break;
+        }
         SegmentIter sit(c, o.T, o.KB, n);
         Segment sg;
         while (ok && sit.next(&sg)) {
@@ -693,7 +751,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_verify_kernel(const __grid_
     const int q = warp & 3;                        // tensor-memory lane quarter this warp may read
     const int half = widx >> 2;
     const uint32_t tq = tmem_base + ((uint32_t)(q * 32) << 16);
-    uint32_t seg = 0;
+    uint32_t seg = 0, attn_blk = 0;
     int ss_buf = 0;
     int phase = 0;      // phases completed by this CTA
     bool ok = true;
@@ -837,13 +895,12 @@ __global__ void __launch_bounds__(kThreads, 1) fused_verify_kernel(const __grid_
       if (!wait_phases(phase)) { ok = false; break; }
       {
         const int n_units = a.n_attn_tiles * a.Hkv * a.attn_splits;
-        for (int u = (int)c; u < n_units; u += (int)n) {
-          const int split = u % a.attn_splits;
-          const int kh = (u / a.attn_splits) % a.Hkv;
-          const int tile = u / (a.attn_splits * a.Hkv);
-          if (a.hd == 128) attn_unit<128>(a, l, attn_sm, tile, kh, split, widx, lane, wtid);
-          else attn_unit<64>(a, l, attn_sm, tile, kh, split, widx, lane, wtid);
+        for (int u = (int)c; u < n_units && ok; u += (int)n) {
+          const AttnUnit t = attn_unit_info(a, u);
+          ok = (a.hd == 128) ? attn_unit_workers<128>(a, ctl, t, attn_sm, tmem_base, q, half, lane, wtid, attn_blk, 0, err)
+                             : attn_unit_workers<64>(a, ctl, t, attn_sm, tmem_base, q, half, lane, wtid, attn_blk, 0, err);
         }
+        if (!ok) break;
       }
       fence_proxy_async_all();   // generic-proxy use of the staging area is over before TMA writes there again
       worker_sync();
@@ -915,6 +972,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_verify_kernel(const __grid_
 }
 
 // ---- host side ----------------------------------------------------------------------------------------------
+// Q tile + two stages of (K block, V block)
 size_t fused_attn_smem_bytes(int hd) { return (size_t)kAttnRows * hd * 2 + (size_t)4 * kAttnBlk * hd * 2; }
 
 int fused_ring_stages(int planes, int Mc, int hd, size_t smem_limit) {

@@ -110,6 +110,7 @@ struct FusedArgs {
   // tensor maps in device memory: 4 per layer (qkv, o, gate-up, down), LM head, then per row-chunk
   // size three activation maps (h, attn, act)
   const CUtensorMap *maps;
+  int map_kv;                    // index of the 5-d map over the paged KV pool (64 elements x 16 positions x head x page x layer*2)
   const __nv_bfloat16 *embed;
   const float *gains;            // g1[0], g2[0], g1[1], ..., gf; gain_stride floats apart
   int gain_stride;

@@ -140,7 +140,7 @@ void make_layout(const ts_model_config &c, Layout *L) {
   L->out_ints = io;
   L->d_in = take((uint64_t)L->in_ints * 4);
   L->d_out = take((uint64_t)L->out_ints * 4);
-  L->n_maps = 4 * c.n_layers + 1 + 3 * 3;
+  L->n_maps = 4 * c.n_layers + 1 + 3 * 3 + 1;
   L->maps = take((uint64_t)L->n_maps * sizeof(CUtensorMap));
   L->slab = take((uint64_t)kMaxFusedCtas * 2 * kFusedMaxRows * 128 * 4);
   L->ss_part = take((uint64_t)(d / 128) * R * 4);
@@ -328,6 +328,7 @@ ts_status run_step_fused(ts_model *m) {
   }
   a.tile_seq = di + L.o_tile128_seq; a.tile_row0 = di + L.o_tile128_row0;
   a.maps = (const CUtensorMap *)m->WS(L.maps);
+  a.map_kv = L.n_maps - 1;
   a.embed = (const __nv_bfloat16 *)m->W(L.embed);
   a.gains = (const float *)m->W(L.g1[0]);
   a.gain_stride = (int)(align_up((uint64_t)c.d_model * 4, 1024) / 4);
@@ -635,6 +636,22 @@ ts_status ts_init_model(const ts_model_config *cfg, const ts_buffers *bufs, void
       maps[4 * c.n_layers + 1 + 3 * i + 1] = m->tm_attn[i];
       maps[4 * c.n_layers + 1 + 3 * i + 2] = m->tm_act[i];
     }
+    {
+      // paged KV pool as a 5-d tensor: 64-element half of a head row, 16 positions of a page, kv head, page,
+      // (layer, K|V); one box = one page of one head = 16 rows of 128 bytes
+      const uint64_t hd = c.head_dim, page_bytes = (uint64_t)c.n_kv_heads * TS_PAGE_SIZE * hd * 2;
+      cuuint64_t gdim[5] = {hd, TS_PAGE_SIZE, (cuuint64_t)c.n_kv_heads, (cuuint64_t)c.max_pages, (cuuint64_t)2 * c.n_layers};
+      cuuint64_t gstr[4] = {hd * 2, TS_PAGE_SIZE * hd * 2, page_bytes, (cuuint64_t)c.max_pages * page_bytes};
+      cuuint32_t box[5] = {64, TS_PAGE_SIZE, 1, 1, 1}, es[5] = {1, 1, 1, 1, 1};
+      CUresult r = enc(&maps[L.n_maps - 1], CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, bufs->kv_pool, gdim, gstr, box, es,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      if (r != CUDA_SUCCESS) return bail(fail(TS_ERR_CUDA, "cuTensorMapEncodeTiled(kv pool) failed with code %d", (int)r));
+    }
+    // Attention multiplies masked positions by zero, so every cache position that can be read must hold a
+    // finite value: start from an all-zero pool.
+    e = cudaMemsetAsync(bufs->kv_pool, 0, L.kv_bytes, m->st);
+    if (e != cudaSuccess) return bail(fail(TS_ERR_CUDA, "cudaMemsetAsync(kv pool): %s", cudaGetErrorString(e)));
     e = cudaMemcpyAsync(m->WS(L.maps), maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, m->st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(m->st);
     if (e != cudaSuccess) return bail(fail(TS_ERR_CUDA, "tensor map upload: %s", cudaGetErrorString(e)));
