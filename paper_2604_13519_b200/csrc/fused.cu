@@ -44,6 +44,7 @@ static constexpr int kMaxMc = 64;
 static constexpr int kAccBufs = 4;      // accumulator buffers in tensor memory (4 x 128 columns at most)
 static constexpr int kAttnRows = 128;   // packed (position, query head) rows per attention unit
 static constexpr int kAttnBlk = 64;     // kv positions per staged block
+static constexpr int kKvStages = 4;     // K/V blocks in flight per CTA during attention
 
 enum : int { OP_QKV = 0, OP_O = 1, OP_GU = 2, OP_D = 3, OP_LM = 4, OP_EMBED = 5 };
 
@@ -56,13 +57,14 @@ struct __align__(16) FusedCtl {
   int flag;
   int attn_epoch;            // attention phases this CTA has finished (ring slots under the staging area are free)
   // attention pipeline: K/V stages (TMA -> MMA), Q tile, score / probability / output-block buffers
-  uint64_t kv_full[2], kv_empty[2], q_full;
+  uint64_t kv_full[kKvStages], kv_empty[kKvStages], q_full;
   uint64_t s_full[2], s_empty[2], p_full[2], o_full[2], o_empty[2];
   float l_half[kAttnRows];
   int row_pos[kMaxMc];       // absolute position of each row
   int row_page[kMaxMc];      // KV page holding that position
   float r_s[kMaxMc];
   float ss_acc[2][4][kMaxMc];
+  FusedArgs args;            // copy of the kernel arguments: cheap to read from the out-of-line device functions
 };
 
 // ---- small device helpers ---------------------------------------------------------------------------
@@ -457,18 +459,29 @@ __device__ __forceinline__ void merge_unit(const FusedArgs &a, int m, int h, int
   float acc[EPL];
 #pragma unroll
   for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-  for (int s = 0; s < S; ++s) {
-    const float ws = __shfl_sync(0xffffffffu, w, s);
-    if (ws != 0.f) {
-      const float *src = a.attn_o + (base + s) * HD + lane * EPL;
+  // eight splits' loads in flight at a time (an empty split never wrote its slot: it is not read)
+  for (int s0 = 0; s0 < S; s0 += 8) {
+    float ws[8];
+    float t[8][EPL];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      ws[u] = __shfl_sync(0xffffffffu, w, (s0 + u) & 31);
+      if (s0 + u >= S) ws[u] = 0.f;
+      const float *src = a.attn_o + (base + s0 + u) * HD + lane * EPL;
       if constexpr (EPL == 4) {
-        const float4 t = __ldcg(reinterpret_cast<const float4 *>(src));
-        acc[0] += ws * t.x; acc[1] += ws * t.y; acc[2] += ws * t.z; acc[3] += ws * t.w;
+        float4 x4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (ws[u] != 0.f) x4 = __ldcg(reinterpret_cast<const float4 *>(src));
+        t[u][0] = x4.x; t[u][1] = x4.y; t[u][2] = x4.z; t[u][3] = x4.w;
       } else {
-        const float2 t = __ldcg(reinterpret_cast<const float2 *>(src));
-        acc[0] += ws * t.x; acc[1] += ws * t.y;
+        float2 x2 = make_float2(0.f, 0.f);
+        if (ws[u] != 0.f) x2 = __ldcg(reinterpret_cast<const float2 *>(src));
+        t[u][0] = x2.x; t[u][1] = x2.y;
       }
     }
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) acc[e] += ws[u] * t[u][e];
   }
   const size_t ld = (size_t)a.Hq * HD;
   const size_t col = (size_t)h * HD + lane * EPL;
@@ -508,6 +521,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_verify_kernel(const __grid_
   int *ctr = a.sync, *err = a.err;
   const int n_gemms = 4 * a.n_layers + (a.skip_lm ? 0 : 1);
 
+  for (int i = threadIdx.x; i < (int)(sizeof(FusedArgs) / 4); i += kThreads)
+    reinterpret_cast<uint32_t *>(&ctl->args)[i] = reinterpret_cast<const uint32_t *>(&a)[i];
   if (threadIdx.x == 0) {
     for (int s = 0; s < R; ++s) {
       mbar_init(smem_u32(&ctl->full[s]), 2);    // weight producer + activation producer
@@ -517,9 +532,11 @@ __global__ void __launch_bounds__(kThreads, 1) fused_verify_kernel(const __grid_
       mbar_init(smem_u32(&ctl->tmem_full[b]), 1);
       mbar_init(smem_u32(&ctl->tmem_empty[b]), 8);   // one arrival per worker warp
     }
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < kKvStages; ++b) {
       mbar_init(smem_u32(&ctl->kv_full[b]), 1);    // producer's expect_tx arrival
       mbar_init(smem_u32(&ctl->kv_empty[b]), 1);   // tcgen05.commit after P V
+    }
+    for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&ctl->s_full[b]), 1);
       mbar_init(smem_u32(&ctl->s_empty[b]), 8);
       mbar_init(smem_u32(&ctl->p_full[b]), 8);
@@ -612,8 +629,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_verify_kernel(const __grid_
             const AttnUnit t = attn_unit_info(a, u);
             const int32_t *btab = a.in.block_tab + (size_t)t.seq * a.in.pages_per_seq;
             for (int b = 0; b < t.nblk; ++b, ++blk) {
-              const uint32_t st = blk & 1;
-              if (!mbar_wait_err(smem_u32(&ctl->kv_empty[st]), ((blk >> 1) & 1) ^ 1, err)) { ok = false; atomicCAS(err, 0, DEV_TIMEOUT_EMPTY); break; }
+              const uint32_t st = blk % kKvStages;
+              if (!mbar_wait_err(smem_u32(&ctl->kv_empty[st]), ((blk / kKvStages) & 1) ^ 1, err)) { ok = false; atomicCAS(err, 0, DEV_TIMEOUT_EMPTY); break; }
               const uint32_t bar = smem_u32(&ctl->kv_full[st]);
               mbar_expect_tx(bar, kv_bytes);
               uint8_t *sK = attn_sm + kAttnRows * a.hd * 2 + st * kv_bytes, *sV = sK + kAttnBlk * a.hd * 2;
@@ -681,13 +698,14 @@ __global__ void __launch_bounds__(kThreads, 1) fused_verify_kernel(const __grid_
             if (!mbar_wait_err(smem_u32(&ctl->p_full[pb]), (bi >> 1) & 1, err)) return false;
             if (!mbar_wait_err(smem_u32(&ctl->o_empty[pb]), ((bi >> 1) & 1) ^ 1, err)) return false;
             tc_fence_after();
-            const uint32_t sV = sQ + kAttnRows * a.hd * 2 + pb * kv_bytes + kAttnBlk * a.hd * 2;
+            const uint32_t vst = bi % kKvStages;
+            const uint32_t sV = sQ + kAttnRows * a.hd * 2 + vst * kv_bytes + kAttnBlk * a.hd * 2;
 #pragma unroll
             for (int ks = 0; ks < kAttnBlk / 16; ++ks)   // 16 positions per instruction
               umma_f16_ts(tmem_base + kColO + pb * a.hd, tmem_base + kColP + pb * 32 + ks * 8,
                           umma_desc_sw128_mn(sV + ks * 2048, kAttnBlk * 128), idesc_pv, ks > 0 ? 1u : 0u);
             umma_commit(smem_u32(&ctl->o_full[pb]));
-            umma_commit(smem_u32(&ctl->kv_empty[pb]));
+            umma_commit(smem_u32(&ctl->kv_empty[vst]));
             return true;
           };
           for (int u = (int)c; u < n_units && ok; u += (int)n) {
@@ -696,11 +714,11 @@ __global__ void __launch_bounds__(kThreads, 1) fused_verify_kernel(const __grid_
             if (!mbar_wait_err(smem_u32(&ctl->q_full), unit_no & 1, err)) { ok = false; break; }
             ++unit_no;
             for (int b = 0; b < t.nblk && ok; ++b, ++blk) {
-              const uint32_t st = blk & 1;
-              if (!mbar_wait_err(smem_u32(&ctl->kv_full[st]), (blk >> 1) & 1, err)) { ok = false; break; }
+              const uint32_t kst = blk % kKvStages, st = blk & 1;
+              if (!mbar_wait_err(smem_u32(&ctl->kv_full[kst]), (blk / kKvStages) & 1, err)) { ok = false; break; }
               if (!mbar_wait_err(smem_u32(&ctl->s_empty[st]), ((blk >> 1) & 1) ^ 1, err)) { ok = false; break; }
               tc_fence_after();
-              const uint32_t sK = sQ + kAttnRows * a.hd * 2 + st * kv_bytes;
+              const uint32_t sK = sQ + kAttnRows * a.hd * 2 + kst * kv_bytes;
               for (int hh = 0; hh < halves; ++hh) {
                 const uint64_t dq = umma_desc_sw128(sQ + hh * (kAttnRows * 128)), dk = umma_desc_sw128(sK + hh * (kAttnBlk * 128));
 #pragma unroll
@@ -897,8 +915,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_verify_kernel(const __grid_
         const int n_units = a.n_attn_tiles * a.Hkv * a.attn_splits;
         for (int u = (int)c; u < n_units && ok; u += (int)n) {
           const AttnUnit t = attn_unit_info(a, u);
-          ok = (a.hd == 128) ? attn_unit_workers<128>(a, ctl, t, attn_sm, tmem_base, q, half, lane, wtid, attn_blk, 0, err)
-                             : attn_unit_workers<64>(a, ctl, t, attn_sm, tmem_base, q, half, lane, wtid, attn_blk, 0, err);
+          ok = (a.hd == 128) ? attn_unit_workers<128>(ctl->args, ctl, t, attn_sm, tmem_base, q, half, lane, wtid, attn_blk, 0, err)
+                             : attn_unit_workers<64>(ctl->args, ctl, t, attn_sm, tmem_base, q, half, lane, wtid, attn_blk, 0, err);
         }
         if (!ok) break;
       }
@@ -972,14 +990,15 @@ __global__ void __launch_bounds__(kThreads, 1) fused_verify_kernel(const __grid_
 }
 
 // ---- host side ----------------------------------------------------------------------------------------------
-// Q tile + two stages of (K block, V block)
-size_t fused_attn_smem_bytes(int hd) { return (size_t)kAttnRows * hd * 2 + (size_t)4 * kAttnBlk * hd * 2; }
+// Q tile + kKvStages stages of (K block, V block)
+size_t fused_attn_smem_bytes(int hd) { return (size_t)kAttnRows * hd * 2 + (size_t)kKvStages * 2 * kAttnBlk * hd * 2; }
 
 int fused_ring_stages(int planes, int Mc, int hd, size_t smem_limit) {
   const size_t stage = kWBytes + (size_t)planes * Mc * kBlockK * 2;
   const size_t fixed = 1024 + sizeof(FusedCtl) + 256;
-  if (smem_limit < fixed + fused_attn_smem_bytes(hd) + 2 * stage) return 0;
-  return (int)std::min<size_t>(kMaxRing, (smem_limit - fixed) / stage);
+  if (smem_limit < fixed + 2 * stage) return 0;
+  const size_t ring = std::min<size_t>(kMaxRing, (smem_limit - fixed) / stage);
+  return ring * stage >= fused_attn_smem_bytes(hd) ? (int)ring : 0;   // the attention staging area lies over the ring
 }
 
 cudaError_t launch_fused(FusedArgs a, size_t smem_limit, cudaStream_t st) {
