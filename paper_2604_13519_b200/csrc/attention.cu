@@ -264,11 +264,18 @@ __global__ void attn_combine_kernel(const AttnArgs a) {
   }
   __syncthreads();
   pdl_launch_dependents();
+  // eight splits' loads in flight at a time (an empty split never wrote its slot: it is not read)
   float num = 0.f;
-#pragma unroll 8
-  for (int s = 0; s < a.n_splits; ++s) {
-    const float w = w_s[s];
-    if (w != 0.f) num += w * a.part_o[(base + s) * a.hd + d];
+  for (int s0 = 0; s0 < a.n_splits; s0 += 8) {
+    float w[8], t[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      w[u] = (s0 + u < a.n_splits) ? w_s[s0 + u] : 0.f;
+      t[u] = 0.f;
+      if (w[u] != 0.f) t[u] = a.part_o[(base + s0 + u) * a.hd + d];
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) num += w[u] * t[u];
   }
   __nv_bfloat16 hi, lo;
   split_bf16(num, hi, lo);

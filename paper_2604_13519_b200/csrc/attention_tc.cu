@@ -1,0 +1,372 @@
+// Paged grouped-query attention of the verify chunk on the 5th-generation tensor cores, as a kernel of its own.
+//
+// One CTA = one unit: (128-row tile of packed (position, query head) rows, kv head, split of the KV positions).
+//   warp 0   K/V producer: TMA loads of 64-position blocks straight from the pages (5-d tensor map over the pool)
+//   warp 1   tensor memory allocation + tcgen05.mma issue:  S = Q K^T  (Q tile and K block K-major in shared
+//            memory, 128 x 64 fp32 result in tensor memory), then  O_blk = P V  with P read from tensor memory
+//            (fp16) and the V block read MN-major from the same [position][64 elements] image K uses
+//   warps 2..5  one row per thread: running max over the block's 64 scores, P = exp2(S - max) written back to
+//            tensor memory as fp16, O_blk added into registers with the running-softmax rescale
+// Each split writes an un-normalised partial output with its (max, sum); attn_combine_kernel merges the splits.
+// Every wait is bounded; on expiry the CTA records an error word and leaves through the normal exit.
+#include <cuda_fp16.h>
+
+#include "kernels.h"
+#include "schedule.h"
+
+namespace ts {
+
+static constexpr int kAttnRows = 128;   // packed rows per unit
+static constexpr int kAttnBlk = 64;     // kv positions per block
+static constexpr int kKvStages = 4;     // K/V blocks in flight
+static constexpr int kTcThreads = 192;
+static constexpr int kWorkers = 128;
+static constexpr int kWorkerWarp0 = 2;
+
+struct __align__(16) AttnCtl {
+  uint64_t kv_full[kKvStages], kv_empty[kKvStages], q_full;
+  uint64_t s_full[2], s_empty[2], p_full[2], o_full[2], o_empty[2];
+  uint32_t tmem_base;
+};
+
+__device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ bool worker_all(bool ok) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\tbar.red.and.pred q, 1, 128, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(r)
+      : "r"((uint32_t)ok)
+      : "memory");
+  return r != 0;
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ bool mbar_wait_err(uint32_t bar, uint32_t parity, const int *err) {
+  uint64_t t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 255u) {
+      if (*reinterpret_cast<const volatile int *>(err) != 0) return false;
+      const uint64_t now = global_timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > 2000000000ull) return false;
+      __nanosleep(32);
+    }
+  }
+}
+
+struct AttnUnit {
+  int tile, kh, split;
+  int seq, row0, rows_here, r_beg, len, G;
+  int pos_beg, pos_end, nblk;
+};
+
+__device__ __forceinline__ AttnUnit attn_unit_info(const AttnTcArgs &a, int u) {
+  AttnUnit t;
+  t.split = u % a.attn_splits;
+  t.kh = (u / a.attn_splits) % a.Hkv;
+  t.tile = u / (a.attn_splits * a.Hkv);
+  t.G = a.Hq / a.Hkv;
+  t.seq = a.tile_seq[t.tile];
+  t.row0 = a.tile_row0[t.tile];
+  t.r_beg = a.in.cu_rows[t.seq];
+  const int k_i = a.in.cu_rows[t.seq + 1] - t.r_beg;
+  t.len = a.in.seq_len[t.seq];
+  t.rows_here = min(kAttnRows, k_i * t.G - t.row0);
+  const int total = t.len + k_i;
+  const int j_max = (t.row0 + t.rows_here - 1) / t.G;
+  int p0, p1;
+  split_pages((total + 15) >> 4, a.attn_splits, t.split, &p0, &p1);
+  t.pos_beg = p0 << 4;
+  t.pos_end = min(min(p1 << 4, total), t.len + j_max + 1);   // nothing beyond the last row's own position is visible
+  t.nblk = t.pos_end > t.pos_beg ? (t.pos_end - t.pos_beg + kAttnBlk - 1) / kAttnBlk : 0;
+  return t;
+}
+
+// tensor-memory columns of the attention phase (they lie over the projection accumulators, which are idle then)
+static constexpr int kColS = 0;      // two score buffers of 64 columns
+static constexpr int kColP = 128;    // two probability buffers of 32 columns (fp16 pairs)
+static constexpr int kColO = 192;    // two output-block buffers of head_dim columns
+
+__device__ __forceinline__ void cp_async16z(uint32_t dst, const void *src, bool valid) {
+  const int sz = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_commit_wait_all() {
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t pack_h2(float x, float y) {
+  __half2 v = __floats2half2_rn(x, y);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// Worker side of one unit.  Thread <-> row (tensor-memory lane q*32 + lane): it takes the row maximum over the
+// block's 64 scores, writes the 64 probabilities back as fp16 and keeps the head_dim output sums in registers.
+// `blk` counts K/V blocks over all units of this CTA (buffer index and barrier parity come from it).
+template <int HD>
+__device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *ctl, const AttnUnit &t, uint8_t *sQ, uint32_t tmem_base,
+                                                  int q, int lane, int wtid, uint32_t &blk, const int *err) {
+  constexpr int CH = HD / 8;          // 16-byte chunks per row
+  const int row = q * 32 + lane;      // row of the tile
+  const int pr = t.row0 + row;        // packed row of the sequence
+  const bool valid = row < t.rows_here;
+  const int j = valid ? pr / t.G : 0, gq = valid ? pr % t.G : 0;
+  const size_t ob = ((size_t)(t.r_beg + j) * a.Hq + t.kh * t.G + gq) * a.attn_splits + t.split;
+  if (t.nblk == 0) {   // nothing visible in this split: mark it empty
+    if (valid) a.attn_ml[ob] = make_float2(-INFINITY, 0.f);
+    return true;
+  }
+  // ---- stage Q: [128 rows][64 elements] images with the 128-byte swizzle, one per 64-element half ----------
+  for (int idx = wtid; idx < kAttnRows * CH; idx += kWorkers) {
+    const int r = idx / CH, c = idx % CH;
+    const int prr = t.row0 + r;
+    const bool v = r < t.rows_here;
+    const int jj = v ? prr / t.G : 0, gg = v ? prr % t.G : 0;
+    const __half *src = a.q + ((size_t)(t.r_beg + jj) * a.Hq + t.kh * t.G + gg) * HD + c * 8;
+    const uint32_t dst = smem_u32(sQ) + (c >> 3) * (kAttnRows * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+    cp_async16z(dst, src, v);
+  }
+  cp_commit_wait_all();
+  fence_proxy_async_all();   // generic-proxy writes -> tcgen05 (async proxy) reads
+  worker_sync();
+  if (wtid == 0) mbar_arrive(smem_u32(&ctl->q_full));
+
+  const uint32_t tq = tmem_base + ((uint32_t)(q * 32) << 16);
+  const int lim = min(t.len + j, t.pos_end - 1);   // last visible position of this row
+  const float scale = rsqrtf((float)HD) * 1.4426950408889634f;
+  float acc[HD];
+#pragma unroll
+  for (int i = 0; i < HD; ++i) acc[i] = 0.f;
+  float m_run = -INFINITY, l_run = 0.f, f_pending = 0.f;
+  bool ok = true;
+
+  auto consume_o = [&](uint32_t bi, float f) {   // acc = acc * f + O_blk
+    const uint32_t buf = bi & 1;
+    if (ok && !mbar_wait_err(smem_u32(&ctl->o_full[buf]), (bi >> 1) & 1, err)) { ok = false; atomicCAS((int *)err, 0, DEV_TIMEOUT_TMEM); }
+    tc_fence_after();
+#pragma unroll
+    for (int i = 0; i < HD / 32; ++i) {
+      uint32_t r0[16], r1[16];
+      tmem_ld16(tq + kColO + buf * HD + i * 32, r0);
+      tmem_ld16(tq + kColO + buf * HD + i * 32 + 16, r1);
+      tmem_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        acc[i * 32 + e] = acc[i * 32 + e] * f + __uint_as_float(r0[e]);
+        acc[i * 32 + 16 + e] = acc[i * 32 + 16 + e] * f + __uint_as_float(r1[e]);
+      }
+    }
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&ctl->o_empty[buf]));
+  };
+
+  for (int b = 0; b < t.nblk; ++b, ++blk) {
+    const uint32_t buf = blk & 1;
+    if (ok && !mbar_wait_err(smem_u32(&ctl->s_full[buf]), (blk >> 1) & 1, err)) { ok = false; atomicCAS((int *)err, 0, DEV_TIMEOUT_TMEM); }
+    tc_fence_after();
+    const int p_base = t.pos_beg + b * kAttnBlk;
+    float sc[64];
+    {
+      uint32_t r0[16], r1[16], r2[16], r3[16];
+      tmem_ld16(tq + kColS + buf * 64, r0);
+      tmem_ld16(tq + kColS + buf * 64 + 16, r1);
+      tmem_ld16(tq + kColS + buf * 64 + 32, r2);
+      tmem_ld16(tq + kColS + buf * 64 + 48, r3);
+      tmem_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        sc[e] = __uint_as_float(r0[e]); sc[16 + e] = __uint_as_float(r1[e]);
+        sc[32 + e] = __uint_as_float(r2[e]); sc[48 + e] = __uint_as_float(r3[e]);
+      }
+    }
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&ctl->s_empty[buf]));
+    float mx = -INFINITY;
+#pragma unroll
+    for (int e = 0; e < 64; ++e) {
+      sc[e] = (p_base + e <= lim) ? sc[e] * scale : -INFINITY;
+      mx = fmaxf(mx, sc[e]);
+    }
+    const float m_new = fmaxf(m_run, mx);
+    const float ref = (m_new == -INFINITY) ? 0.f : m_new;
+    const float f = exp2f(m_run - ref);   // exp2(-inf) = 0 on the first block
+    m_run = m_new;
+    float sum = 0.f;
+    // the P buffer is free: the product that read it two blocks ago was seen complete when its O_blk was taken
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+      uint32_t pk[16];
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        const float e0 = exp2f(sc[g * 32 + 2 * e] - ref), e1 = exp2f(sc[g * 32 + 2 * e + 1] - ref);
+        sum += e0 + e1;
+        pk[e] = pack_h2(e0, e1);
+      }
+      tmem_st16(tq + kColP + buf * 32 + g * 16, pk);
+    }
+    l_run = l_run * f + sum;
+    tmem_wait_st();
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&ctl->p_full[buf]));
+    if (b > 0) consume_o(blk - 1, f_pending);
+    f_pending = f;   // (no CTA-wide barrier per block: a failed wait has set the error word, which ends every other wait)
+  }
+  consume_o(blk - 1, f_pending);
+  if (!worker_all(ok)) return false;
+
+  // ---- partial result of this split: un-normalised output, running max (log2 domain), sum -----------------
+  if (valid) {
+    a.attn_ml[ob] = make_float2(m_run, l_run);
+    float4 *dst = reinterpret_cast<float4 *>(a.attn_o + ob * HD);
+#pragma unroll
+    for (int i = 0; i < HD / 4; ++i) dst[i] = make_float4(acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3]);
+  }
+  return true;
+}
+
+template <int HD>
+__global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_constant__ AttnTcArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  constexpr uint32_t kQBytes = kAttnRows * HD * 2, kKvBytes = 2u * kAttnBlk * HD * 2, kHalves = HD / 64;
+  AttnCtl *ctl = reinterpret_cast<AttnCtl *>(smem + kQBytes + kKvStages * kKvBytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int *err = a.err;
+
+  if (threadIdx.x == 0) {
+    for (int b = 0; b < kKvStages; ++b) {
+      mbar_init(smem_u32(&ctl->kv_full[b]), 1);
+      mbar_init(smem_u32(&ctl->kv_empty[b]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&ctl->s_full[b]), 1);
+      mbar_init(smem_u32(&ctl->s_empty[b]), 4);
+      mbar_init(smem_u32(&ctl->p_full[b]), 4);
+      mbar_init(smem_u32(&ctl->o_full[b]), 1);
+      mbar_init(smem_u32(&ctl->o_empty[b]), 4);
+    }
+    mbar_init(smem_u32(&ctl->q_full), 1);
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&ctl->tmem_base), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+  pdl_wait();   // queries and the chunk's K/V rows come from the previous kernel
+  const AttnUnit t = attn_unit_info(a, (int)blockIdx.x);
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- K/V producer
+    if (lane == 0 && t.nblk > 0) {
+      const uint64_t pol = policy_evict_first();
+      const int32_t *btab = a.in.block_tab + (size_t)t.seq * a.in.pages_per_seq;
+      for (int b = 0; b < t.nblk; ++b) {
+        const uint32_t st = b % kKvStages;
+        if (!mbar_wait_err(smem_u32(&ctl->kv_empty[st]), ((b / kKvStages) & 1) ^ 1, err)) { atomicCAS(a.err, 0, DEV_TIMEOUT_EMPTY); break; }
+        const uint32_t bar = smem_u32(&ctl->kv_full[st]);
+        mbar_expect_tx(bar, kKvBytes);
+        uint8_t *sK = smem + kQBytes + st * kKvBytes, *sV = sK + kAttnBlk * HD * 2;
+        for (int pg = 0; pg < kAttnBlk / 16; ++pg) {
+          // a page past the split's end is never visible; load the last visible page again instead
+          const int pos = min(t.pos_beg + b * kAttnBlk + pg * 16, t.pos_end - 1);
+          const int page = btab[pos >> 4];
+#pragma unroll
+          for (int hh = 0; hh < (int)kHalves; ++hh) {
+            const uint32_t off = hh * (kAttnBlk * 128) + pg * 2048;
+            tma_load_5d(smem_u32(sK + off), a.map_kv, hh * 64, 0, t.kh, page, 2 * a.layer, bar, pol);
+            tma_load_5d(smem_u32(sV + off), a.map_kv, hh * 64, 0, t.kh, page, 2 * a.layer + 1, bar, pol);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issue
+    if (lane == 0 && t.nblk > 0) {
+      const uint32_t idesc_qk = umma_idesc_f16(kAttnRows, kAttnBlk, 0);
+      const uint32_t idesc_pv = umma_idesc_f16(kAttnRows, HD, 1);
+      const uint32_t sQ = smem_u32(smem);
+      bool ok = true;
+      auto issue_pv = [&](uint32_t bi) -> bool {   // O_blk = P V for block bi
+        const uint32_t pb = bi & 1, vst = bi % kKvStages;
+        if (!mbar_wait_err(smem_u32(&ctl->p_full[pb]), (bi >> 1) & 1, err)) return false;
+        if (!mbar_wait_err(smem_u32(&ctl->o_empty[pb]), ((bi >> 1) & 1) ^ 1, err)) return false;
+        tc_fence_after();
+        const uint32_t sV = sQ + kQBytes + vst * kKvBytes + kAttnBlk * HD * 2;
+#pragma unroll
+        for (int ks = 0; ks < kAttnBlk / 16; ++ks)   // 16 positions per instruction
+          umma_f16_ts(tmem_base + kColO + pb * HD, tmem_base + kColP + pb * 32 + ks * 8,
+                      umma_desc_sw128_mn(sV + ks * 2048, kAttnBlk * 128), idesc_pv, ks > 0 ? 1u : 0u);
+        umma_commit(smem_u32(&ctl->o_full[pb]));
+        umma_commit(smem_u32(&ctl->kv_empty[vst]));
+        return true;
+      };
+      ok = mbar_wait_err(smem_u32(&ctl->q_full), 0, err);
+      for (uint32_t b = 0; ok && b < (uint32_t)t.nblk; ++b) {
+        const uint32_t kst = b % kKvStages, st = b & 1;
+        if (!mbar_wait_err(smem_u32(&ctl->kv_full[kst]), (b / kKvStages) & 1, err)) { ok = false; break; }
+        if (!mbar_wait_err(smem_u32(&ctl->s_empty[st]), ((b >> 1) & 1) ^ 1, err)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t sK = sQ + kQBytes + kst * kKvBytes;
+#pragma unroll
+        for (int hh = 0; hh < (int)kHalves; ++hh) {
+          const uint64_t dq = umma_desc_sw128(sQ + hh * (kAttnRows * 128)), dk = umma_desc_sw128(sK + hh * (kAttnBlk * 128));
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)
+            umma_bf16(tmem_base + kColS + st * 64, dq + 2 * kk, dk + 2 * kk, idesc_qk, (hh | kk) != 0 ? 1u : 0u);
+        }
+        umma_commit(smem_u32(&ctl->s_full[st]));
+        if (b > 0) ok = issue_pv(b - 1);
+      }
+      if (ok) ok = issue_pv((uint32_t)t.nblk - 1);
+      if (!ok) atomicCAS(a.err, 0, DEV_TIMEOUT_FULL);
+    }
+  } else {
+    // ---------------------------------------------------------------- workers
+    uint32_t blk = 0;
+    attn_unit_workers<HD>(a, ctl, t, smem, tmem_base, warp & 3, lane, (int)threadIdx.x - kWorkerWarp0 * 32, blk, err);
+  }
+  pdl_launch_dependents();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+static size_t attn_tc_smem(int hd) {
+  return 1024 + (size_t)kAttnRows * hd * 2 + (size_t)kKvStages * 2 * kAttnBlk * hd * 2 + sizeof(AttnCtl) + 64;
+}
+
+cudaError_t launch_attention_tc(const AttnTcArgs &a, cudaStream_t st) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_tc_smem(128));
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_tc_smem(64));
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(a.n_tiles * a.Hkv * a.attn_splits);
+  cfg.blockDim = dim3(kTcThreads);
+  cfg.dynamicSmemBytes = attn_tc_smem(a.hd);
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return (a.hd == 128) ? cudaLaunchKernelEx(&cfg, attn_tc_kernel<128>, a) : cudaLaunchKernelEx(&cfg, attn_tc_kernel<64>, a);
+}
+
+}  // namespace ts

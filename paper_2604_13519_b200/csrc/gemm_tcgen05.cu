@@ -89,9 +89,11 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
         tma_load_3d(smem_u32(smem + (size_t)it * stage_bytes + kWBytes), &tmap_a, (kb0 + it) * kBlockK, m0, 0,
                     bar, pol_a);
       }
+      // slot and round parity are carried along: an integer division per k-block would be a large part of
+      // this single thread's time budget per block
+      int s = (pre == g.stages) ? 0 : pre;
+      uint32_t ph = (pre == g.stages) ? 1 : 0;
       for (int it = pre; it < nkb; ++it) {
-        const int s = it % g.stages;
-        const uint32_t ph = (it / g.stages) & 1;
         if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1)) {
           atomicExch(g.err, DEV_TIMEOUT_EMPTY);
           break;
@@ -101,6 +103,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
         uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
         tma_load_2d(dst, &tmap_w, 0, (blockIdx.x * g.n_kblocks + kb0 + it) * kTileN, bar, pol_w);
         tma_load_3d(dst + kWBytes, &tmap_a, (kb0 + it) * kBlockK, m0, 0, bar, pol_a);
+        if (++s == g.stages) { s = 0; ph ^= 1; }
       }
     } else if (lane == 0) {
       pdl_wait();
@@ -110,9 +113,9 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     if (lane == 0) {
       const uint32_t idesc = umma_idesc_bf16(kTileN, ncols);
       bool ok = true;
+      int s = 0;
+      uint32_t ph = 0;
       for (int it = 0; it < nkb; ++it) {
-        const int s = it % g.stages;
-        const uint32_t ph = (it / g.stages) & 1;
         if (!mbar_wait(smem_u32(&ctl->full[s]), ph)) {
           atomicExch(g.err, DEV_TIMEOUT_FULL);
           ok = false;
@@ -127,6 +130,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
           umma_bf16(tmem_base, da + 2 * kk, db + 2 * kk, idesc, (it | kk) != 0);
         }
         umma_commit(smem_u32(&ctl->empty[s]));
+        if (++s == g.stages) { s = 0; ph ^= 1; }
       }
       if (!ok) ctl->abort_flag = 1;
       umma_commit(smem_u32(&ctl->tmem_full));

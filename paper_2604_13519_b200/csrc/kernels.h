@@ -74,6 +74,21 @@ struct AttnArgs {
 cudaError_t launch_attention_split(const AttnArgs &a, cudaStream_t st);
 cudaError_t launch_attention_combine(const AttnArgs &a, cudaStream_t st);
 
+// tcgen05 attention as a kernel of its own (attention_tc.cu): one CTA per (128-row tile, kv head, split)
+struct AttnTcArgs {
+  StepIn in;
+  int Hq, Hkv, hd, layer;
+  int n_tiles, attn_splits;
+  const int32_t *tile_seq;       // [n_tiles] sequence of each 128-row tile of packed rows
+  const int32_t *tile_row0;      // [n_tiles] first packed row of the tile
+  const __half *q;               // [M][Hq][hd] rotated queries
+  const CUtensorMap *map_kv;     // device copy of the 5-d map over the paged KV pool
+  float *attn_o;                 // [M*Hq][splits][hd] unnormalised partial outputs
+  float2 *attn_ml;               // [M*Hq][splits] (running max in the log2 domain, sum)
+  int *err;                      // device status word
+};
+cudaError_t launch_attention_tc(const AttnTcArgs &a, cudaStream_t st);
+
 // per-row argmax over the LM-head tiles, longest accepted prefix per sequence, new lengths
 struct AcceptArgs {
   StepIn in;

@@ -386,6 +386,22 @@ ts_status run_step(ts_model *m) {
     aa.n_splits = std::max(1, std::min(std::min(s, kMaxAttnSplits), nblk));
   }
 
+  ts::AttnTcArgs at{};
+  at.in = in; at.Hq = c.n_q_heads; at.Hkv = c.n_kv_heads; at.hd = c.head_dim;
+  at.n_tiles = m->last_tiles128;
+  at.tile_seq = di + L.o_tile128_seq; at.tile_row0 = di + L.o_tile128_row0;
+  at.q = q; at.map_kv = (const CUtensorMap *)m->WS(L.maps) + (L.n_maps - 1);
+  at.attn_o = aa.part_o; at.attn_ml = aa.part_ml; at.err = m->d_out() + L.o_err;
+  if (m->fused_ok) {
+    // one unit per CTA: about one CTA per SM, every split at least one 64-position block
+    const int32_t *hi = m->h_in();
+    int max_total = 0;
+    for (int i = 0; i < B; ++i)
+      max_total = std::max(max_total, hi[L.o_len + i] + (hi[L.o_cu + i + 1] - hi[L.o_cu + i]));
+    const int s = m->n_sms / std::max(1, c.n_kv_heads * m->last_tiles128);
+    aa.n_splits = std::max(1, std::min(std::min(s, kMaxAttnSplits), (max_total + 63) / 64));
+  }
+  at.attn_splits = aa.n_splits;
   CU_TRY(ts::launch_embed_norm(in, (const __nv_bfloat16 *)m->W(L.embed), (const float *)m->W(L.g1[0]), c.rms_eps,
                                d, x, h, R, m->planes, (unsigned long long *)m->WS(L.amax), m->st));
   m->launched(3);
@@ -402,7 +418,12 @@ ts_status run_step(ts_model *m) {
                               m->k_pages(l), m->v_pages(l), m->st));
     m->launched(4);
     aa.k_pages = m->k_pages(l); aa.v_pages = m->v_pages(l);
-    CU_TRY(ts::launch_attention_split(aa, m->st));
+    if (m->fused_ok) {   // tensor-memory attention (needs the same device features as the persistent kernel)
+      at.layer = l;
+      CU_TRY(ts::launch_attention_tc(at, m->st));
+    } else {
+      CU_TRY(ts::launch_attention_split(aa, m->st));
+    }
     m->launched(1);
     CU_TRY(ts::launch_attention_combine(aa, m->st));
     m->launched(2);
