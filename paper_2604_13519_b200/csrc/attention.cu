@@ -81,6 +81,7 @@ attn_split_kernel(const AttnArgs a) {
   const int b1 = min(min(nblk, b0 + bps), (len + j_max + 1 + kBlk - 1) / kBlk);
   const int32_t *btab = a.in.block_tab + (size_t)seq * a.in.pages_per_seq;
 
+  pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
   pdl_wait();
 
   // this thread's two rows of the warp's 16-row tile
@@ -213,7 +214,6 @@ attn_split_kernel(const AttnArgs a) {
     __syncthreads();
   }
   cp_async_wait<0>();
-  pdl_launch_dependents();
 
   l_l += __shfl_xor_sync(0xffffffffu, l_l, 1);
   l_l += __shfl_xor_sync(0xffffffffu, l_l, 2);
@@ -240,6 +240,7 @@ attn_split_kernel(const AttnArgs a) {
 // output element over the splits with independent loads.
 __global__ void attn_combine_kernel(const AttnArgs a) {
   __shared__ float w_s[64];
+  pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
   pdl_wait();
   const int m = blockIdx.x, h = blockIdx.y, d = threadIdx.x;
   const size_t base = ((size_t)m * a.Hq + h) * a.n_splits;
@@ -263,7 +264,6 @@ __global__ void attn_combine_kernel(const AttnArgs a) {
     for (int s = threadIdx.x; s < a.n_splits; s += 32) w_s[s] *= inv;
   }
   __syncthreads();
-  pdl_launch_dependents();
   // eight splits' loads in flight at a time (an empty split never wrote its slot: it is not read)
   float num = 0.f;
   for (int s0 = 0; s0 < a.n_splits; s0 += 8) {

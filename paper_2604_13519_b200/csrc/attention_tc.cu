@@ -261,6 +261,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
+  pdl_launch_dependents();   // (this CTA holds its tensor memory; the dependent waits for this kernel's end anyway)
   pdl_wait();   // queries and the chunk's K/V rows come from the previous kernel
   const AttnUnit t = attn_unit_info(a, (int)blockIdx.x);
 
@@ -334,7 +335,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
     uint32_t blk = 0;
     attn_unit_workers<HD>(a, ctl, t, smem, tmem_base, warp & 3, lane, (int)threadIdx.x - kWorkerWarp0 * 32, blk, err);
   }
-  pdl_launch_dependents();
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {

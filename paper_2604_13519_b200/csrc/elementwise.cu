@@ -30,6 +30,7 @@ norm_kernel(const int32_t *tokens, const __nv_bfloat16 *embed, const float *part
             const float *gain, float eps, int d, float *x, __nv_bfloat16 *h, int h_rows, int planes,
             unsigned long long *amax) {
   __shared__ float red[32];
+  pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
   pdl_wait();
   const int m = blockIdx.x;
   float *xr = x + (size_t)m * d;
@@ -62,7 +63,6 @@ norm_kernel(const int32_t *tokens, const __nv_bfloat16 *embed, const float *part
   }
   const float tot = block_sum(ss, red);
   const float r = rsqrtf(tot / (float)d + eps);
-  pdl_launch_dependents();
   for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
     const float4 v = *reinterpret_cast<const float4 *>(xr + c);
     const float4 gn = *reinterpret_cast<const float4 *>(gain + c);
@@ -107,6 +107,40 @@ cudaError_t launch_add_norm(int M, int d, const float *part, int n_splits, int p
                     planes, (unsigned long long *)nullptr);
 }
 
+// grid = (F / 512, M), 256 threads: thread t owns features f = 2t, 2t+1 of the CTA's 512 (one float4 of the
+// interleaved gate/up columns per split-K slab).
+__global__ void __launch_bounds__(256)
+swiglu_kernel(int F, const float *part, int n_splits, int part_rows, __nv_bfloat16 *act, int act_rows, int planes) {
+  pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
+  pdl_wait();
+  const int m = blockIdx.y;
+  const int f = blockIdx.x * 512 + threadIdx.x * 2;
+  if (f >= F) return;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s0 = 0; s0 < n_splits; s0 += 4) {
+    float4 p[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      p[u] = (s0 + u < n_splits) ? *reinterpret_cast<const float4 *>(part + ((size_t)(s0 + u) * part_rows + m) * (2 * (size_t)F) + 2 * f)
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) { acc.x += p[u].x; acc.y += p[u].y; acc.z += p[u].z; acc.w += p[u].w; }
+  }
+  const float a0 = acc.x / (1.f + __expf(-acc.x)) * acc.y;
+  const float a1 = acc.z / (1.f + __expf(-acc.z)) * acc.w;
+  __nv_bfloat16 hi[2], lo[2];
+  split_bf16(a0, hi[0], lo[0]);
+  split_bf16(a1, hi[1], lo[1]);
+  *reinterpret_cast<uint32_t *>(act + (size_t)m * F + f) = *reinterpret_cast<uint32_t *>(hi);
+  if (planes == 2) *reinterpret_cast<uint32_t *>(act + ((size_t)act_rows + m) * F + f) = *reinterpret_cast<uint32_t *>(lo);
+}
+
+cudaError_t launch_swiglu(int M, int F, const float *part, int n_splits, int part_rows, __nv_bfloat16 *act, int act_rows,
+                          int planes, cudaStream_t st) {
+  return launch_pdl(swiglu_kernel, dim3((F + 511) / 512, M), dim3(256), 0, st, F, part, n_splits, part_rows, act,
+                    act_rows, planes);
+}
+
 __device__ __forceinline__ __half to_half_sat(float x) {
   return __float2half_rn(fminf(fmaxf(x, -65504.f), 65504.f));
 }
@@ -115,6 +149,7 @@ __device__ __forceinline__ __half to_half_sat(float x) {
 // (i, i + hd/2) of q or k heads, or elements (i, i + hd/2) of a v head.
 __global__ void rope_kv_kernel(StepIn in, const float *part, int n_splits, int part_rows, int Hq, int Hkv, int hd,
                                const float2 *rope_tab, __half *q_out, __half *k_pages, __half *v_pages) {
+  pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
   pdl_wait();
   const int m = blockIdx.x, head = blockIdx.y, i = threadIdx.x, half = hd >> 1;
   const int N = (Hq + 2 * Hkv) * hd;
@@ -126,7 +161,6 @@ __global__ void rope_kv_kernel(StepIn in, const float *part, int n_splits, int p
     a += ab.x;
     b += ab.y;
   }
-  pdl_launch_dependents();
   const int pos = in.pos[m];
   if (head < Hq + Hkv) {
     const float2 cs = rope_tab[(size_t)pos * half + i];
@@ -189,6 +223,7 @@ cudaError_t launch_retile(const __nv_bfloat16 *src, int n_rows, int r0, int K, R
 // is the number of leading agreements.
 __global__ void __launch_bounds__(64)
 accept_kernel(AcceptArgs a) {
+  pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
   pdl_wait();
   const int seq = blockIdx.x;
   const int r0 = a.in.cu_rows[seq], r1 = a.in.cu_rows[seq + 1];

@@ -44,8 +44,9 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
   const int n0 = blockIdx.x * kTileN;
   const int split = blockIdx.y;
   const int m0 = blockIdx.z * g.Mc;
-  const int kb0 = split * g.kb_per_split;
-  const int kb1 = min(g.n_kblocks, kb0 + g.kb_per_split);
+  // balanced cut of the k-blocks into gridDim.y runs
+  const int kb0 = (int)(((long long)split * g.n_kblocks) / (int)gridDim.y);
+  const int kb1 = (int)(((long long)(split + 1) * g.n_kblocks) / (int)gridDim.y);
   const int nkb = kb1 - kb0;
   const uint32_t ncols = g.planes * g.Mc;
   uint32_t alloc_cols = 32;
@@ -70,6 +71,10 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
+  // Let the next kernel launch now: it waits (griddepcontrol.wait) for this one to finish before it touches
+  // dependent data, so only its launch latency and its own prologue (weight prefetch) move forward.  Placed after
+  // this CTA holds its resources, so a waiting dependent can never starve an earlier kernel.
+  pdl_launch_dependents();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
@@ -211,7 +216,6 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
       }
     }
   }
-  pdl_launch_dependents();
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {

@@ -41,6 +41,7 @@ constexpr int kMaxAttnSplits = 32;
 constexpr int kMcOptions[4] = {16, 32, 64, 128};
 constexpr int kMaxFusedCtas = 256;   // the fused kernel runs one CTA per SM
 constexpr int kFusedMaxRows = 64;    // most rows per step the fused kernel takes
+constexpr bool kSplitGateUp = false;      // split-K gate-up + separate SwiGLU kernel: measured no faster than the fused epilogue
 constexpr bool kAutoPrefersFused = false;   // path = 0 picks the faster of the two on the 8B batch-1 step
 
 struct Layout {
@@ -115,7 +116,7 @@ void make_layout(const ts_model_config &c, Layout *L) {
   o = 0;
   L->x = take(R * d * 4);
   L->h = take(planes * R * d * 2);
-  const uint64_t part_cols = std::max<uint64_t>(L->Nqkv, d);
+  const uint64_t part_cols = std::max<uint64_t>(std::max<uint64_t>(L->Nqkv, d), 2 * F);
   L->part = take((uint64_t)kMaxSplits * R * part_cols * 4);
   L->q = take(R * Nq * 2);
   L->attn_o = take(R * c.n_q_heads * kMaxAttnSplits * hd * 4);
@@ -270,13 +271,21 @@ int pick_mc_index(int M) {
   return 3;
 }
 
-// split-K factor: fill about two CTAs per SM, at least 4 k-blocks per slice
+// split-K factor: two CTAs fit on an SM, so the grid runs in waves of 2 * n_sms CTAs; take the smallest factor
+// (at least 4 k-blocks per slice) whose last wave is at least 95% full, else the one that fills its waves best
 int pick_splits(const ts_model *m, int n_tiles, int m_chunks, int n_kblocks, bool allow) {
   if (!allow) return 1;
-  const int ctas = n_tiles * m_chunks;
-  int s = (2 * m->n_sms) / std::max(1, ctas);
-  s = std::max(1, std::min(s, std::min(kMaxSplits, n_kblocks / 4)));
-  return std::max(1, s);
+  const int ctas = std::max(1, n_tiles * m_chunks), slots = 2 * m->n_sms;
+  const int s_max = std::max(1, std::min(kMaxSplits, n_kblocks / 4));
+  int best = 1;
+  double best_eff = 0.0;
+  for (int s = 1; s <= s_max; ++s) {
+    const int waves = (ctas * s + slots - 1) / slots;
+    const double eff = (double)(ctas * s) / ((double)waves * slots);
+    if (eff > best_eff + 1e-9) { best_eff = eff; best = s; }
+    if (eff >= 0.95) return s;
+  }
+  return best;
 }
 
 struct GemmPlan { int splits, kb_per_split; };
@@ -289,8 +298,7 @@ ts_status run_gemm(ts_model *m, int epi, const CUtensorMap &tw, const CUtensorMa
   g.n_kblocks = K / 64;
   const int m_chunks = (M + g.Mc - 1) / g.Mc;
   int splits = pick_splits(m, N / 128, m_chunks, g.n_kblocks, epi == ts::EPI_PARTIAL);
-  g.kb_per_split = (g.n_kblocks + splits - 1) / splits;
-  splits = (g.n_kblocks + g.kb_per_split - 1) / g.kb_per_split;
+  g.kb_per_split = (g.n_kblocks + splits - 1) / splits;   // (the kernel cuts K into `splits` balanced runs)
   g.out = out; g.out_rows = m->L.rows_alloc;
   g.act_out = act_out; g.act_rows = m->L.rows_alloc; g.out_planes = m->planes;
   g.amax = amax;
@@ -432,8 +440,20 @@ ts_status run_step(ts_model *m) {
     CU_TRY(ts::launch_add_norm(M, d, part, plan.splits, R, (const float *)m->W(L.g2[l]), c.rms_eps, x, h, R,
                                m->planes, m->st));
     m->launched(3);
-    s = run_gemm(m, ts::EPI_SWIGLU, m->tm_gu[l], m->tm_h, 2 * F, d, M, nullptr, act, nullptr, nullptr);
-    if (s) return s;
+    {
+      const int mi = pick_mc_index(M), m_chunks = (M + kMcOptions[mi] - 1) / kMcOptions[mi];
+      const int gu_splits = kSplitGateUp ? pick_splits(m, 2 * F / 128, m_chunks, d / 64, true) : 1;
+      if (gu_splits > 1) {   // split-K for full waves; the SwiGLU then runs over the summed partials
+        GemmPlan gp{};
+        s = run_gemm(m, ts::EPI_PARTIAL, m->tm_gu[l], m->tm_h, 2 * F, d, M, part, nullptr, nullptr, &gp);
+        if (s) return s;
+        CU_TRY(ts::launch_swiglu(M, F, part, gp.splits, R, act, R, m->planes, m->st));
+        m->launched(3);
+      } else {
+        s = run_gemm(m, ts::EPI_SWIGLU, m->tm_gu[l], m->tm_h, 2 * F, d, M, nullptr, act, nullptr, nullptr);
+        if (s) return s;
+      }
+    }
     s = run_gemm(m, ts::EPI_PARTIAL, m->tm_d[l], m->tm_act, d, F, M, part, nullptr, nullptr, &plan);
     if (s) return s;
   }
