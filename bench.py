@@ -43,7 +43,7 @@ METRIC = "verified_tokens_per_s"
 UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the projection GEMM, from the ncu
 # capture summarised under profiles/ (None until a capture exists)
-GEMM_TRAFFIC_BYTES_PER_LAUNCH = None
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = 107.1e6    # (36 x 396.2 MB measured per layer + the LM-head launch by its algorithmic bytes) / 145 launches
 # the same for one launch of the persistent kernel on the default workload
 FUSED_TRAFFIC_BYTES_PER_LAUNCH = None
 
