@@ -107,40 +107,6 @@ cudaError_t launch_add_norm(int M, int d, const float *part, int n_splits, int p
                     planes, (unsigned long long *)nullptr);
 }
 
-// grid = (F / 512, M), 256 threads: thread t owns features f = 2t, 2t+1 of the CTA's 512 (one float4 of the
-// interleaved gate/up columns per split-K slab).
-__global__ void __launch_bounds__(256)
-swiglu_kernel(int F, const float *part, int n_splits, int part_rows, __nv_bfloat16 *act, int act_rows, int planes) {
-  pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
-  pdl_wait();
-  const int m = blockIdx.y;
-  const int f = blockIdx.x * 512 + threadIdx.x * 2;
-  if (f >= F) return;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int s0 = 0; s0 < n_splits; s0 += 4) {
-    float4 p[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u)
-      p[u] = (s0 + u < n_splits) ? *reinterpret_cast<const float4 *>(part + ((size_t)(s0 + u) * part_rows + m) * (2 * (size_t)F) + 2 * f)
-                                 : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-    for (int u = 0; u < 4; ++u) { acc.x += p[u].x; acc.y += p[u].y; acc.z += p[u].z; acc.w += p[u].w; }
-  }
-  const float a0 = acc.x / (1.f + __expf(-acc.x)) * acc.y;
-  const float a1 = acc.z / (1.f + __expf(-acc.z)) * acc.w;
-  __nv_bfloat16 hi[2], lo[2];
-  split_bf16(a0, hi[0], lo[0]);
-  split_bf16(a1, hi[1], lo[1]);
-  *reinterpret_cast<uint32_t *>(act + (size_t)m * F + f) = *reinterpret_cast<uint32_t *>(hi);
-  if (planes == 2) *reinterpret_cast<uint32_t *>(act + ((size_t)act_rows + m) * F + f) = *reinterpret_cast<uint32_t *>(lo);
-}
-
-cudaError_t launch_swiglu(int M, int F, const float *part, int n_splits, int part_rows, __nv_bfloat16 *act, int act_rows,
-                          int planes, cudaStream_t st) {
-  return launch_pdl(swiglu_kernel, dim3((F + 511) / 512, M), dim3(256), 0, st, F, part, n_splits, part_rows, act,
-                    act_rows, planes);
-}
-
 __device__ __forceinline__ __half to_half_sat(float x) {
   return __float2half_rn(fminf(fmaxf(x, -65504.f), 65504.f));
 }

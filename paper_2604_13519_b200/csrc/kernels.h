@@ -51,9 +51,6 @@ cudaError_t launch_embed_norm(const StepIn &in, const __nv_bfloat16 *embed, cons
 // x[m] += sum_s part[s][m]; h = rmsnorm(x) * gain -> bf16 (hi[, lo])
 cudaError_t launch_add_norm(int M, int d, const float *part, int n_splits, int part_rows, const float *gain,
                             float eps, float *x, __nv_bfloat16 *h, int h_rows, int planes, cudaStream_t st);
-// act[m][f] = silu(g) * u with g, u = sums over the split-K partials of columns 2f, 2f+1 -> bf16 (hi[, lo])
-cudaError_t launch_swiglu(int M, int F, const float *part, int n_splits, int part_rows, __nv_bfloat16 *act, int act_rows,
-                          int planes, cudaStream_t st);
 // qkv = sum of split-K partials; rotary on q and k; q -> fp16 [M][Hq][hd]; k, v -> fp16 pages
 cudaError_t launch_rope_kv(const StepIn &in, const float *part, int n_splits, int part_rows, int Hq, int Hkv,
                            int hd, const float2 *rope_tab, __half *q_out, __half *k_pages, __half *v_pages,

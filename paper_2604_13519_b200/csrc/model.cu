@@ -41,7 +41,6 @@ constexpr int kMaxAttnSplits = 32;
 constexpr int kMcOptions[4] = {16, 32, 64, 128};
 constexpr int kMaxFusedCtas = 256;   // the fused kernel runs one CTA per SM
 constexpr int kFusedMaxRows = 64;    // most rows per step the fused kernel takes
-constexpr bool kSplitGateUp = false;      // split-K gate-up + separate SwiGLU kernel: measured no faster than the fused epilogue
 constexpr bool kAutoPrefersFused = false;   // path = 0 picks the faster of the two on the 8B batch-1 step
 
 struct Layout {
@@ -116,7 +115,7 @@ void make_layout(const ts_model_config &c, Layout *L) {
   o = 0;
   L->x = take(R * d * 4);
   L->h = take(planes * R * d * 2);
-  const uint64_t part_cols = std::max<uint64_t>(std::max<uint64_t>(L->Nqkv, d), 2 * F);
+  const uint64_t part_cols = std::max<uint64_t>(L->Nqkv, d);
   L->part = take((uint64_t)kMaxSplits * R * part_cols * 4);
   L->q = take(R * Nq * 2);
   L->attn_o = take(R * c.n_q_heads * kMaxAttnSplits * hd * 4);
@@ -440,20 +439,10 @@ ts_status run_step(ts_model *m) {
     CU_TRY(ts::launch_add_norm(M, d, part, plan.splits, R, (const float *)m->W(L.g2[l]), c.rms_eps, x, h, R,
                                m->planes, m->st));
     m->launched(3);
-    {
-      const int mi = pick_mc_index(M), m_chunks = (M + kMcOptions[mi] - 1) / kMcOptions[mi];
-      const int gu_splits = kSplitGateUp ? pick_splits(m, 2 * F / 128, m_chunks, d / 64, true) : 1;
-      if (gu_splits > 1) {   // split-K for full waves; the SwiGLU then runs over the summed partials
-        GemmPlan gp{};
-        s = run_gemm(m, ts::EPI_PARTIAL, m->tm_gu[l], m->tm_h, 2 * F, d, M, part, nullptr, nullptr, &gp);
-        if (s) return s;
-        CU_TRY(ts::launch_swiglu(M, F, part, gp.splits, R, act, R, m->planes, m->st));
-        m->launched(3);
-      } else {
-        s = run_gemm(m, ts::EPI_SWIGLU, m->tm_gu[l], m->tm_h, 2 * F, d, M, nullptr, act, nullptr, nullptr);
-        if (s) return s;
-      }
-    }
+    // (gate-up keeps its SwiGLU epilogue and so cannot split K: 192 tiles run as 1.3 waves.  Splitting K
+    // three ways with a separate SwiGLU kernel filled the waves but cost as much as it saved.)
+    s = run_gemm(m, ts::EPI_SWIGLU, m->tm_gu[l], m->tm_h, 2 * F, d, M, nullptr, act, nullptr, nullptr);
+    if (s) return s;
     s = run_gemm(m, ts::EPI_PARTIAL, m->tm_d[l], m->tm_act, d, F, M, part, nullptr, nullptr, &plan);
     if (s) return s;
   }
