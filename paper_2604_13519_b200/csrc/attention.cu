@@ -235,47 +235,32 @@ attn_split_kernel(const AttnArgs a) {
   }
 }
 
-// grid = (M, Hq), hd threads: merge the splits of one (row, query head).  The first warp turns the
-// splits' (max, sum) pairs into normalised weights in shared memory; every thread then sums its
-// output element over the splits with independent loads.
+// grid = (M, Hq), hd threads: merge the splits of one (row, query head).  Every thread issues the loads of its
+// output element for all splits at once, together with the splits' (max, sum) pairs (lane s of each warp takes
+// split s and turns it into a normalised weight), so the kernel costs one round trip to L2.  NS = compile-time bound
+// on the number of splits.
+template <int NS>
 __global__ void attn_combine_kernel(const AttnArgs a) {
-  __shared__ float w_s[64];
   pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
   pdl_wait();
-  const int m = blockIdx.x, h = blockIdx.y, d = threadIdx.x;
+  const int m = blockIdx.x, h = blockIdx.y, d = threadIdx.x, lane = threadIdx.x & 31;
   const size_t base = ((size_t)m * a.Hq + h) * a.n_splits;
-  if (threadIdx.x < 32) {
-    float mx = -INFINITY;
-    for (int s = threadIdx.x; s < a.n_splits; s += 32) {
-      const float2 ml = a.part_ml[base + s];
-      if (ml.y > 0.f) mx = fmaxf(mx, ml.x);
-    }
+  const float2 ml = lane < a.n_splits ? a.part_ml[base + lane] : make_float2(-INFINITY, 0.f);
+  // (an empty split never wrote its slot; whatever is read there is dropped by its zero weight below)
+  float t[NS];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    float den = 0.f;
-    for (int s = threadIdx.x; s < a.n_splits; s += 32) {
-      const float2 ml = a.part_ml[base + s];
-      const float w = ml.y > 0.f ? exp2f(ml.x - mx) : 0.f;
-      w_s[s] = w;
-      den += w * ml.y;
-    }
-    den = warp_sum(den);
-    const float inv = 1.f / den;
-    for (int s = threadIdx.x; s < a.n_splits; s += 32) w_s[s] *= inv;
-  }
-  __syncthreads();
-  // eight splits' loads in flight at a time (an empty split never wrote its slot: it is not read)
+  for (int s = 0; s < NS; ++s) t[s] = (s < a.n_splits) ? a.part_o[(base + s) * a.hd + d] : 0.f;
+  float mx = ml.y > 0.f ? ml.x : -INFINITY;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  float w = ml.y > 0.f ? exp2f(ml.x - mx) : 0.f;
+  const float den = warp_sum(w * ml.y);
+  w *= 1.f / den;
   float num = 0.f;
-  for (int s0 = 0; s0 < a.n_splits; s0 += 8) {
-    float w[8], t[8];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      w[u] = (s0 + u < a.n_splits) ? w_s[s0 + u] : 0.f;
-      t[u] = 0.f;
-      if (w[u] != 0.f) t[u] = a.part_o[(base + s0 + u) * a.hd + d];
-    }
-#pragma unroll
-    for (int u = 0; u < 8; ++u) num += w[u] * t[u];
+  for (int s = 0; s < NS; ++s) {
+    const float ws = __shfl_sync(0xffffffffu, w, s);
+    if (ws != 0.f) num += ws * t[s];
   }
   __nv_bfloat16 hi, lo;
   split_bf16(num, hi, lo);
@@ -318,7 +303,13 @@ cudaError_t launch_attention_split(const AttnArgs &a, cudaStream_t st) {
 }
 
 cudaError_t launch_attention_combine(const AttnArgs &a, cudaStream_t st) {
-  return launch_attn_pdl(attn_combine_kernel, dim3(a.in.M, a.Hq), dim3(a.hd), 0, st, a);
+  if (a.n_splits < 1 || a.n_splits > kAttnMaxSplits) return cudaErrorInvalidValue;
+  const dim3 grid(a.in.M, a.Hq), block(a.hd);
+  if (a.n_splits <= 2) return launch_attn_pdl(attn_combine_kernel<2>, grid, block, 0, st, a);
+  if (a.n_splits <= 4) return launch_attn_pdl(attn_combine_kernel<4>, grid, block, 0, st, a);
+  if (a.n_splits <= 8) return launch_attn_pdl(attn_combine_kernel<8>, grid, block, 0, st, a);
+  if (a.n_splits <= 16) return launch_attn_pdl(attn_combine_kernel<16>, grid, block, 0, st, a);
+  return launch_attn_pdl(attn_combine_kernel<32>, grid, block, 0, st, a);
 }
 
 }  // namespace ts

@@ -24,7 +24,7 @@ constexpr int kMaxTiles = 512;
 constexpr size_t kTileBytes = 2 * kMaxTiles * sizeof(int32_t);
 constexpr size_t kScratchBytes = kPartOBytes + kPartMlBytes + kTileBytes;
 constexpr int kMaxDevices = 64;
-constexpr int kMaxAttnSplits = 32;
+constexpr int kMaxAttnSplits = ts::kAttnMaxSplits;
 
 static __device__ __align__(256) unsigned char g_attn_scratch[kScratchBytes];
 

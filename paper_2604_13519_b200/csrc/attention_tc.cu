@@ -78,7 +78,7 @@ __device__ __forceinline__ AttnUnit attn_unit_info(const AttnTcArgs &a, int u) {
   const int total = t.len + k_i;
   const int j_max = (t.row0 + t.rows_here - 1) / t.G;
   int p0, p1;
-  split_pages((total + 15) >> 4, a.attn_splits, t.split, &p0, &p1);
+  split_blocks((total + 15) >> 4, a.attn_splits, t.split, &p0, &p1);
   t.pos_beg = p0 << 4;
   t.pos_end = min(min(p1 << 4, total), t.len + j_max + 1);   // nothing beyond the last row's own position is visible
   t.nblk = t.pos_end > t.pos_beg ? (t.pos_end - t.pos_beg + kAttnBlk - 1) / kAttnBlk : 0;
@@ -96,6 +96,12 @@ __device__ __forceinline__ void cp_async16z(uint32_t dst, const void *src, bool 
 }
 __device__ __forceinline__ void cp_commit_wait_all() {
   asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+// 2^x for x <= 0 (and 0 for -inf); tiny results flush to zero
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 __device__ __forceinline__ uint32_t pack_h2(float x, float y) {
   __half2 v = __floats2half2_rn(x, y);
@@ -135,6 +141,7 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
 
   const uint32_t tq = tmem_base + ((uint32_t)(q * 32) << 16);
   const int lim = min(t.len + j, t.pos_end - 1);   // last visible position of this row
+  const int lim_all = min(t.len + t.row0 / t.G, t.pos_end - 1);   // ... of the tile's first row: every row sees up to here
   const float scale = rsqrtf((float)HD) * 1.4426950408889634f;
   float acc[HD];
 #pragma unroll
@@ -185,29 +192,36 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
     tc_fence_before();
     __syncwarp();
     if (lane == 0) mbar_arrive(smem_u32(&ctl->s_empty[buf]));
-    float mx = -INFINITY;
+    // a block every row sees whole needs no mask (all but the last blocks of a sequence's last split)
+    if (p_base + kAttnBlk - 1 > lim_all) {
 #pragma unroll
-    for (int e = 0; e < 64; ++e) {
-      sc[e] = (p_base + e <= lim) ? sc[e] * scale : -INFINITY;
-      mx = fmaxf(mx, sc[e]);
+      for (int e = 0; e < 64; ++e) sc[e] = (p_base + e <= lim) ? sc[e] : -INFINITY;
     }
-    const float m_new = fmaxf(m_run, mx);
+    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+    for (int e = 0; e < 64; e += 4) {
+      mx0 = fmaxf(mx0, sc[e]); mx1 = fmaxf(mx1, sc[e + 1]); mx2 = fmaxf(mx2, sc[e + 2]); mx3 = fmaxf(mx3, sc[e + 3]);
+    }
+    // running maximum in the log2 domain: scores times log2(e)/sqrt(head_dim), folded into one multiply-add per score
+    const float m_new = fmaxf(m_run, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale);
     const float ref = (m_new == -INFINITY) ? 0.f : m_new;
-    const float f = exp2f(m_run - ref);   // exp2(-inf) = 0 on the first block
+    const float f = ex2_approx(m_run - ref);   // exp2(-inf) = 0 on the first block
     m_run = m_new;
-    float sum = 0.f;
+    float sum0 = 0.f, sum1 = 0.f;
     // the P buffer is free: the product that read it two blocks ago was seen complete when its O_blk was taken
 #pragma unroll
     for (int g = 0; g < 2; ++g) {
       uint32_t pk[16];
 #pragma unroll
       for (int e = 0; e < 16; ++e) {
-        const float e0 = exp2f(sc[g * 32 + 2 * e] - ref), e1 = exp2f(sc[g * 32 + 2 * e + 1] - ref);
-        sum += e0 + e1;
+        const float e0 = ex2_approx(fmaf(sc[g * 32 + 2 * e], scale, -ref));
+        const float e1 = ex2_approx(fmaf(sc[g * 32 + 2 * e + 1], scale, -ref));
+        sum0 += e0; sum1 += e1;
         pk[e] = pack_h2(e0, e1);
       }
       tmem_st16(tq + kColP + buf * 32 + g * 16, pk);
     }
+    const float sum = sum0 + sum1;
     l_run = l_run * f + sum;
     tmem_wait_st();
     tc_fence_before();
@@ -262,7 +276,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
   pdl_launch_dependents();   // (this CTA holds its tensor memory; the dependent waits for this kernel's end anyway)
-  pdl_wait();   // queries and the chunk's K/V rows come from the previous kernel
+  // The step's integer inputs were copied in before the step's first kernel started, so they may be read here.
   const AttnUnit t = attn_unit_info(a, (int)blockIdx.x);
 
   if (warp == 0) {
@@ -270,9 +284,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
     if (lane == 0 && t.nblk > 0) {
       const uint64_t pol = policy_evict_first();
       const int32_t *btab = a.in.block_tab + (size_t)t.seq * a.in.pages_per_seq;
-      for (int b = 0; b < t.nblk; ++b) {
+      auto load_block = [&](int b) {
         const uint32_t st = b % kKvStages;
-        if (!mbar_wait_err(smem_u32(&ctl->kv_empty[st]), ((b / kKvStages) & 1) ^ 1, err)) { atomicCAS(a.err, 0, DEV_TIMEOUT_EMPTY); break; }
         const uint32_t bar = smem_u32(&ctl->kv_full[st]);
         mbar_expect_tx(bar, kKvBytes);
         uint8_t *sK = smem + kQBytes + st * kKvBytes, *sV = sK + kAttnBlk * HD * 2;
@@ -287,6 +300,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
             tma_load_5d(smem_u32(sV + off), a.map_kv, hh * 64, 0, t.kh, page, 2 * a.layer + 1, bar, pol);
           }
         }
+      };
+      // blocks wholly inside the cache of earlier steps do not depend on the previous kernel: fill the ring with them
+      int b = 0;
+      for (; b < min(t.nblk, kKvStages) && t.pos_beg + (b + 1) * kAttnBlk <= t.len; ++b) load_block(b);
+      pdl_wait();   // the chunk's own K/V rows come from the previous kernel
+      for (; b < t.nblk; ++b) {
+        if (!mbar_wait_err(smem_u32(&ctl->kv_empty[b % kKvStages]), ((b / kKvStages) & 1) ^ 1, err)) { atomicCAS(a.err, 0, DEV_TIMEOUT_EMPTY); break; }
+        load_block(b);
       }
     }
   } else if (warp == 1) {
@@ -333,6 +354,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
   } else {
     // ---------------------------------------------------------------- workers
     uint32_t blk = 0;
+    pdl_wait();   // the rotated queries come from the previous kernel
     attn_unit_workers<HD>(a, ctl, t, smem, tmem_base, warp & 3, lane, (int)threadIdx.x - kWorkerWarp0 * 32, blk, err);
   }
   tc_fence_before();

@@ -56,6 +56,8 @@ cudaError_t launch_rope_kv(const StepIn &in, const float *part, int n_splits, in
                            int hd, const float2 *rope_tab, __half *q_out, __half *k_pages, __half *v_pages,
                            cudaStream_t st);
 
+constexpr int kAttnMaxSplits = 32;   // KV splits per (row tile, kv head): one lane of the merge kernel each
+
 struct AttnArgs {
   StepIn in;
   const __half *q;               // [M][Hq][hd] rotated queries, fp16

@@ -37,7 +37,7 @@ ts_status fail(ts_status code, const char *fmt, ...) {
 inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
 constexpr int kMaxSplits = 12;
-constexpr int kMaxAttnSplits = 32;
+constexpr int kMaxAttnSplits = ts::kAttnMaxSplits;
 constexpr int kMcOptions[4] = {16, 32, 64, 128};
 constexpr int kMaxFusedCtas = 256;   // the fused kernel runs one CTA per SM
 constexpr int kFusedMaxRows = 64;    // most rows per step the fused kernel takes
@@ -287,6 +287,40 @@ int pick_splits(const ts_model *m, int n_tiles, int m_chunks, int n_kblocks, boo
   return best;
 }
 
+// KV splits per (row tile, kv head) of the tensor-memory attention kernel.  A unit (one CTA) costs a fixed part plus
+// a part per 64-position block; a step's units are spread over the SMs by the hardware scheduler, so the kernel
+// takes about max(longest unit, all units / SMs, waves x shortest unit), and the merge kernel grows with the
+// number of splits.  Take the smallest split count within 3% of the best estimate.
+int pick_attn_splits(const ts_model *m) {
+  const ts_model_config &c = m->c;
+  const Layout &L = m->L;
+  const int32_t *hi = m->h_in();
+  const int G = c.n_q_heads / c.n_kv_heads;
+  const double c_unit = 5.0, c_blk = 0.9, c_merge = 0.3;   // microseconds, measured on the 8B shape
+  double est[kMaxAttnSplits + 1], best = 1e30;
+  for (int s = 1; s <= kMaxAttnSplits; ++s) {
+    double longest = 0.0, total = 0.0, shortest = 1e30;
+    long units = 0;
+    for (int i = 0; i < m->last_B; ++i) {
+      const int k = hi[L.o_cu + i + 1] - hi[L.o_cu + i];
+      const int blocks = (hi[L.o_len + i] + k + 63) / 64;
+      const int tiles = (k * G + 127) / 128;
+      const int live = std::min(s, blocks);                       // splits that hold at least one block
+      const double unit = c_unit + c_blk * ((blocks + live - 1) / live);
+      longest = std::max(longest, unit);
+      shortest = std::min(shortest, unit);
+      total += (double)tiles * c.n_kv_heads * (live * unit + (s - live) * c_unit);
+      units += (long)tiles * c.n_kv_heads * s;
+    }
+    const double waves = (double)((units + m->n_sms - 1) / m->n_sms);
+    est[s] = std::max(std::max(longest, total / m->n_sms), waves * shortest) + c_merge * s;
+    best = std::min(best, est[s]);
+  }
+  for (int s = 1; s <= kMaxAttnSplits; ++s)
+    if (est[s] <= 1.03 * best) return s;
+  return 1;
+}
+
 struct GemmPlan { int splits, kb_per_split; };
 
 ts_status run_gemm(ts_model *m, int epi, const CUtensorMap &tw, const CUtensorMap *ta4, int N, int K, int M,
@@ -399,15 +433,7 @@ ts_status run_step(ts_model *m) {
   at.tile_seq = di + L.o_tile128_seq; at.tile_row0 = di + L.o_tile128_row0;
   at.q = q; at.map_kv = (const CUtensorMap *)m->WS(L.maps) + (L.n_maps - 1);
   at.attn_o = aa.part_o; at.attn_ml = aa.part_ml; at.err = m->d_out() + L.o_err;
-  if (m->fused_ok) {
-    // one unit per CTA: about one CTA per SM, every split at least one 64-position block
-    const int32_t *hi = m->h_in();
-    int max_total = 0;
-    for (int i = 0; i < B; ++i)
-      max_total = std::max(max_total, hi[L.o_len + i] + (hi[L.o_cu + i + 1] - hi[L.o_cu + i]));
-    const int s = m->n_sms / std::max(1, c.n_kv_heads * m->last_tiles128);
-    aa.n_splits = std::max(1, std::min(std::min(s, kMaxAttnSplits), (max_total + 63) / 64));
-  }
+  if (m->fused_ok) aa.n_splits = pick_attn_splits(m);
   at.attn_splits = aa.n_splits;
   CU_TRY(ts::launch_embed_norm(in, (const __nv_bfloat16 *)m->W(L.embed), (const float *)m->W(L.g1[0]), c.rms_eps,
                                d, x, h, R, m->planes, (unsigned long long *)m->WS(L.amax), m->st));
@@ -506,14 +532,26 @@ ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::ve
       hi[L.o_tile_row0 + tiles] = r0;
       ++tiles;
     }
-    for (int r0 = 0; r0 < k * G; r0 += 128) {
-      hi[L.o_tile128_seq + tiles128] = i;
-      hi[L.o_tile128_row0 + tiles128] = r0;
-      ++tiles128;
-    }
+    tiles128 += (k * G + 127) / 128;
     std::memcpy(hi + L.o_btab + (size_t)i * L.pages_per_seq, s->pages.data(), s->pages.size() * sizeof(int32_t));
     M += k;
     hi[L.o_cu + i + 1] = M;
+  }
+  {
+    // 128-row tiles, longest sequence first: the attention kernel's CTAs are handed out in tile order, so the long
+    // units start first and the short ones fill the tail
+    std::vector<int> order(B);
+    for (int i = 0; i < B; ++i) order[i] = i;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+      return hi[L.o_len + a] + (hi[L.o_cu + a + 1] - hi[L.o_cu + a]) > hi[L.o_len + b] + (hi[L.o_cu + b + 1] - hi[L.o_cu + b]);
+    });
+    int t = 0;
+    for (int i : order)
+      for (int r0 = 0; r0 < (hi[L.o_cu + i + 1] - hi[L.o_cu + i]) * G; r0 += 128) {
+        hi[L.o_tile128_seq + t] = i;
+        hi[L.o_tile128_row0 + t] = r0;
+        ++t;
+      }
   }
   const bool can_fuse = m->fused_ok && M <= kFusedMaxRows;
   if (c.path == 2 && !can_fuse)
