@@ -51,16 +51,19 @@ def _gaussian_bf16(seed: int, tid: int, rows: int, cols: int, pool) -> torch.Ten
     return t.view(rows, cols)
 
 
-def make_weights(shape: ModelShape, seed: int = MASTER_SEED, layers=None):
+def make_weights(shape: ModelShape, seed: int = MASTER_SEED, layers=None, with_globals: bool = True):
     """dict name -> torch.bfloat16 CPU tensor [out][in]; norm gains (fp32, all ones) under
-    'l{l}.g1', 'l{l}.g2', 'gf'.  `layers` restricts generation to some layer indices (global
-    tensors are always produced)."""
+    'l{l}.g1', 'l{l}.g2', 'gf'.  `layers` restricts generation to some layer indices; the global
+    tensors (embedding, LM head) are produced unless `with_globals` is false.  A tensor's values
+    depend only on (seed, its index in tensor_names), so a model can be generated piece by piece."""
     w = {}
     with ThreadPoolExecutor(max_workers=os.cpu_count() or 4) as pool:
         for tid, (name, (r, c)) in enumerate(tensor_names(shape)):
-            if layers is not None and name.startswith("l") and name[1].isdigit():
-                if int(name[1:name.index(".")]) not in layers:
-                    continue
+            per_layer = name.startswith("l") and name[1].isdigit()
+            if per_layer and layers is not None and int(name[1:name.index(".")]) not in layers:
+                continue
+            if not per_layer and not with_globals:
+                continue
             w[name] = _gaussian_bf16(seed, tid, r, c, pool)
     for l in range(shape.n_layers):
         if layers is not None and l not in layers:

@@ -1,0 +1,101 @@
+"""Full-size parity: the 8B-shaped decoder at full depth (36 layers) against the float64 oracle on every
+logit of the chunk, in three configurations:
+
+  * batch 1, 8192-token context, k = 32 -- the workload and the launch configuration the benchmark
+    times -- once per step implementation (one kernel per stage, persistent kernel);
+  * a ragged batch of three sessions (8192 / 2500 / 5000 cached tokens, k = 32 / 17 / 64) on the
+    default implementation: several row tiles, several sequences, uneven KV splits.
+
+The model is too large to hold twice on the host, so all sides are fed layer by layer from the same
+seeded generators: a layer's weights and the sessions' synthetic context K/V are generated once,
+loaded into the GPU models, pushed through the oracle's own layer routine (one sequence at a time),
+and dropped.  The oracle then applies its head to the final residual rows; each GPU model runs one
+ordinary `ts_verify`.  Nothing the oracle consumes comes from the GPU.
+
+These are the only tests that run all 36 layers, so they also check that the error of the bf16
+(hi, lo) activations and the fp16 attention path stays inside the logit tolerance at depth.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+import paper_2604_13519_b200 as ts
+from paper_2604_13519_b200 import binding as B
+from gpu_util import check_step
+
+pytestmark = pytest.mark.gpu
+
+LAYER_KINDS = dict(wq=B.TS_W_Q, wk=B.TS_W_K, wv=B.TS_W_V, wo=B.TS_W_O, wg=B.TS_W_GATE, wu=B.TS_W_UP,
+                   wd=B.TS_W_DOWN, g1=B.TS_W_GAIN1, g2=B.TS_W_GAIN2)
+SEQS = [(8192, 32), (2500, 17), (5000, 64)]       # (cached tokens, chunk rows) per sequence; stream = index
+
+
+def _model(shape, seqs, path):
+    """The benchmark's model configuration for these sequences."""
+    lens, ks = [n for n, _ in seqs], [k for _, k in seqs]
+    k_max = max(max(ks), 8)
+    pages = sum((n + 2 * k_max + 15) // 16 for n in lens) + 8
+    return ts.Model(shape, max_pages=pages, max_batch=len(seqs), k_max=k_max, max_rows=max(sum(ks), k_max),
+                    max_ctx=max(lens) + 2 * k_max, act_split=True, path=path)
+
+
+def test_8b_full_depth():
+    shape = synth.SHAPES["8b"]
+    assert shape.n_layers == 36
+    # (model, indices into SEQS): the first two are the benchmark's default workload
+    cases = [(_model(shape, SEQS[:1], 1), [0]), (_model(shape, SEQS[:1], 2), [0]), (_model(shape, SEQS, 0), [0, 1, 2])]
+    sessions = [[ts.Session(gm, None, None) for _ in idx] for gm, idx in cases]
+
+    glob = synth.make_weights(shape, layers=[])              # embedding, LM head, final gain
+    for gm, _ in cases:
+        gm.load_tensor(B.TS_W_EMBED, 0, glob["embed"])
+        gm.load_tensor(B.TS_W_LM_HEAD, 0, glob["lm_head"])
+        gm.load_tensor(B.TS_W_FINAL_GAIN, 0, glob["gf"].float())
+
+    pending = synth.Vocab(shape.vocab).tool_call
+    g = np.random.Generator(np.random.Philox(key=[260413519, 0x8B36]))
+    drafts = [[int(t) for t in g.integers(64, shape.vocab, size=k - 1)] for _, k in SEQS]
+    x = [glob["embed"][torch.tensor([pending] + d)].to(torch.float64) for d in drafts]
+
+    for l in range(shape.n_layers):
+        wl = synth.make_weights(shape, layers=[l], with_globals=False)
+        for gm, _ in cases:
+            for n, kind in LAYER_KINDS.items():
+                t = wl[f"l{l}.{n}"]
+                gm.load_tensor(kind, l, t.float() if n[0] == "g" else t)
+        om = oracle.OracleModel(shape, wl)
+        for i, (n_ctx, k) in enumerate(SEQS):
+            Kl, Vl = synth.make_synthetic_kv(shape, n_ctx, stream=i, layers=[l])
+            for (gm, idx), ss in zip(cases, sessions):
+                if i in idx:
+                    ss[idx.index(i)].import_kv(l, Kl[0], Vl[0])
+            x[i], _, _ = om._layer(l, x[i], torch.arange(k) + n_ctx, Kl[0].to(torch.float64), Vl[0].to(torch.float64),
+                                   torch.arange(n_ctx))
+        del wl, om, Kl, Vl
+
+    head = oracle.OracleModel(shape, glob)
+    refs = []
+    for i, d in enumerate(drafts):
+        logits = head._head(x[i])
+        t = oracle.argmax_lowest(logits)
+        n_acc = 0
+        while n_acc < len(d) and t[n_acc] == d[n_acc]:
+            n_acc += 1
+        refs.append(dict(logits=logits, argmax=t, accept_len=n_acc, emitted=d[:n_acc] + [t[n_acc]]))
+
+    for (gm, idx), ss in zip(cases, sessions):
+        for s, i in zip(ss, idx):
+            s.set_cache(SEQS[i][0], pending)
+        res = ts.ts_verify(gm, ss, [drafts[i] for i in idx])
+        row0 = 0
+        for r, i in zip(res, idx):
+            k = SEQS[i][1]
+            got = gm.read_logits(row0, k)
+            assert np.isfinite(got).all()
+            where = f"8b x 36 layers, path {gm.cfg.path}, batch {len(idx)}, sequence {i} (ctx {SEQS[i][0]}, k {k})"
+            mx, mean = check_step(r, got, refs[i], where=where)
+            print(f"{where}: logits max-abs {mx:.3e}, mean-abs {mean:.3e}")
+            row0 += k
+        gm.close()
