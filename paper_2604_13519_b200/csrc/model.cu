@@ -289,15 +289,18 @@ int pick_splits(const ts_model *m, int n_tiles, int m_chunks, int n_kblocks, boo
 
 // KV splits per (row tile, kv head) of the tensor-memory attention kernel.  A unit (one CTA) costs a fixed part plus
 // a part per 64-position block; a step's units are spread over the SMs by the hardware scheduler, so the kernel
-// takes about max(longest unit, all units / SMs, waves x shortest unit), and the merge kernel grows with the
-// number of splits.  Take the smallest split count within 3% of the best estimate.
+// takes about max(longest unit, all units / slots, waves x shortest unit), and the merge kernel adds a little per
+// split.  One eighth of the SMs is left out of the slots: the kernels that follow launch early and park their
+// prologues (weight prefetch) there, and measured on the 8B step 128 units beat 136 and 144 on 148 SMs.
 int pick_attn_splits(const ts_model *m) {
   const ts_model_config &c = m->c;
   const Layout &L = m->L;
   const int32_t *hi = m->h_in();
   const int G = c.n_q_heads / c.n_kv_heads;
-  const double c_unit = 5.0, c_blk = 0.9, c_merge = 0.3;   // microseconds, measured on the 8B shape
+  const double c_unit = 5.0, c_blk = 0.9, c_merge = 0.03;   // microseconds, measured on the 8B shape
+  const int slots = std::max(1, m->n_sms - m->n_sms / 8);
   double est[kMaxAttnSplits + 1], best = 1e30;
+  long n_units[kMaxAttnSplits + 1];
   for (int s = 1; s <= kMaxAttnSplits; ++s) {
     double longest = 0.0, total = 0.0, shortest = 1e30;
     long units = 0;
@@ -312,13 +315,19 @@ int pick_attn_splits(const ts_model *m) {
       total += (double)tiles * c.n_kv_heads * (live * unit + (s - live) * c_unit);
       units += (long)tiles * c.n_kv_heads * s;
     }
-    const double waves = (double)((units + m->n_sms - 1) / m->n_sms);
-    est[s] = std::max(std::max(longest, total / m->n_sms), waves * shortest) + c_merge * s;
+    const double waves = (double)((units + slots - 1) / slots);
+    est[s] = std::max(std::max(longest, total / slots), waves * shortest) + c_merge * s;
+    n_units[s] = units;
     best = std::min(best, est[s]);
   }
-  for (int s = 1; s <= kMaxAttnSplits; ++s)
-    if (est[s] <= 1.03 * best) return s;
-  return 1;
+  // among the counts within 3% of the best estimate: the largest that still runs as one wave (more CTAs stream
+  // more bytes at once), else the smallest
+  int pick = 0;
+  for (int s = kMaxAttnSplits; s >= 1 && !pick; --s)
+    if (est[s] <= 1.03 * best && n_units[s] <= slots) pick = s;
+  for (int s = 1; s <= kMaxAttnSplits && !pick; ++s)
+    if (est[s] <= 1.03 * best) pick = s;
+  return std::max(1, pick);
 }
 
 struct GemmPlan { int splits, kb_per_split; };
