@@ -57,15 +57,17 @@ def rope(x: torch.Tensor, pos: torch.Tensor, theta: float) -> torch.Tensor:
 
 
 def attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, q_pos: torch.Tensor,
-              k_pos: torch.Tensor) -> torch.Tensor:
-    """Grouped-query causal attention.  q: [Tq, Hq, hd]; k, v: [Tk, Hkv, hd]; a query at position
-    p attends to every key at position <= p.  Query head h uses kv head h // (Hq / Hkv).
+              k_pos: torch.Tensor, allowed: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Grouped-query attention.  q: [Tq, Hq, hd]; k, v: [Tk, Hkv, hd].  By default causal: a query
+    at position p attends to every key at position <= p.  `allowed` ([Tq, Tk] bool) replaces that
+    rule (the tree-structured mask of Appendix A.1).  Query head h uses kv head h // (Hq / Hkv).
     Returns [Tq, Hq, hd]."""
     Tq, Hq, hd = q.shape
     Hkv = k.shape[1]
     G = Hq // Hkv
     scale = 1.0 / math.sqrt(hd)
-    allowed = k_pos[None, :] <= q_pos[:, None]              # [Tq, Tk]
+    if allowed is None:
+        allowed = k_pos[None, :] <= q_pos[:, None]          # [Tq, Tk]
     out = torch.empty_like(q)
     for h in range(Hq):
         kh = h // G
@@ -130,7 +132,7 @@ class OracleModel:
 
     # -- the row arithmetic shared by both drivers ------------------------------------------
     def _layer(self, l: int, x: torch.Tensor, pos: torch.Tensor, k_prev, v_prev, pos_prev,
-               probe: Optional[dict] = None):
+               probe: Optional[dict] = None, allowed: Optional[torch.Tensor] = None):
         s, w = self.s, self.w
         T = x.shape[0]
         h = rmsnorm(x, w[f"l{l}.g1"], s.rms_eps)
@@ -142,7 +144,7 @@ class OracleModel:
         k_all = torch.cat([k_prev, k], dim=0)
         v_all = torch.cat([v_prev, v], dim=0)
         pos_all = torch.cat([pos_prev, pos])
-        o = attention(q, k_all, v_all, pos, pos_all).reshape(T, s.n_q_heads * s.head_dim)
+        o = attention(q, k_all, v_all, pos, pos_all, allowed).reshape(T, s.n_q_heads * s.head_dim)
         x = x + _wt(o, w[f"l{l}.wo"])
         h2 = rmsnorm(x, w[f"l{l}.g2"], s.rms_eps)
         a = swiglu(_wt(h2, w[f"l{l}.wg"]), _wt(h2, w[f"l{l}.wu"]))
