@@ -183,6 +183,26 @@ ts_status ts_verify(ts_model *m, ts_session *const *sessions, int32_t B,
                     const int32_t *draft_tokens, const int32_t *draft_offsets, uint32_t flags,
                     ts_verify_result *out);
 
+/* ts_verify_tree — PackDraftsAsTree's output verified in one forward pass under the tree-structured attention
+ * mask (Appendix A.1 "Parallel Verification"; Algorithm 1: Verification, SelectLongestAcceptedPrefix).
+ * Sequence i's chunk has node 0 = its pending token and node j+1 = draft_tokens[draft_offsets[i] + j], whose
+ * parent is node draft_parents[draft_offsets[i] + j], a value in [0, j] (a parent precedes its children; a
+ * chain is parents 0, 1, 2, ...).  At most 64 nodes per sequence.  A node attends to the cache and to its
+ * ancestors and itself; its rotary position is cache length + depth; its K/V rows go to cache slot
+ * cache length + node index.  Acceptance walks from the root: at node u with model token t_u it moves to the
+ * lowest-numbered child of u whose token is t_u, and stops when there is none.  out[i]: accept_len = nodes on
+ * the path after the root, emitted = their tokens followed by the model's token at the last node, argmax = t_u
+ * for every node.  path_out (host, B x TS_K_MAX, may be NULL): node indices of the path, root first, -1 after
+ * the end.  Before returning, the K/V rows of the path are moved to consecutive slots (cache length + 0, 1, ..),
+ * so ts_commit advances the session exactly as after ts_verify.  The rows of rejected nodes are lost.
+ * Runs on the one-kernel-per-stage path only (TS_ERR_UNIMPLEMENTED with path = 2 or without tensor-memory
+ * attention); flags must not contain TS_FLAG_SKIP_LM_HEAD.  Other errors as ts_verify, plus TS_ERR_ARG for a
+ * parent outside [0, j]. */
+ts_status ts_verify_tree(ts_model *m, ts_session *const *sessions, int32_t B,
+                         const int32_t *draft_tokens, const int32_t *draft_parents,
+                         const int32_t *draft_offsets, uint32_t flags, ts_verify_result *out,
+                         int32_t *path_out);
+
 /* Enqueue again the device work of the last ts_verify call on its inputs, which are still resident
  * in device memory; no host<->device copy, no synchronisation.  The step is idempotent because
  * sessions advance only in ts_commit.  For timing the kernels alone. */

@@ -95,6 +95,8 @@ _SIGNATURES = {
     "ts_prefill": [_P, _P, _I32P, C.c_int32],
     "ts_draft": [_P, C.c_int32, _I32P, _I32P, _I32P],
     "ts_verify": [_P, C.POINTER(_P), C.c_int32, _I32P, _I32P, C.c_uint32, C.POINTER(ts_verify_result)],
+    "ts_verify_tree": [_P, C.POINTER(_P), C.c_int32, _I32P, _I32P, _I32P, C.c_uint32, C.POINTER(ts_verify_result),
+                       _I32P],
     "ts_verify_replay": [_P],
     "ts_profile_step": [_P, C.POINTER(C.c_float), _I32P, C.c_int32],
     "ts_commit": [_P, C.POINTER(ts_verify_result)],
@@ -369,6 +371,25 @@ def ts_verify(model: Model, sessions: Sequence[Session], drafts: Sequence[Sequen
     out = (ts_verify_result * B)()
     _check(lib().ts_verify(model.h, hs, B, _i32(flat), _i32(offs), flags, out))
     return list(out)
+
+
+def ts_verify_tree(model: Model, sessions: Sequence[Session], drafts: Sequence[Sequence[int]],
+                   parents: Sequence[Sequence[int]], flags: int = 0):
+    """Draft trees: drafts[i][j] is node j+1 of sequence i, parents[i][j] its parent node (0 = the pending
+    token).  Returns (list of ts_verify_result, list of accepted paths as node indices, root first)."""
+    B = len(sessions)
+    hs = (_P * B)(*[s.h for s in sessions])
+    flat, par, offs = [], [], [0]
+    for d, p in zip(drafts, parents):
+        assert len(d) == len(p)
+        flat += list(d)
+        par += list(p)
+        offs.append(len(flat))
+    out = (ts_verify_result * B)()
+    path = (C.c_int32 * (B * TS_K_MAX))()
+    _check(lib().ts_verify_tree(model.h, hs, B, _i32(flat), _i32(par), _i32(offs), flags, out, path))
+    paths = [[path[i * TS_K_MAX + j] for j in range(out[i].accept_len + 1)] for i in range(B)]
+    return list(out), paths
 
 
 def ts_verify_replay(model: Model):

@@ -140,8 +140,10 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
   if (wtid == 0) mbar_arrive(smem_u32(&ctl->q_full));
 
   const uint32_t tq = tmem_base + ((uint32_t)(q * 32) << 16);
-  const int lim = min(t.len + j, t.pos_end - 1);   // last visible position of this row
-  const int lim_all = min(t.len + t.row0 / t.G, t.pos_end - 1);   // ... of the tile's first row: every row sees up to here
+  // Visibility: the whole cache, and of the chunk the rows named by this row's mask (itself and its ancestors in
+  // the draft tree; in a chain, rows 0..j), up to the end of this split.
+  const int lim_all = min(t.len, t.pos_end) - 1;   // every row sees every position up to here
+  const unsigned long long anc = ((unsigned long long)a.in.anc[2 * (t.r_beg + j) + 1] << 32) | a.in.anc[2 * (t.r_beg + j)];
   const float scale = rsqrtf((float)HD) * 1.4426950408889634f;
   float acc[HD];
 #pragma unroll
@@ -195,7 +197,11 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
     // a block every row sees whole needs no mask (all but the last blocks of a sequence's last split)
     if (p_base + kAttnBlk - 1 > lim_all) {
 #pragma unroll
-      for (int e = 0; e < 64; ++e) sc[e] = (p_base + e <= lim) ? sc[e] : -INFINITY;
+      for (int e = 0; e < 64; ++e) {
+        const int p = p_base + e, rel = p - t.len;   // rel < 64: the chunk has at most 64 rows and p < pos_end below
+        const bool vis = p < t.pos_end && (rel < 0 || ((anc >> (rel & 63)) & 1ull) != 0ull);
+        sc[e] = vis ? sc[e] : -INFINITY;
+      }
     }
     float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll

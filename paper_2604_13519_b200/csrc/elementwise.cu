@@ -139,11 +139,14 @@ __global__ void rope_kv_kernel(StepIn in, const float *part, int n_splits, int p
     q[i] = to_half_sat(a);
     q[i + half] = to_half_sat(b);
   } else {
+    // cache slot = cached length + the row's index in its chunk (equal to its position in a chain; in a draft
+    // tree the position is the depth, and siblings still need slots of their own)
     const int seq = in.row_seq[m];
-    const int page = in.block_tab[(size_t)seq * in.pages_per_seq + (pos >> 4)];
+    const int slot = in.seq_len[seq] + (m - in.cu_rows[seq]);
+    const int page = in.block_tab[(size_t)seq * in.pages_per_seq + (slot >> 4)];
     const bool is_k = head < Hq + Hkv;
     const int kh = is_k ? head - Hq : head - Hq - Hkv;
-    __half *dst = (is_k ? k_pages : v_pages) + (((size_t)page * Hkv + kh) * 16 + (pos & 15)) * hd;
+    __half *dst = (is_k ? k_pages : v_pages) + (((size_t)page * Hkv + kh) * 16 + (slot & 15)) * hd;
     dst[i] = to_half_sat(a);
     dst[i + half] = to_half_sat(b);
   }
@@ -185,8 +188,9 @@ cudaError_t launch_retile(const __nv_bfloat16 *src, int n_rows, int r0, int K, R
 
 // One CTA per sequence.  Each row's argmax was reduced by the LM-head epilogue into a packed
 // (ordered value bits, ~token id) word, so the largest word is the largest logit with the lowest id.
-// Thread 0 then walks the draft: row j predicted the token that row j+1 was fed; the accepted length
-// is the number of leading agreements.
+// Thread 0 then walks the draft from the root: at row u the model predicted t_u; the walk moves to the
+// lowest-numbered child of u that was fed t_u and stops when there is none.  In a chain (parent of row j
+// = j - 1) this is the number of leading agreements between the drafts and the predictions.
 __global__ void __launch_bounds__(64)
 accept_kernel(AcceptArgs a) {
   pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
@@ -198,15 +202,49 @@ accept_kernel(AcceptArgs a) {
   __syncthreads();
   if (threadIdx.x == 0) {
     const int k = r1 - r0;
-    int l = 0;
-    while (l < k - 1 && a.argmax[r0 + l] == a.in.tokens[r0 + l + 1]) ++l;
-    a.accept_len[seq] = l;
     int32_t *em = a.emitted + (size_t)seq * a.k_max;
-    for (int j = 0; j < l; ++j) em[j] = a.in.tokens[r0 + j + 1];
-    em[l] = a.argmax[r0 + l];
+    int32_t *path = a.path + (size_t)seq * a.k_max;
+    int l = 0, u = 0;
+    path[0] = 0;
+    for (;;) {
+      const int32_t t = a.argmax[r0 + u];
+      int c = u + 1;
+      while (c < k && !(a.in.parent[r0 + c] == u && a.in.tokens[r0 + c] == t)) ++c;
+      if (c >= k) break;
+      em[l] = t;
+      u = c;
+      path[++l] = u;
+    }
+    a.accept_len[seq] = l;
+    em[l] = a.argmax[r0 + u];
     a.new_len[seq] = a.in.seq_len[seq] + l + 1;   // rejected rows stay in their pages, uncounted
-    a.new_pending[seq] = a.argmax[r0 + l];
+    a.new_pending[seq] = a.argmax[r0 + u];
   }
+}
+
+// grid = (B, layers, kv heads), hd threads.  Path entry j (chunk row path[j]) moves from cache slot len + path[j]
+// to slot len + j.  path is increasing with path[j] >= j, so going through j in ascending order never overwrites
+// a row that is still to be moved; thread i moves element i of every row, so no barrier is needed.
+__global__ void kv_compact_kernel(CompactArgs a) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int seq = blockIdx.x, layer = blockIdx.y, kh = blockIdx.z, i = threadIdx.x;
+  const int l = a.accept_len[seq], len = a.in.seq_len[seq];
+  const int32_t *path = a.path + (size_t)seq * a.k_max;
+  const int32_t *btab = a.in.block_tab + (size_t)seq * a.in.pages_per_seq;
+  __half *kp = a.kv_pool + (uint64_t)layer * a.layer_stride;
+  for (int j = 1; j <= l; ++j) {
+    const int src = len + path[j], dst = len + j;
+    if (src == dst) continue;
+    const size_t so = (((size_t)btab[src >> 4] * a.Hkv + kh) * 16 + (src & 15)) * a.hd + i;
+    const size_t dof = (((size_t)btab[dst >> 4] * a.Hkv + kh) * 16 + (dst & 15)) * a.hd + i;
+    kp[dof] = kp[so];
+    kp[a.v_offset + dof] = kp[a.v_offset + so];
+  }
+}
+
+cudaError_t launch_kv_compact(const CompactArgs &a, cudaStream_t st) {
+  return launch_pdl(kv_compact_kernel, dim3(a.in.B, a.n_layers, a.Hkv), dim3(a.hd), 0, st, a);
 }
 
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t st) {

@@ -40,6 +40,9 @@ struct StepIn {
   const int32_t *cu_rows;    // [B+1]
   const int32_t *seq_len;    // [B] tokens already in the cache
   const int32_t *block_tab;  // [B][pages_per_seq] page ids
+  const int32_t *parent;     // [M] parent of each row inside its chunk (row index relative to the chunk; -1 = root)
+  const uint32_t *anc;       // [M][2] low / high word of the row's visibility mask over its chunk: bit i = row i of
+                             // the chunk is the row itself or one of its ancestors (a chain: bits 0..j)
   int pages_per_seq;
   int B, M;
 };
@@ -100,9 +103,22 @@ struct AcceptArgs {
   int32_t *emitted;        // [B][k_max]
   int32_t *new_len;        // [B]  cache length after the commit
   int32_t *new_pending;    // [B]
+  int32_t *path;           // [B][k_max] chunk rows of the accepted path, root first (accept_len + 1 entries)
   int k_max;
 };
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t st);
+
+// After a tree step: move the K/V rows of the accepted path to consecutive cache positions len, len+1, ...
+struct CompactArgs {
+  StepIn in;
+  const int32_t *accept_len;   // [B]
+  const int32_t *path;         // [B][k_max]
+  int k_max;
+  __half *kv_pool;             // layer l: K pages at kv_pool + l * layer_stride, V pages v_offset further
+  uint64_t layer_stride, v_offset;
+  int n_layers, Hkv, hd;
+};
+cudaError_t launch_kv_compact(const CompactArgs &a, cudaStream_t st);
 
 // Where a source row of an uploaded matrix goes in the stored matrix: row r -> base + r * mul, or, with
 // hd != 0, base + (r / hd) * hd + p(r % hd) with p(e) = 2e for e < hd/2 and 2(e - hd/2) + 1 otherwise.

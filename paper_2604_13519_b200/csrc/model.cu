@@ -57,6 +57,7 @@ struct Layout {
   int n_maps, n_counters, n_phases, max_tiles128, o_tile128_seq, o_tile128_row0;
   // step io (int32 offsets inside d_in / h_in)
   int o_tokens, o_pos, o_rowseq, o_cu, o_len, o_tile_seq, o_tile_row0, o_btab, in_ints;
+  int o_parent, o_anc, o_path;
   // step out (int32 offsets)
   int o_argmax, o_accept, o_emitted, o_newlen, o_newpend, o_err, out_ints;
   int rows_alloc, pages_per_seq, max_tiles, Nqkv, n_vocab_tiles;
@@ -132,11 +133,13 @@ void make_layout(const ts_model_config &c, Layout *L) {
   L->o_tile_seq = itake(L->max_tiles); L->o_tile_row0 = itake(L->max_tiles);
   L->max_tiles128 = c.max_batch * ((c.k_max * G + 127) / 128);
   L->o_tile128_seq = itake(L->max_tiles128); L->o_tile128_row0 = itake(L->max_tiles128);
-  L->o_btab = itake(c.max_batch * L->pages_per_seq);
+  L->o_parent = itake(c.max_rows); L->o_anc = itake(2 * c.max_rows);
+  L->o_btab = itake(c.max_batch * L->pages_per_seq);   // (last: only the used part is copied per step)
   L->in_ints = io;
   io = 0;
   L->o_argmax = itake(c.max_rows); L->o_accept = itake(c.max_batch); L->o_emitted = itake(c.max_batch * c.k_max);
   L->o_newlen = itake(c.max_batch); L->o_newpend = itake(c.max_batch); L->o_err = itake(4);
+  L->o_path = itake(c.max_batch * c.k_max);
   L->out_ints = io;
   L->d_in = take((uint64_t)L->in_ints * 4);
   L->d_out = take((uint64_t)L->out_ints * 4);
@@ -190,6 +193,7 @@ struct ts_model {
   int64_t launches = 0, h2d = 0, d2h = 0;
   bool use_pdl = true;
   bool fused_ok = false, last_fused = false;   // device can run the fused kernel; the staged step uses it
+  bool last_tree = false;                      // the staged step verifies a draft tree (not a chain)
   size_t smem_optin = 0;
   // per-kernel timing pass (ts_profile_step): one event after every launch
   bool profiling = false;
@@ -362,6 +366,7 @@ ts_status run_step_fused(ts_model *m) {
   a.V = c.vocab; a.Hq = c.n_q_heads; a.Hkv = c.n_kv_heads; a.hd = c.head_dim; a.eps = c.rms_eps;
   a.in.tokens = di + L.o_tokens; a.in.pos = di + L.o_pos; a.in.row_seq = di + L.o_rowseq; a.in.cu_rows = di + L.o_cu;
   a.in.seq_len = di + L.o_len; a.in.block_tab = di + L.o_btab; a.in.pages_per_seq = L.pages_per_seq;
+  a.in.parent = di + L.o_parent; a.in.anc = (const uint32_t *)(di + L.o_anc);
   a.in.B = m->last_B; a.in.M = m->last_M;
   a.mc_index = pick_mc_index(m->last_M); a.Mc = kMcOptions[a.mc_index]; a.planes = m->planes;
   a.n_ctas = m->n_sms; a.skip_lm = (m->last_flags & TS_FLAG_SKIP_LM_HEAD) ? 1 : 0;
@@ -409,6 +414,7 @@ ts_status run_step(ts_model *m) {
   int32_t *di = m->d_in();
   in.tokens = di + L.o_tokens; in.pos = di + L.o_pos; in.row_seq = di + L.o_rowseq; in.cu_rows = di + L.o_cu;
   in.seq_len = di + L.o_len; in.block_tab = di + L.o_btab; in.pages_per_seq = L.pages_per_seq;
+  in.parent = di + L.o_parent; in.anc = (const uint32_t *)(di + L.o_anc);
   in.B = B; in.M = M;
   float *x = (float *)m->WS(L.x);
   __nv_bfloat16 *h = (__nv_bfloat16 *)m->WS(L.h);
@@ -494,8 +500,17 @@ ts_status run_step(ts_model *m) {
   ac.in = in; ac.amax = amax;
   ac.argmax = dout + L.o_argmax; ac.accept_len = dout + L.o_accept; ac.emitted = dout + L.o_emitted;
   ac.new_len = dout + L.o_newlen; ac.new_pending = dout + L.o_newpend; ac.k_max = c.k_max;
+  ac.path = dout + L.o_path;
   CU_TRY(ts::launch_accept(ac, m->st));
   m->launched(5);
+  if (m->last_tree) {   // the accepted path's K/V rows become the next cache positions
+    ts::CompactArgs ca{};
+    ca.in = in; ca.accept_len = ac.accept_len; ca.path = ac.path; ca.k_max = c.k_max;
+    ca.kv_pool = (__half *)m->b.kv_pool; ca.layer_stride = L.kv_layer_stride; ca.v_offset = L.kv_v_offset;
+    ca.n_layers = c.n_layers; ca.Hkv = c.n_kv_heads; ca.hd = c.head_dim;
+    CU_TRY(ts::launch_kv_compact(ca, m->st));
+    m->launched(5);
+  }
   return TS_OK;
 }
 
@@ -512,8 +527,9 @@ ts_status ensure_pages(ts_session *s, int tokens) {
 }
 
 // Stage one step: rows[i] = chunk ids of sequence i.  Copies inputs, runs, copies results back, syncs.
+// parents (optional): parents[i][j] = chunk row that row j of sequence i hangs from (-1 for row 0); a chain if null.
 ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::vector<std::vector<int32_t>> &rows,
-                        uint32_t flags) {
+                        uint32_t flags, const std::vector<std::vector<int32_t>> *parents = nullptr) {
   const ts_model_config &c = m->c;
   const Layout &L = m->L;
   int32_t *hi = m->h_in();
@@ -530,10 +546,24 @@ ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::ve
       if (t < 0 || t >= c.vocab) return fail(TS_ERR_TOKEN_RANGE, "token id %d outside [0, %d)", t, c.vocab);
     ts_status st = ensure_pages(s, s->cache_len + k);
     if (st) return st;
+    if (parents && k > 64) return fail(TS_ERR_K_TOO_LARGE, "sequence %d: a draft tree holds at most 64 rows", i);
+    uint64_t anc[64];
+    int depth[64];
     for (int j = 0; j < k; ++j) {
+      const int par = parents ? (*parents)[i][j] : j - 1;
+      if (parents) {
+        if ((j == 0) != (par == -1) || par >= j || par < -1)
+          return fail(TS_ERR_ARG, "sequence %d: parent of row %d must be an earlier row (-1 only for row 0)", i, j);
+        depth[j] = j == 0 ? 0 : depth[par] + 1;
+        anc[j] = (j == 0 ? 0ull : anc[par]) | (1ull << j);
+      }
+      const uint64_t mask = parents ? anc[j] : (j >= 63 ? ~0ull : ((2ull << j) - 1ull));
       hi[L.o_tokens + M + j] = rows[i][j];
-      hi[L.o_pos + M + j] = s->cache_len + j;
+      hi[L.o_pos + M + j] = s->cache_len + (parents ? depth[j] : j);
       hi[L.o_rowseq + M + j] = i;
+      hi[L.o_parent + M + j] = par;
+      hi[L.o_anc + 2 * (M + j)] = (int32_t)(uint32_t)(mask & 0xFFFFFFFFull);
+      hi[L.o_anc + 2 * (M + j) + 1] = (int32_t)(uint32_t)(mask >> 32);
     }
     hi[L.o_len + i] = s->cache_len;
     for (int r0 = 0; r0 < k * G; r0 += 64) {
@@ -566,7 +596,10 @@ ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::ve
   if (c.path == 2 && !can_fuse)
     return fail(TS_ERR_K_TOO_LARGE, "the fused kernel takes at most %d rows on a device that supports it (step has %d)",
                 kFusedMaxRows, M);
-  m->last_fused = can_fuse && (c.path == 2 || (c.path == 0 && kAutoPrefersFused));
+  m->last_tree = parents != nullptr;
+  if (m->last_tree && (c.path == 2 || !m->fused_ok))
+    return fail(TS_ERR_UNIMPLEMENTED, "draft trees need the one-kernel-per-stage path with tensor-memory attention");
+  m->last_fused = !m->last_tree && can_fuse && (c.path == 2 || (c.path == 0 && kAutoPrefersFused));
   m->last_B = B; m->last_M = M; m->last_tiles = tiles; m->last_tiles128 = tiles128; m->last_flags = flags;
   m->have_step = true;
   const size_t in_bytes = (size_t)(L.o_btab + (size_t)B * L.pages_per_seq) * 4;
@@ -962,11 +995,14 @@ ts_status ts_draft(ts_session *s, int32_t max_draft, int32_t *out_tokens, int32_
   return TS_OK;
 }
 
-ts_status ts_verify(ts_model *m, ts_session *const *ss, int32_t B, const int32_t *draft_tokens,
-                    const int32_t *draft_offsets, uint32_t flags, ts_verify_result *out) {
+namespace {
+// ts_verify and ts_verify_tree: draft_parents = nullptr for chains
+ts_status verify_impl(ts_model *m, ts_session *const *ss, int32_t B, const int32_t *draft_tokens,
+                      const int32_t *draft_parents, const int32_t *draft_offsets, uint32_t flags,
+                      ts_verify_result *out, int32_t *path_out) {
   if (!m || !ss || !draft_offsets || !out) return fail(TS_ERR_ARG, "null argument");
   if (B < 1 || B > m->c.max_batch) return fail(TS_ERR_ARG, "batch %d outside [1, %d]", B, m->c.max_batch);
-  std::vector<std::vector<int32_t>> rows(B);
+  std::vector<std::vector<int32_t>> rows(B), parents(B);
   for (int i = 0; i < B; ++i) {
     ts_session *s = ss[i];
     if (!s || s->m != m) return fail(TS_ERR_ARG, "session %d is null or belongs to another model", i);
@@ -980,8 +1016,12 @@ ts_status ts_verify(ts_model *m, ts_session *const *ss, int32_t B, const int32_t
     rows[i].reserve(n + 1);
     rows[i].push_back(s->pending);
     for (int j = 0; j < n; ++j) rows[i].push_back(draft_tokens[draft_offsets[i] + j]);
+    if (draft_parents) {
+      parents[i].push_back(-1);
+      for (int j = 0; j < n; ++j) parents[i].push_back(draft_parents[draft_offsets[i] + j]);
+    }
   }
-  ts_status st = stage_and_run(m, ss, B, rows, flags);
+  ts_status st = stage_and_run(m, ss, B, rows, flags, draft_parents ? &parents : nullptr);
   if (st) return st;
   const Layout &L = m->L;
   const int32_t *ho = m->h_out();
@@ -997,10 +1037,37 @@ ts_status ts_verify(ts_model *m, ts_session *const *ss, int32_t B, const int32_t
       r.n_emitted = r.accept_len + 1;
       for (int j = 0; j < r.n_emitted; ++j) r.emitted[j] = ho[L.o_emitted + i * m->c.k_max + j];
       for (int j = 0; j < r.k; ++j) r.argmax[j] = ho[L.o_argmax + row + j];
+      if (path_out) {
+        for (int j = 0; j < TS_K_MAX; ++j)
+          path_out[i * TS_K_MAX + j] = j <= r.accept_len ? ho[L.o_path + i * m->c.k_max + j] : -1;
+      }
+      if (draft_parents) {
+        // the cache now holds the accepted path's rows at consecutive positions: record what sits there, so that
+        // a later forced commit is checked against the right ids
+        std::vector<int32_t> kept;
+        for (int j = 0; j <= r.accept_len; ++j) kept.push_back(rows[i][ho[L.o_path + i * m->c.k_max + j]]);
+        ss[i]->last_chunk = kept;
+      }
     }
     row += r.k;
   }
   return TS_OK;
+}
+}  // namespace
+
+ts_status ts_verify(ts_model *m, ts_session *const *ss, int32_t B, const int32_t *draft_tokens,
+                    const int32_t *draft_offsets, uint32_t flags, ts_verify_result *out) {
+  return verify_impl(m, ss, B, draft_tokens, nullptr, draft_offsets, flags, out, nullptr);
+}
+
+ts_status ts_verify_tree(ts_model *m, ts_session *const *ss, int32_t B, const int32_t *draft_tokens,
+                         const int32_t *draft_parents, const int32_t *draft_offsets, uint32_t flags,
+                         ts_verify_result *out, int32_t *path_out) {
+  if (!draft_parents && draft_offsets && B >= 1 && draft_offsets[B] > draft_offsets[0])
+    return fail(TS_ERR_ARG, "null draft_parents");
+  if (flags & TS_FLAG_SKIP_LM_HEAD) return fail(TS_ERR_ARG, "a draft tree cannot be run without acceptance");
+  static const int32_t none = 0;
+  return verify_impl(m, ss, B, draft_tokens, draft_parents ? draft_parents : &none, draft_offsets, flags, out, path_out);
 }
 
 ts_status ts_verify_replay(ts_model *m) {
