@@ -5,8 +5,8 @@ leg.  The product package never imports it and shares no code with it.
 """
 from .transformer import (OracleModel, KVCache, rmsnorm, rope, attention, swiglu,   # noqa: F401
                           argmax_lowest, top2_gap)
-from .drafter import (SchemaFsm, Datastore, Drafter, suffix_match, validate_prefix,   # noqa: F401
+from .drafter import (SchemaFsm, Datastore, Drafter, suffix_match, suffix_matches, validate_prefix,   # noqa: F401
                       Q_O, Q_T, Q_P, Q_V, Q_DONE, SUFFIX_LENGTHS, DEFAULT_N_CAP)
-from .loop import prefill, vanilla_greedy, speculative_decode                        # noqa: F401
+from .loop import prefill, vanilla_greedy, speculative_decode, speculative_decode_tree  # noqa: F401
 from .tree import (verify_tree, forward_tree, accepted_path, ancestor_mask, node_depths,  # noqa: F401
                    pack_candidates)

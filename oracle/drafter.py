@@ -30,6 +30,8 @@ Q_O, Q_T, Q_P, Q_V, Q_DONE = "q_o", "q_t", "q_p", "q_v", "done"
 
 SUFFIX_LENGTHS = (7, 6, 5)      # Appendix B.2: longest first, from 7 to 5
 DEFAULT_N_CAP = 32              # Appendix B.2: first continuation length
+LATER_CAPS = (16, 8, 8)         # Appendix B.2: lengths of the second to fourth continuation
+MAX_TOOL_CANDIDATES = 8         # tool names verified in parallel in q_t (a reading: the paper says "all")
 
 
 class SchemaFsm:
@@ -222,6 +224,66 @@ def suffix_match(y: Sequence[int], store: Datastore, ranks: Optional[Sequence[in
     return [], (0, -1, -1)
 
 
+def suffix_matches(y: Sequence[int], store: Datastore, ranks: Optional[Sequence[int]],
+                   caps: Sequence[int], max_draft: int) -> List[List[int]]:
+    """The candidate set of retrieval drafting (Eq. 4 with Appendix B.2's continuation lengths): hits
+    are taken in the order (L descending, candidate rank ascending, match position ascending); a
+    position already taken at a longer L is not taken again; the i-th hit contributes
+    y'[m : m + min(caps[i], max_draft)].  At most len(caps) continuations; the first one is
+    suffix_match's draft."""
+    order = list(range(len(store.entries))) if ranks is None else list(ranks)
+    out: List[List[int]] = []
+    taken = set()
+    if max_draft <= 0:
+        return out
+    for L in SUFFIX_LENGTHS:
+        if len(y) < L:
+            continue
+        s = list(y[-L:])
+        for c in order:
+            e = store.entries[c]
+            if len(e) <= L:
+                continue
+            a = np.asarray(e)
+            ok = np.ones(a.shape[0] - L, dtype=bool)
+            for i in range(L):
+                ok &= a[i:i + a.shape[0] - L] == s[i]
+            for start in np.flatnonzero(ok):
+                m = int(start) + L
+                if (c, m) in taken:
+                    continue
+                taken.add((c, m))
+                out.append(e[m:m + min(caps[len(out)], max_draft)])
+                if len(out) == len(caps):
+                    return out
+    return out
+
+
+def pack_candidates(candidates: Sequence[Sequence[int]], max_nodes: int):
+    """PackDraftsAsTree (Algorithm 1): merge candidate chains (each a continuation of the pending
+    token) into a token trie.  Nodes are numbered in creation order, candidates inserted in the
+    given order, so a parent always precedes its children; a candidate stops adding nodes once the
+    chunk holds max_nodes nodes (root included).  Returns (tokens of nodes 1.., parents of all
+    nodes, parents[0] = -1)."""
+    tokens: List[int] = []
+    parents: List[int] = [-1]
+    children = [dict()]
+    for cand in candidates:
+        u = 0
+        for t in cand:
+            nxt = children[u].get(t)
+            if nxt is None:
+                if len(parents) >= max_nodes:
+                    break
+                nxt = len(parents)
+                parents.append(u)
+                tokens.append(int(t))
+                children.append(dict())
+                children[u][t] = nxt
+            u = nxt
+    return tokens, parents
+
+
 def _first_match_np(e: Sequence[int], s: Sequence[int]) -> int:
     """Same scan as the loop in suffix_match, vectorised (used only for very large stores)."""
     a = np.asarray(e)
@@ -274,6 +336,33 @@ class Drafter:
             return d, 2
         d = self.fsm.draft(self.guess_tool)[:max_draft]
         return (d, 1) if d else ([], 0)
+
+    def draft_candidates(self, max_draft: int) -> Tuple[List[List[int]], int]:
+        """The candidate set B of Algorithm 1: up to four retrieved continuations (lengths n_cap, 16,
+        8, 8), else the schema drafts -- in q_t with the name still open one chain per compatible
+        tool (Eq. 2: the guessed tool first, then ascending tool id, at most MAX_TOOL_CANDIDATES),
+        otherwise the single deterministic chain.  The first candidate is always draft()'s chain."""
+        if max_draft <= 0:
+            return [], 0
+        cands = suffix_matches(self.y, self.store, self.ranks, (self.n_cap,) + LATER_CAPS, max_draft)
+        if cands:
+            return cands, 2
+        f = self.fsm
+        if f.kind == Q_T and f.stage != "mid":
+            prefix = [] if f.stage == "pfx" else f.name_prefix
+            g = self.guess_tool(prefix)
+            if g >= 0:
+                order = [g] + [t for t in f.compatible_tools(prefix) if t != g]
+                cands = [f.draft(lambda _p, t=t: t)[:max_draft] for t in order[:MAX_TOOL_CANDIDATES]]
+                return cands, 1
+        d = f.draft(self.guess_tool)[:max_draft]
+        return ([d], 1) if d else ([], 0)
+
+    def draft_tree(self, max_nodes: int) -> Tuple[List[int], List[int], int]:
+        """(tokens of nodes 1.., parents of all nodes, source): the candidates packed as a trie."""
+        cands, src = self.draft_candidates(max_nodes - 1)
+        toks, par = pack_candidates(cands, max_nodes)
+        return toks, par, (src if toks else 0)
 
     def commit(self, emitted: Sequence[int], eos: int, max_new_tokens: int) -> Tuple[int, bool]:
         """Append emitted ids to y one at a time, applying delta to each; stop at the first id

@@ -60,3 +60,30 @@ def speculative_decode(model: OracleModel, schema, store: Datastore, prompt: Seq
         pending = res["emitted"][consumed - 1]
         steps += 1
     return d.y
+
+
+def speculative_decode_tree(model: OracleModel, schema, store: Datastore, prompt: Sequence[int],
+                            eos: int, max_new_tokens: int, max_nodes: int, n_cap: int = 32,
+                            ranks: Optional[Sequence[int]] = None, cache=None, pending=None,
+                            max_steps: Optional[int] = None, trace: Optional[list] = None) -> List[int]:
+    """Algorithm 1 with its candidate set: draft candidates -> PackDraftsAsTree -> one verification
+    forward under the tree mask -> longest accepted path + bonus token -> append -> FSM update."""
+    from .tree import verify_tree
+    if cache is None:
+        cache, pending = prefill(model, prompt)
+    d = Drafter(schema, store, n_cap=n_cap, ranks=ranks)
+    d.feed_prompt(prompt)
+    steps = 0
+    while not d.finished(eos, max_new_tokens) and (max_steps is None or steps < max_steps):
+        toks, par, source = d.draft_tree(max_nodes)
+        n0 = cache.length
+        res = verify_tree(model, pending, toks, par, cache)
+        consumed, _fin = d.commit(res["emitted"], eos, max_new_tokens)
+        cache.truncate(n0 + consumed)
+        if trace is not None:
+            trace.append(dict(pending=pending, tokens=list(toks), parents=list(par), source=source,
+                              accept_len=res["accept_len"], emitted=list(res["emitted"]),
+                              consumed=consumed, path=list(res["path"])))
+        pending = res["emitted"][consumed - 1]
+        steps += 1
+    return d.y

@@ -20,6 +20,7 @@ from typing import List, Sequence
 import torch
 
 from .transformer import OracleModel, KVCache, argmax_lowest, F64
+from .drafter import pack_candidates  # noqa: F401  (PackDraftsAsTree lives with the drafters)
 
 
 def check_parents(parents: Sequence[int]):
@@ -45,30 +46,6 @@ def ancestor_mask(parents: Sequence[int]) -> torch.Tensor:
             m[j, u] = True
             u = parents[u]
     return m
-
-
-def pack_candidates(candidates: Sequence[Sequence[int]], max_nodes: int):
-    """PackDraftsAsTree: merge candidate chains (each a continuation of the pending token) into a
-    token trie.  Nodes are numbered in creation order, candidates inserted in the given order, so a
-    parent always precedes its children; insertion stops adding nodes once the chunk holds
-    max_nodes nodes (root included).  Returns (tokens of nodes 1.., parents of all nodes)."""
-    tokens: List[int] = []
-    parents: List[int] = [-1]
-    children = [dict()]
-    for cand in candidates:
-        u = 0
-        for t in cand:
-            nxt = children[u].get(t)
-            if nxt is None:
-                if len(parents) >= max_nodes:
-                    break
-                nxt = len(parents)
-                parents.append(u)
-                tokens.append(int(t))
-                children.append(dict())
-                children[u][t] = nxt
-            u = nxt
-    return tokens, parents
 
 
 def forward_tree(model: OracleModel, z: Sequence[int], parents: Sequence[int], cache: KVCache):

@@ -217,3 +217,119 @@ def test_validator_rejects_bad_sequences():
         v = schema.vocab
         swapped = list(v.pfx) + tool.name + list(v.mid) + tool.keys[1] + list(v.kvsep)
         assert tool.keys[0] == tool.keys[1] or not oracle.validate_prefix(schema, swapped)
+
+
+# ---- candidate sets and PackDraftsAsTree (Algorithm 1; Appendix B.2's continuation lengths) --------------
+def test_continuation_lengths_are_the_printed_ones():
+    g = _gold()
+    assert tuple(int(x) for x in g["continuation_lengths"].split()) == (oracle.DEFAULT_N_CAP,) + oracle.drafter.LATER_CAPS
+
+
+def _brute_force_hits(y, entries, order, caps, max_draft):
+    hits = []
+    for L in (5, 6, 7):
+        if len(y) < L:
+            continue
+        for rank, c in enumerate(order):
+            e = entries[c]
+            for m in range(L, len(e)):
+                if e[m - L:m] == list(y[-L:]):
+                    hits.append((-L, rank, m, c))
+    out, seen = [], set()
+    for negL, rank, m, c in sorted(hits):
+        if (c, m) in seen:
+            continue
+        seen.add((c, m))
+        out.append(entries[c][m:m + min(caps[len(out)], max_draft)])
+        if len(out) == len(caps):
+            break
+    return out
+
+
+def test_suffix_matches_equal_brute_force_and_start_with_the_chain_draft():
+    rnd = random.Random(11)
+    nonempty = 0
+    for trial in range(300):
+        alphabet = rnd.choice([2, 3, 5])
+        n_e = rnd.randint(1, 6)
+        st = oracle.Datastore(1)
+        for _ in range(n_e):
+            st.add([rnd.randrange(alphabet) for _ in range(rnd.randint(1, 40))], 0)
+        y = [rnd.randrange(alphabet) for _ in range(rnd.randint(0, 12))]
+        ranks = None if trial % 2 else rnd.sample(range(n_e), rnd.randint(1, n_e))
+        caps = (rnd.choice([1, 4, 32]), 16, 8, 8)
+        max_draft = rnd.choice([1, 7, 63])
+        got = oracle.suffix_matches(y, st, ranks, caps, max_draft)
+        order = list(range(n_e)) if ranks is None else ranks
+        assert got == _brute_force_hits(y, st.entries, order, caps, max_draft)
+        first, _ = oracle.suffix_match(y, st, ranks, caps[0], max_draft)
+        assert (got[0] if got else []) == first
+        nonempty += len(got) > 1
+    assert nonempty > 20          # several hits do occur in this sweep
+
+
+def _leaf_paths(tokens, parents):
+    kids = {}
+    for j in range(1, len(parents)):
+        kids.setdefault(parents[j], []).append(j)
+    out = []
+
+    def walk(u, acc):
+        if u not in kids:
+            out.append(acc)
+        for c in kids.get(u, []):
+            walk(c, acc + [tokens[c - 1]])
+    walk(0, [])
+    return out
+
+
+def test_tool_name_candidates_are_valid_and_cover_the_guess():
+    schema = _schema(seed=3, n_tools=12)
+    st, inv = _store(schema, seed=3)
+    v = schema.vocab
+    for tid, toks in inv[:30]:
+        d = oracle.Drafter(schema, oracle.Datastore(len(schema.tools)))       # no retrieval
+        d.feed_prompt([77, v.tool_call])
+        for i, t in enumerate(toks):
+            cands, src = d.draft_candidates(63)
+            chain, csrc = d.draft(63)
+            assert (cands[0] if cands else []) == chain and src == csrc       # first candidate = chain draft
+            toks_t, par_t, _ = d.draft_tree(64)
+            for leaf in _leaf_paths(toks_t, par_t):
+                assert oracle.validate_prefix(schema, toks[:i] + leaf), (tid, i, leaf)
+            if d.fsm.kind == Q_T and d.fsm.stage != "mid":
+                # with the name open, the true tool is among the candidates whenever at most
+                # MAX_TOOL_CANDIDATES tools are compatible, and then its whole scaffold is a root path
+                prefix = [] if d.fsm.stage == "pfx" else d.fsm.name_prefix
+                comp = d.fsm.compatible_tools(prefix)
+                assert len(cands) == min(len(comp), oracle.drafter.MAX_TOOL_CANDIDATES)
+                if len(comp) <= oracle.drafter.MAX_TOOL_CANDIDATES:
+                    truth = d.fsm.draft(lambda _p: tid)
+                    assert truth in cands and toks[i:i + len(truth)] == truth
+            else:
+                assert len(cands) <= 1
+            d.commit([t], v.eos, 10 ** 6)
+
+
+def test_tree_loop_equals_vanilla_greedy_on_a_tiny_model():
+    """Algorithm 1 with candidate trees preserves the model's output (Section 5.2, Table 5)."""
+    import torch  # noqa: F401
+    from test_oracle_pins import _small_shape, _rand_weights
+    shape = _small_shape(vocab=4096)
+    om = oracle.OracleModel(shape, _rand_weights(shape, seed=9))
+    schema = _schema(seed=4, n_tools=8)
+    v = schema.vocab
+    st, inv = _store(schema, n=32, seed=4)
+    prompt = synth.make_context(4096, 24, seed=4)
+    ref = oracle.vanilla_greedy(om, schema, prompt, v.eos, 40)
+    # self-history: the model's own output, intact and with planted errors, among the historical invocations
+    bad = list(ref)
+    for p in (8, 19, 30):
+        bad[p] = (bad[p] + 1) % 4096
+    for e in (bad, ref, ref[:15] + bad[15:]):
+        st.add(e, -1)
+    trace = []
+    out = oracle.speculative_decode_tree(om, schema, st, prompt, v.eos, 40, max_nodes=24, trace=trace)
+    assert out == ref
+    assert len(trace) < len(ref)                                     # drafts were accepted
+    assert any(len(set(t["parents"])) < len(t["parents"]) for t in trace)       # and some trees did branch
