@@ -183,6 +183,19 @@ ts_status ts_verify(ts_model *m, ts_session *const *sessions, int32_t B,
                     const int32_t *draft_tokens, const int32_t *draft_offsets, uint32_t flags,
                     ts_verify_result *out);
 
+/* ts_draft_tree — the candidate set B of Algorithm 1 packed as a tree (PackDraftsAsTree).  Retrieval first: up to
+ * four continuations of the suffix match, taken in the order (L = 7, 6, 5; candidate rank; match position), a
+ * position already taken at a longer L skipped, of at most n_cap, 16, 8 and 8 ids (Appendix B.2's lengths).  If
+ * retrieval yields nothing: the schema drafts (Section 4.2) -- with the tool name still open, one chain per tool
+ * whose name extends the ids emitted so far (Eq. 2; the tool ts_draft would guess first, then ascending tool id,
+ * at most 8 tools); otherwise ts_draft's single chain.  The chains are merged into a token trie: node 0 is the
+ * pending token, nodes are numbered in creation order, nothing is added once the chunk holds max_nodes nodes
+ * (<= TS_K_MAX).  out_tokens[j], out_parents[j]: token and parent node of node j + 1, in the form ts_verify_tree
+ * takes; *out_n = nodes after the root; *out_source: 0 none, 1 schema, 2 retrieval.  The first root-to-leaf path
+ * is ts_draft's chain.  Host only; never fails on "no draft". */
+ts_status ts_draft_tree(ts_session *s, int32_t max_nodes, int32_t *out_tokens, int32_t *out_parents,
+                        int32_t *out_n, int32_t *out_source);
+
 /* ts_verify_tree — PackDraftsAsTree's output verified in one forward pass under the tree-structured attention
  * mask (Appendix A.1 "Parallel Verification"; Algorithm 1: Verification, SelectLongestAcceptedPrefix).
  * Sequence i's chunk has node 0 = its pending token and node j+1 = draft_tokens[draft_offsets[i] + j], whose

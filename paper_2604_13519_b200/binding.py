@@ -94,6 +94,7 @@ _SIGNATURES = {
     "ts_session_destroy": [_P],
     "ts_prefill": [_P, _P, _I32P, C.c_int32],
     "ts_draft": [_P, C.c_int32, _I32P, _I32P, _I32P],
+    "ts_draft_tree": [_P, C.c_int32, _I32P, _I32P, _I32P, _I32P],
     "ts_verify": [_P, C.POINTER(_P), C.c_int32, _I32P, _I32P, C.c_uint32, C.POINTER(ts_verify_result)],
     "ts_verify_tree": [_P, C.POINTER(_P), C.c_int32, _I32P, _I32P, _I32P, C.c_uint32, C.POINTER(ts_verify_result),
                        _I32P],
@@ -371,6 +372,15 @@ def ts_verify(model: Model, sessions: Sequence[Session], drafts: Sequence[Sequen
     out = (ts_verify_result * B)()
     _check(lib().ts_verify(model.h, hs, B, _i32(flat), _i32(offs), flags, out))
     return list(out)
+
+
+def ts_draft_tree(session: Session, max_nodes: int):
+    """(tokens of nodes 1.., parent node of each of them, source)."""
+    toks = (C.c_int32 * TS_K_MAX)()
+    par = (C.c_int32 * TS_K_MAX)()
+    n, src = C.c_int32(0), C.c_int32(0)
+    _check(lib().ts_draft_tree(session.h, max_nodes, toks, par, C.byref(n), C.byref(src)))
+    return list(toks[:n.value]), list(par[:n.value]), src.value
 
 
 def ts_verify_tree(model: Model, sessions: Sequence[Session], drafts: Sequence[Sequence[int]],

@@ -218,4 +218,74 @@ void suffix_match(const std::vector<int32_t> &y, const ts_datastore &d, const st
   }
 }
 
+void suffix_matches(const std::vector<int32_t> &y, const ts_datastore &d, const std::vector<int32_t> *ranks,
+                    const int32_t *caps, int32_t n_caps, int32_t max_draft, std::vector<std::vector<int32_t>> *out) {
+  out->clear();
+  const int32_t ny = (int32_t)y.size();
+  if (max_draft <= 0 || n_caps <= 0 || ny < 5 || d.n_entries() == 0) return;
+  const int32_t *tail = y.data() + ny;
+  auto matches = [&](const int32_t *p, int32_t m, int32_t L) {
+    return m >= L && std::memcmp(p + m - L, tail - L, sizeof(int32_t) * L) == 0;
+  };
+  std::vector<std::pair<int32_t, int32_t>> taken;   // (entry, m) of the hits so far: at most n_caps
+  auto take = [&](int32_t c, const int32_t *p, int32_t len, int32_t m) -> bool {   // true once the set is full
+    for (const auto &t : taken)
+      if (t.first == c && t.second == m) return false;
+    taken.push_back({c, m});
+    const int32_t n = std::min(caps[out->size()], max_draft);
+    out->emplace_back(p + m, p + std::min(len, m + n));
+    return (int32_t)out->size() == n_caps;
+  };
+  if (ranks) {
+    for (int32_t L = 7; L >= 5; --L) {
+      if (ny < L) continue;
+      for (int32_t c : *ranks) {
+        int32_t len;
+        const int32_t *p = d.entry(c, &len);
+        for (int32_t m = L; m < len; ++m)
+          if (matches(p, m, L) && take(c, p, len, m)) return;
+      }
+    }
+    return;
+  }
+  d.ensure_index();
+  ts_datastore::Posting probe{gram_key(tail - 5), INT32_MIN, INT32_MIN};
+  auto lo = std::lower_bound(d.index.begin(), d.index.end(), probe,
+                             [](const ts_datastore::Posting &a, const ts_datastore::Posting &b) {
+                               if (a.key != b.key) return a.key < b.key;
+                               if (a.entry != b.entry) return a.entry < b.entry;
+                               return a.m < b.m;
+                             });
+  for (int32_t L = 7; L >= 5; --L) {
+    if (ny < L) continue;
+    for (auto it = lo; it != d.index.end() && it->key == probe.key; ++it) {
+      int32_t len;
+      const int32_t *p = d.entry(it->entry, &len);
+      if (matches(p, it->m, L) && take(it->entry, p, len, it->m)) return;
+    }
+  }
+}
+
+void pack_candidates(const std::vector<std::vector<int32_t>> &cands, int32_t max_nodes, std::vector<int32_t> *tokens,
+                     std::vector<int32_t> *parents) {
+  tokens->clear();
+  parents->clear();
+  // children of node u are found by scanning the nodes created so far (a chunk has at most 64 nodes)
+  for (const auto &cand : cands) {
+    int32_t u = 0;
+    for (int32_t t : cand) {
+      int32_t nxt = -1;
+      for (size_t j = 0; j < tokens->size(); ++j)
+        if ((*parents)[j] == u && (*tokens)[j] == t) { nxt = (int32_t)j + 1; break; }
+      if (nxt < 0) {
+        if ((int32_t)tokens->size() + 1 >= max_nodes) break;
+        tokens->push_back(t);
+        parents->push_back(u);
+        nxt = (int32_t)tokens->size();
+      }
+      u = nxt;
+    }
+  }
+}
+
 }  // namespace ts

@@ -72,4 +72,16 @@ struct Fsm {
 void suffix_match(const std::vector<int32_t> &y, const ts_datastore &d, const std::vector<int32_t> *ranks,
                   int32_t n, std::vector<int32_t> *out);
 
+// The retrieval candidate set: hits in the order (L descending, candidate rank ascending, position ascending), a
+// position already taken at a longer L skipped; hit i contributes at most caps[i] ids (and at most max_draft);
+// at most n_caps continuations.  The first one equals suffix_match's draft for n = min(caps[0], max_draft).
+void suffix_matches(const std::vector<int32_t> &y, const ts_datastore &d, const std::vector<int32_t> *ranks,
+                    const int32_t *caps, int32_t n_caps, int32_t max_draft, std::vector<std::vector<int32_t>> *out);
+
+// PackDraftsAsTree: merge candidate chains into a token trie, nodes numbered in creation order (node 0 = the
+// pending token), no node added once the chunk holds max_nodes nodes.  tokens: nodes 1..; parents: parent of
+// node j + 1 at index j.
+void pack_candidates(const std::vector<std::vector<int32_t>> &cands, int32_t max_nodes, std::vector<int32_t> *tokens,
+                     std::vector<int32_t> *parents);
+
 }  // namespace ts

@@ -37,6 +37,7 @@ ts_status fail(ts_status code, const char *fmt, ...) {
 inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
 constexpr int kMaxSplits = 12;
+constexpr int kMaxToolCandidates = 8;   // tool names verified in parallel while the name is open
 constexpr int kMaxAttnSplits = ts::kAttnMaxSplits;
 constexpr int kMcOptions[4] = {16, 32, 64, 128};
 constexpr int kMaxFusedCtas = 256;   // the fused kernel runs one CTA per SM
@@ -992,6 +993,57 @@ ts_status ts_draft(ts_session *s, int32_t max_draft, int32_t *out_tokens, int32_
   }
   std::memcpy(out_tokens, d.data(), d.size() * sizeof(int32_t));
   *out_n = (int32_t)d.size();
+  return TS_OK;
+}
+
+ts_status ts_draft_tree(ts_session *s, int32_t max_nodes, int32_t *out_tokens, int32_t *out_parents, int32_t *out_n,
+                        int32_t *out_source) {
+  if (!s || !out_n || !out_source || (max_nodes > 1 && (!out_tokens || !out_parents)))
+    return fail(TS_ERR_ARG, "null argument");
+  *out_n = 0; *out_source = 0;
+  if (max_nodes > TS_K_MAX) return fail(TS_ERR_K_TOO_LARGE, "a draft tree holds at most %d nodes", TS_K_MAX);
+  const int max_draft = max_nodes - 1;
+  if (max_draft <= 0 || s->finished) return TS_OK;
+  std::vector<std::vector<int32_t>> cands;
+  int source = 0;
+  if (s->store) {
+    const int32_t caps[4] = {s->cfg.n_cap, 16, 8, 8};   // Appendix B.2: continuation lengths in candidate order
+    ts::suffix_matches(s->y, *s->store, s->have_ranks ? &s->ranks : nullptr, caps, 4, max_draft, &cands);
+    if (!cands.empty()) source = 2;
+  }
+  if (cands.empty() && s->schema) {
+    std::vector<int32_t> d;
+    if (s->fsm.kind == ts::Q_T && s->fsm.stage != ts::ST_MID) {
+      // one chain per tool whose name extends what was emitted so far: the guessed tool first, then ascending ids
+      const int guess = guess_tool(s);
+      if (guess >= 0) {
+        const ts::TrieNode &node = s->schema->trie[s->fsm.stage == ts::ST_NAME ? s->fsm.node : 0];
+        std::vector<int32_t> order{guess};
+        for (int32_t t : node.tools)
+          if (t != guess && (int)order.size() < kMaxToolCandidates) order.push_back(t);
+        for (int32_t t : order) {
+          s->fsm.draft(t, &d);
+          if ((int)d.size() > max_draft) d.resize(max_draft);
+          cands.push_back(d);
+        }
+      } else {
+        s->fsm.draft(-1, &d);
+        if ((int)d.size() > max_draft) d.resize(max_draft);
+        if (!d.empty()) cands.push_back(d);
+      }
+    } else {
+      s->fsm.draft(-1, &d);
+      if ((int)d.size() > max_draft) d.resize(max_draft);
+      if (!d.empty()) cands.push_back(d);
+    }
+    if (!cands.empty()) source = 1;
+  }
+  std::vector<int32_t> toks, par;
+  ts::pack_candidates(cands, max_nodes, &toks, &par);
+  std::memcpy(out_tokens, toks.data(), toks.size() * sizeof(int32_t));
+  std::memcpy(out_parents, par.data(), par.size() * sizeof(int32_t));
+  *out_n = (int32_t)toks.size();
+  *out_source = toks.empty() ? 0 : source;
   return TS_OK;
 }
 

@@ -148,3 +148,57 @@ def test_tree_argument_errors():
         ts.ts_verify_tree(gm2, [s2], [[100]], [[0]])
     assert e.value.code == -8
     gm2.close()
+
+
+def test_tree_decode_loop_follows_the_oracle():
+    """Algorithm 1's loop with candidate trees on the tiny decoder: ts_draft_tree -> ts_verify_tree ->
+    ts_commit against the oracle's trajectory, real prefill on both sides, self-history in the datastore
+    so that retrieved branches are accepted fully and partially."""
+    shape = synth.SHAPES["tiny"]
+    om, gm = make_pair(shape, k_max=24, max_ctx=512, path=1)
+    schema = synth.make_schema(shape.vocab, 8)
+    inv = synth.make_datastore(schema, 64)
+    v = schema.vocab
+    prompt = synth.make_context(shape.vocab, 200)
+    y_ref = oracle.vanilla_greedy(om, schema, prompt, v.eos, 60)
+    bad = list(y_ref)
+    for p in (9, 17, 22, 40):
+        bad[p] = (bad[p] + 1) % shape.vocab
+    inv = inv + [(-1, bad), (-1, y_ref), (-1, y_ref[:30] + bad[30:])]
+    st_o, st_c = oracle.Datastore(len(schema.tools)), ts.Datastore(len(schema.tools))
+    for tid, toks in inv:
+        st_o.add(toks, tid)
+        st_c.add(toks, tid)
+    sc = ts.Schema(schema.vocab, schema.tools)
+    d = oracle.Drafter(schema, st_o)
+    d.feed_prompt(prompt)
+    cache, pending = oracle.prefill(om, prompt)
+    s = ts.Session(gm, sc, st_c, max_new_tokens=60)
+    ts.ts_prefill(gm, s, prompt)
+    accepted, branched = [], 0
+    for step in range(30):
+        wt, wp, wsrc = d.draft_tree(24)
+        gt, gp, gsrc = ts.ts_draft_tree(s, 24)
+        assert (gt, gp, gsrc) == (wt, wp[1:], wsrc)
+        branched += len(set(wp)) < len(wp)
+        n0 = cache.length
+        ref = oracle.verify_tree(om, pending, wt, wp, cache, want_logits=True)
+        res, paths = ts.ts_verify_tree(gm, [s], [gt], [gp])
+        same = _check_tree(res[0], paths[0], gm.read_logits(0, len(wt) + 1), ref, f"loop step {step}")
+        if not same:
+            break                                          # permitted near-tie: the trajectories part
+        used, fin = d.commit(ref["emitted"], v.eos, 60)
+        cache.truncate(n0 + used)
+        ts.ts_commit(s, res[0])
+        pending = ref["emitted"][used - 1]
+        info = s.state()
+        assert (info.cache_len, info.pending, bool(info.finished)) == (cache.length, pending, fin)
+        accepted.append(ref["accept_len"])
+        if fin:
+            break
+    else:
+        raise AssertionError("the generation did not finish in 30 steps")
+    if same:
+        assert s.output() == d.y == y_ref[:len(d.y)]
+        assert max(accepted) >= 8 and branched >= 1
+    gm.close()

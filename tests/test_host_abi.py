@@ -94,6 +94,11 @@ def test_draft_and_commit_bit_exact_with_oracle(seed, n_tools, n_inv, ranks):
             want, src = d.draft(md)
             got, gsrc = ts.ts_draft(s, md)
             assert (got, gsrc) == (want, src), (trial, pos)
+            # the candidate set packed as a tree: same nodes, same parents, same source
+            mn = rnd.choice([1, 2, 9, 24, 64])
+            wt, wp, wsrc = d.draft_tree(mn)
+            gt, gp, gtsrc = ts.ts_draft_tree(s, mn)
+            assert (gt, gp, gtsrc) == (wt, wp[1:], wsrc), (trial, pos, mn)
             n = rnd.randrange(1, 8)
             span = script[pos:pos + n]
             used, fin = d.commit(span, v.eos, 200)
@@ -126,9 +131,13 @@ def test_large_store_whole_index_search():
         ts.ts_commit_forced(s, d.y)
         want, _ = oracle.suffix_match(d.y, d.store, None, 64, 63)
         got, src = ts.ts_draft(s, 63)
+        wt, wp, wsrc = d.draft_tree(64)
+        gt, gp, gtsrc = ts.ts_draft_tree(s, 64)
+        assert (gt, gp, gtsrc) == (wt, wp[1:], wsrc)
         if want:
             hits += 1
             assert src == 2 and got == want
+            assert gtsrc == 2 and gt[:len(want)] == want[:len(gt)]      # the chain draft is the first branch
         else:
             assert src != 2
     assert hits > 20
