@@ -148,6 +148,20 @@ class ClockSampler:
                     samples=len(sm))
 
 
+def tree_parents(k):
+    """Parent node of each of the k - 1 draft nodes: four chains hanging from the root (node 0), of about
+    1/2, 1/4, 1/8 and 1/8 of the drafts -- the proportions of the 32/16/8/8 continuation lengths."""
+    n = k - 1
+    lens = [n - n // 2, n // 2 - n // 4, n // 4 - n // 8, n // 8]
+    par, node = [], 1
+    for ln in lens:
+        for j in range(ln):
+            par.append(0 if j == 0 else node - 1)
+            node += 1
+    assert len(par) == n
+    return par
+
+
 def dist_env():
     return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
 
@@ -274,6 +288,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-act-split", action="store_true")
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 one kernel per stage, 2 single persistent kernel")
+    ap.add_argument("--tree", action="store_true",
+                    help="verify each chunk as a draft tree (four branches from the root, lengths about 1/2, 1/4, 1/8, "
+                         "1/8 of the drafts: the shape of the retrieval candidate set) through ts_verify_tree")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -299,6 +316,12 @@ def main():
     M = sum(ks)
     drafts = [[64 + (7 * j + i) % (shape.vocab - 64) for j in range(k - 1)] for i, k in enumerate(ks)]
     stream = torch.cuda.current_stream()
+    parents = [tree_parents(k) for k in ks] if args.tree else None
+
+    def verify():
+        if parents is None:
+            return ts.ts_verify(model, sessions, drafts)
+        return ts.ts_verify_tree(model, sessions, drafts, parents)
 
     def barrier():
         if world > 1:
@@ -307,12 +330,12 @@ def main():
 
     # ---- e2e arm: the public call with host buffers --------------------------------------------
     for _ in range(args.warmup):
-        ts.ts_verify(model, sessions, drafts)
+        verify()
     l0, h0, d0 = model.counters()
     barrier()
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        ts.ts_verify(model, sessions, drafts)
+        verify()
     torch.cuda.synchronize()
     e2e_ms = 1e3 * (time.perf_counter() - t0) / args.steps
     l1, h1, d1 = model.counters()
@@ -414,7 +437,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload, "batch": len(lens), "context": lens, "k": ks,
-                       "act_split": planes == 2, "kv_dtype": "f16", "l2": "inputs (weights) far larger than L2",
+                       "act_split": planes == 2, "draft_tree": bool(args.tree), "kv_dtype": "f16", "l2": "inputs (weights) far larger than L2",
                        "parallelism": "replicas" if world > 1 else "single"},
             "latency_ms": {"p50": statistics.median(lat), "p90": sorted(lat)[int(0.9 * (len(lat) - 1))]},
             "clocks": clocks,
