@@ -37,6 +37,7 @@ WORKLOADS = {
     "c5_8b_b4_ctx8192_k64": ("8b", [8192] * 4, [64] * 4),
     # reduced-depth case for profiler captures (same per-layer kernels and grids as c3)
     "prof_8b4l_ctx8192_k32": ("8b-4l", [8192], [32]),
+    "prof_8b4l_b4_ctx2048_k64": ("8b-4l", [2048] * 4, [64] * 4),
 }
 DEFAULT_WORKLOAD = "c3_8b_ctx8192_k32"
 METRIC = "verified_tokens_per_s"
