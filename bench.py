@@ -289,6 +289,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-act-split", action="store_true")
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 one kernel per stage, 2 single persistent kernel")
+    ap.add_argument("--temperature", type=float, default=0.0,
+                    help="> 0: speculative-sampling acceptance at this temperature (ts_verify_sampled) with fixed uniforms")
     ap.add_argument("--tree", action="store_true",
                     help="verify each chunk as a draft tree (four branches from the root, lengths about 1/2, 1/4, 1/8, "
                          "1/8 of the drafts: the shape of the retrieval candidate set) through ts_verify_tree")
@@ -319,7 +321,11 @@ def main():
     stream = torch.cuda.current_stream()
     parents = [tree_parents(k) for k in ks] if args.tree else None
 
+    uniforms = [((37 * r + 11) % 100) / 100.0 for r in range(M)]
+
     def verify():
+        if args.temperature > 0:
+            return ts.ts_verify_sampled(model, sessions, drafts, args.temperature, uniforms)
         if parents is None:
             return ts.ts_verify(model, sessions, drafts)
         return ts.ts_verify_tree(model, sessions, drafts, parents)
@@ -438,7 +444,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload, "batch": len(lens), "context": lens, "k": ks,
-                       "act_split": planes == 2, "draft_tree": bool(args.tree), "kv_dtype": "f16", "l2": "inputs (weights) far larger than L2",
+                       "act_split": planes == 2, "draft_tree": bool(args.tree), "temperature": args.temperature, "kv_dtype": "f16", "l2": "inputs (weights) far larger than L2",
                        "parallelism": "replicas" if world > 1 else "single"},
             "latency_ms": {"p50": statistics.median(lat), "p90": sorted(lat)[int(0.9 * (len(lat) - 1))]},
             "clocks": clocks,

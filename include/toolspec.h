@@ -216,6 +216,21 @@ ts_status ts_verify_tree(ts_model *m, ts_session *const *sessions, int32_t B,
                          const int32_t *draft_offsets, uint32_t flags, ts_verify_result *out,
                          int32_t *path_out);
 
+/* ts_verify_sampled — ts_verify with speculative sampling as the acceptance rule (Appendix B.2) at temperature
+ * T > 0 instead of the greedy match.  The drafts are deterministic, so the draft distribution is a point mass on
+ * the drafted id x: row j accepts draft j + 1 = x with probability p_j(x), p_j = softmax(logits_j / T); the first
+ * rejection emits one sample of p_j with x removed (renormalised) and ends the step; if all drafts pass, one sample
+ * of the last row's p is emitted.  The emitted ids are then distributed as token-by-token sampling from the model.
+ * uniforms (host): one value in [0, 1) per chunk row, rows in the order of the chunks (draft_offsets[B] + B values);
+ * within a chunk of k rows, value j < k - 1 decides draft j + 1 (accepted iff it is below p_j(x)) and value k - 1
+ * draws the step's one sample: the smallest id whose running sum of weights exp((l - max) / T), in id order,
+ * exceeds it times the total.  The library draws no random numbers.  out[i] as ts_verify (argmax still reports
+ * the per-row argmax).  Runs on the one-kernel-per-stage path (TS_ERR_UNIMPLEMENTED with path = 2); TS_ERR_ARG for
+ * a temperature outside (0, 1e4) or a uniform outside [0, 1).  Other errors as ts_verify. */
+ts_status ts_verify_sampled(ts_model *m, ts_session *const *sessions, int32_t B,
+                            const int32_t *draft_tokens, const int32_t *draft_offsets, float temperature,
+                            const float *uniforms, uint32_t flags, ts_verify_result *out);
+
 /* Enqueue again the device work of the last ts_verify call on its inputs, which are still resident
  * in device memory; no host<->device copy, no synchronisation.  The step is idempotent because
  * sessions advance only in ts_commit.  For timing the kernels alone. */

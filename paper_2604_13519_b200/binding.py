@@ -98,6 +98,8 @@ _SIGNATURES = {
     "ts_verify": [_P, C.POINTER(_P), C.c_int32, _I32P, _I32P, C.c_uint32, C.POINTER(ts_verify_result)],
     "ts_verify_tree": [_P, C.POINTER(_P), C.c_int32, _I32P, _I32P, _I32P, C.c_uint32, C.POINTER(ts_verify_result),
                        _I32P],
+    "ts_verify_sampled": [_P, C.POINTER(_P), C.c_int32, _I32P, _I32P, C.c_float, C.POINTER(C.c_float), C.c_uint32,
+                          C.POINTER(ts_verify_result)],
     "ts_verify_replay": [_P],
     "ts_profile_step": [_P, C.POINTER(C.c_float), _I32P, C.c_int32],
     "ts_commit": [_P, C.POINTER(ts_verify_result)],
@@ -400,6 +402,22 @@ def ts_verify_tree(model: Model, sessions: Sequence[Session], drafts: Sequence[S
     _check(lib().ts_verify_tree(model.h, hs, B, _i32(flat), _i32(par), _i32(offs), flags, out, path))
     paths = [[path[i * TS_K_MAX + j] for j in range(out[i].accept_len + 1)] for i in range(B)]
     return list(out), paths
+
+
+def ts_verify_sampled(model: Model, sessions: Sequence[Session], drafts: Sequence[Sequence[int]],
+                      temperature: float, uniforms: Sequence[float], flags: int = 0):
+    """Speculative-sampling acceptance; uniforms: one value in [0, 1) per chunk row, chunk after chunk."""
+    B = len(sessions)
+    hs = (_P * B)(*[s.h for s in sessions])
+    flat, offs = [], [0]
+    for d in drafts:
+        flat += list(d)
+        offs.append(len(flat))
+    assert len(uniforms) == len(flat) + B
+    u = (C.c_float * len(uniforms))(*uniforms)
+    out = (ts_verify_result * B)()
+    _check(lib().ts_verify_sampled(model.h, hs, B, _i32(flat), _i32(offs), temperature, u, flags, out))
+    return list(out)
 
 
 def ts_verify_replay(model: Model):

@@ -108,6 +108,20 @@ struct AcceptArgs {
 };
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t st);
 
+// Speculative-sampling acceptance (sampling.cu): per-row softmax statistics, accept tests, the step's one sample.
+struct SampleArgs {
+  StepIn in;
+  const float *logits;              // [M][V]
+  const unsigned long long *amax;   // [M] packed per-row maxima (argmax is still reported)
+  const float *uni;                 // [M] uniforms in [0, 1): row j of a chunk decides draft j + 1, the last row's draws the sample
+  float *part;                      // [M][16] scratch: per-slice sums of exp((l - max) / T)
+  int V;
+  float inv_t;                      // 1 / temperature
+  int32_t *argmax, *accept_len, *emitted, *new_len, *new_pending, *path;
+  int k_max;
+};
+cudaError_t launch_sample_accept(const SampleArgs &a, cudaStream_t st);
+
 // After a tree step: move the K/V rows of the accepted path to consecutive cache positions len, len+1, ...
 struct CompactArgs {
   StepIn in;

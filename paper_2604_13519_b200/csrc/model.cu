@@ -58,7 +58,8 @@ struct Layout {
   int n_maps, n_counters, n_phases, max_tiles128, o_tile128_seq, o_tile128_row0;
   // step io (int32 offsets inside d_in / h_in)
   int o_tokens, o_pos, o_rowseq, o_cu, o_len, o_tile_seq, o_tile_row0, o_btab, in_ints;
-  int o_parent, o_anc, o_path;
+  int o_parent, o_anc, o_path, o_uni;
+  uint64_t samp_stats;
   // step out (int32 offsets)
   int o_argmax, o_accept, o_emitted, o_newlen, o_newpend, o_err, out_ints;
   int rows_alloc, pages_per_seq, max_tiles, Nqkv, n_vocab_tiles;
@@ -126,6 +127,7 @@ void make_layout(const ts_model_config &c, Layout *L) {
   L->act = take(planes * R * F * 2);
   L->logits = take(R * V * 4);
   L->amax = take(R * 8);
+  L->samp_stats = take(R * 16 * 4);
   L->rope = take((uint64_t)c.max_ctx * (hd / 2) * 8);
   int io = 0;
   auto itake = [&](int n) { int r = io; io += (n + 3) / 4 * 4; return r; };
@@ -134,7 +136,7 @@ void make_layout(const ts_model_config &c, Layout *L) {
   L->o_tile_seq = itake(L->max_tiles); L->o_tile_row0 = itake(L->max_tiles);
   L->max_tiles128 = c.max_batch * ((c.k_max * G + 127) / 128);
   L->o_tile128_seq = itake(L->max_tiles128); L->o_tile128_row0 = itake(L->max_tiles128);
-  L->o_parent = itake(c.max_rows); L->o_anc = itake(2 * c.max_rows);
+  L->o_parent = itake(c.max_rows); L->o_anc = itake(2 * c.max_rows); L->o_uni = itake(c.max_rows);
   L->o_btab = itake(c.max_batch * L->pages_per_seq);   // (last: only the used part is copied per step)
   L->in_ints = io;
   io = 0;
@@ -195,6 +197,8 @@ struct ts_model {
   bool use_pdl = true;
   bool fused_ok = false, last_fused = false;   // device can run the fused kernel; the staged step uses it
   bool last_tree = false;                      // the staged step verifies a draft tree (not a chain)
+  bool last_sample = false;                    // the staged step accepts by speculative sampling
+  float last_inv_t = 1.f;                      // 1 / temperature of that step
   size_t smem_optin = 0;
   // per-kernel timing pass (ts_profile_step): one event after every launch
   bool profiling = false;
@@ -496,8 +500,20 @@ ts_status run_step(ts_model *m) {
   ts_status s = run_gemm(m, ts::EPI_LOGITS, m->tm_lm, m->tm_h, c.vocab, d, M, (float *)m->WS(L.logits), nullptr,
                          amax, nullptr);
   if (s) return s;
-  ts::AcceptArgs ac{};
   int32_t *dout = m->d_out();
+  if (m->last_sample) {
+    ts::SampleArgs sa{};
+    sa.in = in; sa.logits = (const float *)m->WS(L.logits); sa.amax = amax;
+    sa.uni = (const float *)(di + L.o_uni); sa.part = (float *)m->WS(L.samp_stats);
+    sa.V = c.vocab; sa.inv_t = m->last_inv_t; sa.k_max = c.k_max;
+    sa.argmax = dout + L.o_argmax; sa.accept_len = dout + L.o_accept; sa.emitted = dout + L.o_emitted;
+    sa.new_len = dout + L.o_newlen; sa.new_pending = dout + L.o_newpend; sa.path = dout + L.o_path;
+    CU_TRY(ts::launch_sample_accept(sa, m->st));
+    m->launched(5);
+    m->launched(5);
+    return TS_OK;
+  }
+  ts::AcceptArgs ac{};
   ac.in = in; ac.amax = amax;
   ac.argmax = dout + L.o_argmax; ac.accept_len = dout + L.o_accept; ac.emitted = dout + L.o_emitted;
   ac.new_len = dout + L.o_newlen; ac.new_pending = dout + L.o_newpend; ac.k_max = c.k_max;
@@ -530,7 +546,8 @@ ts_status ensure_pages(ts_session *s, int tokens) {
 // Stage one step: rows[i] = chunk ids of sequence i.  Copies inputs, runs, copies results back, syncs.
 // parents (optional): parents[i][j] = chunk row that row j of sequence i hangs from (-1 for row 0); a chain if null.
 ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::vector<std::vector<int32_t>> &rows,
-                        uint32_t flags, const std::vector<std::vector<int32_t>> *parents = nullptr) {
+                        uint32_t flags, const std::vector<std::vector<int32_t>> *parents = nullptr,
+                        const float *uniforms = nullptr, float temperature = 0.f) {
   const ts_model_config &c = m->c;
   const Layout &L = m->L;
   int32_t *hi = m->h_in();
@@ -600,7 +617,14 @@ ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::ve
   m->last_tree = parents != nullptr;
   if (m->last_tree && (c.path == 2 || !m->fused_ok))
     return fail(TS_ERR_UNIMPLEMENTED, "draft trees need the one-kernel-per-stage path with tensor-memory attention");
-  m->last_fused = !m->last_tree && can_fuse && (c.path == 2 || (c.path == 0 && kAutoPrefersFused));
+  m->last_sample = uniforms != nullptr;
+  if (m->last_sample) {
+    if (c.path == 2) return fail(TS_ERR_UNIMPLEMENTED, "sampling acceptance needs the one-kernel-per-stage path");
+    if (m->last_tree) return fail(TS_ERR_UNIMPLEMENTED, "sampling acceptance over a draft tree");
+    m->last_inv_t = 1.f / temperature;
+    std::memcpy(hi + L.o_uni, uniforms, sizeof(float) * M);
+  }
+  m->last_fused = !m->last_tree && !m->last_sample && can_fuse && (c.path == 2 || (c.path == 0 && kAutoPrefersFused));
   m->last_B = B; m->last_M = M; m->last_tiles = tiles; m->last_tiles128 = tiles128; m->last_flags = flags;
   m->have_step = true;
   const size_t in_bytes = (size_t)(L.o_btab + (size_t)B * L.pages_per_seq) * 4;
@@ -1051,7 +1075,8 @@ namespace {
 // ts_verify and ts_verify_tree: draft_parents = nullptr for chains
 ts_status verify_impl(ts_model *m, ts_session *const *ss, int32_t B, const int32_t *draft_tokens,
                       const int32_t *draft_parents, const int32_t *draft_offsets, uint32_t flags,
-                      ts_verify_result *out, int32_t *path_out) {
+                      ts_verify_result *out, int32_t *path_out, const float *uniforms = nullptr,
+                      float temperature = 0.f) {
   if (!m || !ss || !draft_offsets || !out) return fail(TS_ERR_ARG, "null argument");
   if (B < 1 || B > m->c.max_batch) return fail(TS_ERR_ARG, "batch %d outside [1, %d]", B, m->c.max_batch);
   std::vector<std::vector<int32_t>> rows(B), parents(B);
@@ -1073,7 +1098,7 @@ ts_status verify_impl(ts_model *m, ts_session *const *ss, int32_t B, const int32
       for (int j = 0; j < n; ++j) parents[i].push_back(draft_parents[draft_offsets[i] + j]);
     }
   }
-  ts_status st = stage_and_run(m, ss, B, rows, flags, draft_parents ? &parents : nullptr);
+  ts_status st = stage_and_run(m, ss, B, rows, flags, draft_parents ? &parents : nullptr, uniforms, temperature);
   if (st) return st;
   const Layout &L = m->L;
   const int32_t *ho = m->h_out();
@@ -1110,6 +1135,20 @@ ts_status verify_impl(ts_model *m, ts_session *const *ss, int32_t B, const int32
 ts_status ts_verify(ts_model *m, ts_session *const *ss, int32_t B, const int32_t *draft_tokens,
                     const int32_t *draft_offsets, uint32_t flags, ts_verify_result *out) {
   return verify_impl(m, ss, B, draft_tokens, nullptr, draft_offsets, flags, out, nullptr);
+}
+
+ts_status ts_verify_sampled(ts_model *m, ts_session *const *ss, int32_t B, const int32_t *draft_tokens,
+                            const int32_t *draft_offsets, float temperature, const float *uniforms, uint32_t flags,
+                            ts_verify_result *out) {
+  if (!uniforms) return fail(TS_ERR_ARG, "null uniforms");
+  if (!(temperature > 0.f) || !(temperature < 1e4f)) return fail(TS_ERR_ARG, "temperature must be in (0, 1e4)");
+  if (flags & TS_FLAG_SKIP_LM_HEAD) return fail(TS_ERR_ARG, "sampling acceptance needs the logits");
+  if (draft_offsets && B >= 1 && B <= 4096) {
+    const int M = draft_offsets[B] - draft_offsets[0] + B;
+    for (int r = 0; r < M; ++r)
+      if (!(uniforms[r] >= 0.f && uniforms[r] < 1.f)) return fail(TS_ERR_ARG, "uniform %d outside [0, 1)", r);
+  }
+  return verify_impl(m, ss, B, draft_tokens, nullptr, draft_offsets, flags, out, nullptr, uniforms, temperature);
 }
 
 ts_status ts_verify_tree(ts_model *m, ts_session *const *ss, int32_t B, const int32_t *draft_tokens,
