@@ -278,6 +278,34 @@ def run_reference(args, shape, lens, ks, name):
     }))
 
 
+def run_retrieval(args, shape):
+    """Top-K of Eq. 3 over N seeded N(0,1) hidden states (bf16), K = 10: one pass over N x d x 2 bytes."""
+    import torch
+    import paper_2604_13519_b200 as ts
+    tiny = ts.Model(shape if shape.n_layers <= 4 else __import__("synth").SHAPES[shape.name + "-2l"], max_pages=8, max_batch=1,
+                    k_max=8, max_rows=8, max_ctx=64, act_split=True, path=1)
+    d, N = shape.d_model, args.retrieval
+    g = torch.Generator(device="cuda").manual_seed(260413519)
+    H = torch.randn(N, d, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    q = torch.randn(d, generator=g, device="cuda", dtype=torch.float32)
+    for _ in range(max(args.warmup, 3)):
+        ts.ts_topk_cosine(tiny, H, 10, query=q)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        ts.ts_topk_cosine(tiny, H, 10, query=q)
+    torch.cuda.synchronize()
+    ms = 1e3 * (time.perf_counter() - t0) / args.steps
+    peaks = measured_peaks()
+    gbs = N * d * 2 / (ms * 1e-3) / 1e9
+    print(json.dumps({"metric": "topk_cosine_ms", "value": ms, "unit": "ms", "n_gpus": 1, "steps": args.steps,
+                      "warmup": max(args.warmup, 3), "higher_is_better": False, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": f"retrieval over {N} hidden states of width {d}, K = 10",
+                                 "timing": "host clock around the public call (launches, result copy, stream sync)"},
+                      "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -289,6 +317,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-act-split", action="store_true")
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 one kernel per stage, 2 single persistent kernel")
+    ap.add_argument("--retrieval", type=int, default=0,
+                    help="N > 0: time ts_topk_cosine (K = 10) over N synthetic hidden states of the workload's width "
+                         "instead of the verify step, and print its own JSON line")
     ap.add_argument("--temperature", type=float, default=0.0,
                     help="> 0: speculative-sampling acceptance at this temperature (ts_verify_sampled) with fixed uniforms")
     ap.add_argument("--tree", action="store_true",
@@ -310,6 +341,9 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the verify path has no CPU fallback")
     torch.cuda.set_device(local_rank)
+    if args.retrieval > 0:
+        run_retrieval(args, shape)
+        return
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))

@@ -265,6 +265,23 @@ ts_status ts_session_state(const ts_session *s, ts_session_info *out);
 /* Copy the generated output y (at most cap ids) to out (host); *n receives |y|. */
 ts_status ts_session_output(const ts_session *s, int32_t *out, int32_t cap, int32_t *n);
 
+/* ts_topk_cosine — Top-K of Eq. 3 (Section 4.3): the K datastore entries whose hidden state is most similar (cosine)
+ * to the query's; their indices, best first, are what ts_session_set_ranks takes as the candidate order of the
+ * suffix match (the paper uses K = 10).  hidden_dev: device, bf16 [n_entries][d_model] row-major, 16-byte aligned,
+ * owned by the caller (the paper stores the hidden representation of each historical question at its final token).
+ * query_dev: device fp32 [d_model], or NULL to use the final-norm hidden state of row `row` of the last step (row 0
+ * of a session's first step is its question's last token).  scores_dev: device scratch of
+ * TS_TOPK_SCRATCH_FLOATS(n_entries, K) floats, 8-byte aligned, owned by the caller, overwritten.  out_index / out_score: host, K entries (out_score may be NULL).  Ties go to the
+ * lower index; an entry or query of zero norm scores -2 (ranks last).  Synchronises the model's stream.
+ * Errors: TS_ERR_ARG (K outside [1, min(64, n_entries)], bad row), TS_ERR_STATE (no hidden state available). */
+#define TS_TOPK_SCRATCH_FLOATS(n, k) ((n) + 2 * (k) + 1 + 2 * (k) * (((n) + 4095) / 4096))
+ts_status ts_topk_cosine(ts_model *m, const void *hidden_dev, int32_t n_entries, const float *query_dev,
+                         int32_t row, int32_t K, float *scores_dev, int32_t *out_index, float *out_score);
+/* The final-norm hidden state (the LM head's input) of row `row` of the last step, as fp32 [d_model] on the host:
+ * what a caller stores per question to build the datastore's hidden states.  TS_ERR_STATE if the last step skipped
+ * the LM head or ran as the persistent kernel. */
+ts_status ts_last_hidden(ts_model *m, int32_t row, float *host_out);
+
 /* ---- test / benchmark support ------------------------------------------------------------------- */
 /* Overwrite the session's cache for one layer with n_tokens rows of host float32 K and V
  * ([n_tokens][n_kv_heads][head_dim]); values are rounded to the cache's storage type (fp16,

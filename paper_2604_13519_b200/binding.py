@@ -100,6 +100,8 @@ _SIGNATURES = {
                        _I32P],
     "ts_verify_sampled": [_P, C.POINTER(_P), C.c_int32, _I32P, _I32P, C.c_float, C.POINTER(C.c_float), C.c_uint32,
                           C.POINTER(ts_verify_result)],
+    "ts_topk_cosine": [_P, _P, C.c_int32, _P, C.c_int32, C.c_int32, _P, _I32P, C.POINTER(C.c_float)],
+    "ts_last_hidden": [_P, C.c_int32, C.POINTER(C.c_float)],
     "ts_verify_replay": [_P],
     "ts_profile_step": [_P, C.POINTER(C.c_float), _I32P, C.c_int32],
     "ts_commit": [_P, C.POINTER(ts_verify_result)],
@@ -418,6 +420,27 @@ def ts_verify_sampled(model: Model, sessions: Sequence[Session], drafts: Sequenc
     out = (ts_verify_result * B)()
     _check(lib().ts_verify_sampled(model.h, hs, B, _i32(flat), _i32(offs), temperature, u, flags, out))
     return list(out)
+
+
+def ts_topk_cosine(model: Model, hidden, K: int, query=None, row: int = 0):
+    """hidden: CUDA bf16 tensor [N][d]; query: CUDA float32 tensor [d] or None (hidden state of `row` of the last
+    step).  Returns (indices, scores), best first."""
+    torch = model.torch
+    N = hidden.shape[0]
+    assert hidden.is_cuda and hidden.dtype == torch.bfloat16 and hidden.is_contiguous()
+    scratch = torch.empty(N + 2 * K + 1 + 2 * K * ((N + 4095) // 4096), dtype=torch.float32, device=hidden.device)
+    idx = (C.c_int32 * K)()
+    sc = (C.c_float * K)()
+    q = _P(query.data_ptr()) if query is not None else None
+    _check(lib().ts_topk_cosine(model.h, _P(hidden.data_ptr()), N, q, row, K, _P(scratch.data_ptr()), idx, sc))
+    return list(idx), list(sc)
+
+
+def ts_last_hidden(model: Model, row: int):
+    import numpy as np
+    out = np.empty(model.cfg.d_model, dtype=np.float32)
+    _check(lib().ts_last_hidden(model.h, row, out.ctypes.data_as(C.POINTER(C.c_float))))
+    return out
 
 
 def ts_verify_replay(model: Model):

@@ -122,6 +122,11 @@ struct SampleArgs {
 };
 cudaError_t launch_sample_accept(const SampleArgs &a, cudaStream_t st);
 
+// Cosine Top-K over datastore hidden states (retrieval.cu).  scores: [N + 2K] floats; the result pairs (index as int
+// bits, score), best first, follow the N scores.  The query is q_dev (fp32 [d]) or, if null, bf16 planes of a row.
+cudaError_t launch_topk_cosine(const __nv_bfloat16 *H, int N, int d, const float *q_dev, const __nv_bfloat16 *q_planes,
+                               int plane_stride, int planes, int K, float *scores, cudaStream_t st);
+
 // After a tree step: move the K/V rows of the accepted path to consecutive cache positions len, len+1, ...
 struct CompactArgs {
   StepIn in;

@@ -1337,6 +1337,49 @@ ts_status ts_read_logits(ts_model *m, int32_t row0, int32_t n_rows, float *host_
   return TS_OK;
 }
 
+ts_status ts_last_hidden(ts_model *m, int32_t row, float *host_out) {
+  if (!m || !host_out) return fail(TS_ERR_ARG, "null argument");
+  if (!m->have_step || (m->last_flags & TS_FLAG_SKIP_LM_HEAD) || m->last_fused)
+    return fail(TS_ERR_STATE, "the last step left no final hidden state (it must run the LM head on the one-kernel-per-stage path)");
+  if (row < 0 || row >= m->last_M) return fail(TS_ERR_ARG, "row outside the last step");
+  const size_t d = m->c.d_model, R = m->L.rows_alloc;
+  std::vector<__nv_bfloat16> tmp(2 * d);
+  const __nv_bfloat16 *h = (const __nv_bfloat16 *)m->WS(m->L.h);
+  CU_TRY(cudaMemcpyAsync(tmp.data(), h + (size_t)row * d, d * 2, cudaMemcpyDeviceToHost, m->st));
+  if (m->planes == 2)
+    CU_TRY(cudaMemcpyAsync(tmp.data() + d, h + (R + (size_t)row) * d, d * 2, cudaMemcpyDeviceToHost, m->st));
+  CU_TRY(cudaStreamSynchronize(m->st));
+  for (size_t i = 0; i < d; ++i)
+    host_out[i] = __bfloat162float(tmp[i]) + (m->planes == 2 ? __bfloat162float(tmp[d + i]) : 0.f);
+  return TS_OK;
+}
+
+ts_status ts_topk_cosine(ts_model *m, const void *hidden_dev, int32_t n_entries, const float *query_dev, int32_t row,
+                         int32_t K, float *scores_dev, int32_t *out_index, float *out_score) {
+  if (!m || !hidden_dev || !scores_dev || !out_index) return fail(TS_ERR_ARG, "null argument");
+  if (n_entries < 1 || K < 1 || K > 64 || K > n_entries) return fail(TS_ERR_ARG, "K must be in [1, min(64, n_entries)]");
+  if (m->c.d_model % 8 || m->c.d_model > 16384) return fail(TS_ERR_ARG, "d_model must be a multiple of 8, at most 16384");
+  const __nv_bfloat16 *planes = nullptr;
+  if (!query_dev) {
+    if (!m->have_step || (m->last_flags & TS_FLAG_SKIP_LM_HEAD) || m->last_fused)
+      return fail(TS_ERR_STATE, "no final hidden state: pass a query, or run a step with the LM head on the one-kernel-per-stage path first");
+    if (row < 0 || row >= m->last_M) return fail(TS_ERR_ARG, "row outside the last step");
+    planes = (const __nv_bfloat16 *)m->WS(m->L.h) + (size_t)row * m->c.d_model;
+  }
+  CU_TRY(ts::launch_topk_cosine((const __nv_bfloat16 *)hidden_dev, n_entries, m->c.d_model, query_dev, planes,
+                                (int)(m->L.rows_alloc * m->c.d_model), m->planes, K, scores_dev, m->st));
+  std::vector<float> res(2 * (size_t)K);
+  CU_TRY(cudaMemcpyAsync(res.data(), scores_dev + n_entries, res.size() * 4, cudaMemcpyDeviceToHost, m->st));
+  CU_TRY(cudaStreamSynchronize(m->st));
+  for (int j = 0; j < K; ++j) {
+    int32_t idx;
+    std::memcpy(&idx, &res[2 * j], 4);
+    out_index[j] = idx;
+    if (out_score) out_score[j] = res[2 * j + 1];
+  }
+  return TS_OK;
+}
+
 ts_status ts_debug_read_buffer(ts_model *m, int32_t which, void *host_out, uint64_t bytes) {
   if (!m || !host_out) return fail(TS_ERR_ARG, "null argument");
   const Layout &L = m->L;
