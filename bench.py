@@ -320,6 +320,8 @@ def main():
     ap.add_argument("--retrieval", type=int, default=0,
                     help="N > 0: time ts_topk_cosine (K = 10) over N synthetic hidden states of the workload's width "
                          "instead of the verify step, and print its own JSON line")
+    ap.add_argument("--want-topk", action="store_true",
+                    help="also take the per-position Top-K of the logits (TS_FLAG_WANT_TOPK), as the recycling drafter needs")
     ap.add_argument("--temperature", type=float, default=0.0,
                     help="> 0: speculative-sampling acceptance at this temperature (ts_verify_sampled) with fixed uniforms")
     ap.add_argument("--tree", action="store_true",
@@ -357,12 +359,14 @@ def main():
 
     uniforms = [((37 * r + 11) % 100) / 100.0 for r in range(M)]
 
+    vflags = ts.TS_FLAG_WANT_TOPK if args.want_topk else 0
+
     def verify():
         if args.temperature > 0:
-            return ts.ts_verify_sampled(model, sessions, drafts, args.temperature, uniforms)
+            return ts.ts_verify_sampled(model, sessions, drafts, args.temperature, uniforms, flags=vflags)
         if parents is None:
-            return ts.ts_verify(model, sessions, drafts)
-        return ts.ts_verify_tree(model, sessions, drafts, parents)
+            return ts.ts_verify(model, sessions, drafts, flags=vflags)
+        return ts.ts_verify_tree(model, sessions, drafts, parents, flags=vflags)
 
     def barrier():
         if world > 1:
@@ -478,7 +482,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload, "batch": len(lens), "context": lens, "k": ks,
-                       "act_split": planes == 2, "draft_tree": bool(args.tree), "temperature": args.temperature, "kv_dtype": "f16", "l2": "inputs (weights) far larger than L2",
+                       "act_split": planes == 2, "draft_tree": bool(args.tree), "temperature": args.temperature, "per_position_topk": bool(args.want_topk), "kv_dtype": "f16", "l2": "inputs (weights) far larger than L2",
                        "parallelism": "replicas" if world > 1 else "single"},
             "latency_ms": {"p50": statistics.median(lat), "p90": sorted(lat)[int(0.9 * (len(lat) - 1))]},
             "clocks": clocks,

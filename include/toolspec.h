@@ -171,6 +171,8 @@ typedef struct {
 } ts_verify_result;
 
 #define TS_FLAG_SKIP_LM_HEAD 1u  /* no logits, no acceptance: rows only extend the KV cache */
+#define TS_FLAG_WANT_TOPK 2u     /* also take the TS_TOPK highest logits of every row (ts_last_topk; successor tables) */
+#define TS_TOPK 8
 
 /* ts_verify — Verification + SelectLongestAcceptedPrefix for B sequences in one batched forward.
  * Sequence i's chunk is [pending_i, draft_tokens[draft_offsets[i] .. draft_offsets[i+1])], k_i rows
@@ -195,6 +197,23 @@ ts_status ts_verify(ts_model *m, ts_session *const *sessions, int32_t B,
  * is ts_draft's chain.  Host only; never fails on "no draft". */
 ts_status ts_draft_tree(ts_session *s, int32_t max_nodes, int32_t *out_tokens, int32_t *out_parents,
                         int32_t *out_n, int32_t *out_source);
+
+/* General speculative drafting for the open-ended states q_v and q_o (Section 4.2 defers them to a general method and
+ * names Token Recycling; Appendix A.1: a pre-defined static tree there; the ablation of Section 5.3 falls back to a
+ * suffix match inside the input context).  Off by default.  When on, ts_draft_tree, after retrieval and the schema
+ * both yield nothing, (source 3) matches the last 7, 6, 5 ids of the context (prompt followed by the output) against
+ * an earlier occurrence in the context, earliest first, and drafts its continuation (at most n_cap ids); failing
+ * that, (source 4) builds the static tree over recycled successors: 17 slots in breadth-first order (four successors
+ * of the pending token; 3, 2, 1, 1 below them; then 2, 1, 1; then a chain of two), slot i carrying the rank-th entry
+ * of its parent's successor list.  A token's successor list is the TS_TOPK ids the model ranked highest right after
+ * it, refreshed by every ts_verify / ts_verify_tree call that carries TS_FLAG_WANT_TOPK, from all rows of the chunk. */
+ts_status ts_session_enable_general_sd(ts_session *s, int32_t on);
+/* Install / read one successor list (TS_TOPK ids, best first); *found = 0 if the token has none. */
+ts_status ts_session_set_successors(ts_session *s, int32_t token, const int32_t *ids);
+ts_status ts_session_successors(const ts_session *s, int32_t token, int32_t *ids, int32_t *found);
+/* The TS_TOPK highest logits of row `row` of the last step (run with TS_FLAG_WANT_TOPK): ids best first, lowest id on
+ * ties; values may be NULL. */
+ts_status ts_last_topk(ts_model *m, int32_t row, int32_t *ids, float *values);
 
 /* ts_verify_tree — PackDraftsAsTree's output verified in one forward pass under the tree-structured attention
  * mask (Appendix A.1 "Parallel Verification"; Algorithm 1: Verification, SelectLongestAcceptedPrefix).

@@ -32,6 +32,11 @@ SUFFIX_LENGTHS = (7, 6, 5)      # Appendix B.2: longest first, from 7 to 5
 DEFAULT_N_CAP = 32              # Appendix B.2: first continuation length
 LATER_CAPS = (16, 8, 8)         # Appendix B.2: lengths of the second to fourth continuation
 MAX_TOOL_CANDIDATES = 8         # tool names verified in parallel in q_t (a reading: the paper says "all")
+TOPK = 8                        # successors kept per token by the recycling drafter (a reading)
+# Static tree of the recycling drafter (Appendix A.1: "a pre-defined static tree"; the shape is a reading): slots in
+# breadth-first order, slot i + 1 = (parent slot, rank of the parent's successor it carries); slot 0 = pending token.
+RECYCLE_TREE = ((0, 0), (0, 1), (0, 2), (0, 3), (1, 0), (1, 1), (1, 2), (2, 0), (2, 1), (3, 0),
+                (4, 0), (5, 0), (5, 1), (6, 0), (8, 0), (12, 0), (16, 0))
 
 
 class SchemaFsm:
@@ -259,6 +264,41 @@ def suffix_matches(y: Sequence[int], store: Datastore, ranks: Optional[Sequence[
     return out
 
 
+def context_match(ctx: Sequence[int], n: int) -> List[int]:
+    """Suffix match inside the context itself (prompt followed by the output), the fallback the ablation of
+    Section 5.3 describes: L = 7, 6, 5 ids at the end of the context, the earliest earlier occurrence (the suffix
+    matching itself excluded), continuation of at most n ids."""
+    ctx = list(ctx)
+    if n <= 0:
+        return []
+    for L in SUFFIX_LENGTHS:
+        if len(ctx) <= L:
+            continue
+        s = ctx[-L:]
+        for m in range(L, len(ctx)):
+            if ctx[m - L:m] == s:
+                return ctx[m:m + n]
+    return []
+
+
+def recycled_tree(pending: int, table: dict, max_nodes: int):
+    """Static draft tree over recycled successors (Token Recycling as Section 2 describes it: the top-k
+    candidates of previous steps kept per token, a tree built breadth-first).  A slot whose parent is left out
+    or whose parent's token has no successor list is left out; nodes are numbered in creation order; nothing is
+    added once the chunk holds max_nodes nodes.  Returns (tokens of nodes 1.., parents of all nodes)."""
+    tokens: List[int] = []
+    parents: List[int] = [-1]
+    node_of, tok_of = {0: 0}, {0: pending}
+    for i, (ps, rank) in enumerate(RECYCLE_TREE, start=1):
+        if ps not in node_of or len(parents) >= max_nodes or tok_of[ps] not in table:
+            continue
+        t = table[tok_of[ps]][rank]
+        tokens.append(int(t))
+        parents.append(node_of[ps])
+        node_of[i], tok_of[i] = len(parents) - 1, int(t)
+    return tokens, parents
+
+
 def pack_candidates(candidates: Sequence[Sequence[int]], max_nodes: int):
     """PackDraftsAsTree (Algorithm 1): merge candidate chains (each a continuation of the pending
     token) into a token trie.  Nodes are numbered in creation order, candidates inserted in the
@@ -301,15 +341,24 @@ class Drafter:
     """Per-session drafter state: FSM, generated output y, candidate rank list."""
 
     def __init__(self, schema, store: Datastore, n_cap: int = DEFAULT_N_CAP,
-                 ranks: Optional[Sequence[int]] = None):
+                 ranks: Optional[Sequence[int]] = None, general_sd: bool = False):
         self.schema, self.store, self.n_cap = schema, store, n_cap
+        self.general_sd = general_sd        # drafts for q_v / q_o: context match, then recycled successors
+        self.prompt: List[int] = []
+        self.successors: dict = {}          # token -> the model's TOPK ids right after it, best first
         self.ranks = None if ranks is None else list(ranks)
         self.fsm = SchemaFsm(schema)
         self.y: List[int] = []
 
     def feed_prompt(self, tokens: Sequence[int]):
+        self.prompt = list(tokens)
         for t in tokens:
             self.fsm.step(t)
+
+    def update_successors(self, chunk: Sequence[int], topk_rows: Sequence[Sequence[int]]):
+        """After a verification: row j was fed chunk[j]; its TOPK highest logits become that token's list."""
+        for t, ids in zip(chunk, topk_rows):
+            self.successors[int(t)] = [int(i) for i in ids[:TOPK]]
 
     def guess_tool(self, prefix: Sequence[int]) -> int:
         comp = self.fsm.compatible_tools(prefix)
@@ -361,6 +410,14 @@ class Drafter:
     def draft_tree(self, max_nodes: int) -> Tuple[List[int], List[int], int]:
         """(tokens of nodes 1.., parents of all nodes, source): the candidates packed as a trie."""
         cands, src = self.draft_candidates(max_nodes - 1)
+        if not cands and self.general_sd and max_nodes > 1:
+            d = context_match(self.prompt + self.y, min(self.n_cap, max_nodes - 1))
+            if d:
+                cands, src = [d], 3
+            else:
+                pending = self.y[-1] if self.y else self.prompt[-1]
+                toks, par = recycled_tree(pending, self.successors, max_nodes)
+                return toks, par, (4 if toks else 0)
         toks, par = pack_candidates(cands, max_nodes)
         return toks, par, (src if toks else 0)
 

@@ -65,19 +65,26 @@ def speculative_decode(model: OracleModel, schema, store: Datastore, prompt: Seq
 def speculative_decode_tree(model: OracleModel, schema, store: Datastore, prompt: Sequence[int],
                             eos: int, max_new_tokens: int, max_nodes: int, n_cap: int = 32,
                             ranks: Optional[Sequence[int]] = None, cache=None, pending=None,
-                            max_steps: Optional[int] = None, trace: Optional[list] = None) -> List[int]:
+                            max_steps: Optional[int] = None, trace: Optional[list] = None,
+                            general_sd: bool = False) -> List[int]:
     """Algorithm 1 with its candidate set: draft candidates -> PackDraftsAsTree -> one verification
-    forward under the tree mask -> longest accepted path + bonus token -> append -> FSM update."""
+    forward under the tree mask -> longest accepted path + bonus token -> append -> FSM update.
+    With general_sd the open-ended states draft too (context match, recycled successors), and every
+    verification refreshes the successor lists from the per-row top-k of its logits."""
     from .tree import verify_tree
+    from .transformer import topk_lowest
+    from .drafter import TOPK
     if cache is None:
         cache, pending = prefill(model, prompt)
-    d = Drafter(schema, store, n_cap=n_cap, ranks=ranks)
+    d = Drafter(schema, store, n_cap=n_cap, ranks=ranks, general_sd=general_sd)
     d.feed_prompt(prompt)
     steps = 0
     while not d.finished(eos, max_new_tokens) and (max_steps is None or steps < max_steps):
         toks, par, source = d.draft_tree(max_nodes)
         n0 = cache.length
-        res = verify_tree(model, pending, toks, par, cache)
+        res = verify_tree(model, pending, toks, par, cache, want_logits=general_sd)
+        if general_sd:
+            d.update_successors([pending] + list(toks), [topk_lowest(row, TOPK) for row in res["logits"]])
         consumed, _fin = d.commit(res["emitted"], eos, max_new_tokens)
         cache.truncate(n0 + consumed)
         if trace is not None:

@@ -211,6 +211,12 @@ class OracleModel:
         return res
 
 
+def topk_lowest(logits_row: torch.Tensor, k: int) -> List[int]:
+    """The k ids with the highest logits, best first, lowest id on ties."""
+    v = logits_row.tolist()
+    return sorted(range(len(v)), key=lambda i: (-v[i], i))[:k]
+
+
 def top2_gap(logits_row: torch.Tensor) -> float:
     """Difference between the largest and second-largest logit of a row."""
     v = torch.topk(logits_row, 2).values

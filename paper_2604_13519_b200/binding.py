@@ -14,6 +14,8 @@ LIB_PATH = os.path.join(_HERE, "libtoolspec.so")
 TS_K_MAX = 64
 TS_PAGE_SIZE = 16
 TS_FLAG_SKIP_LM_HEAD = 1
+TS_FLAG_WANT_TOPK = 2
+TS_TOPK = 8
 
 STATUS = {0: "TS_OK", -1: "TS_ERR_ARG", -2: "TS_ERR_STATE", -3: "TS_ERR_OOM_PAGES",
           -4: "TS_ERR_K_TOO_LARGE", -5: "TS_ERR_TOKEN_RANGE", -6: "TS_ERR_DEVICE_TIMEOUT",
@@ -102,6 +104,10 @@ _SIGNATURES = {
                           C.POINTER(ts_verify_result)],
     "ts_topk_cosine": [_P, _P, C.c_int32, _P, C.c_int32, C.c_int32, _P, _I32P, C.POINTER(C.c_float)],
     "ts_last_hidden": [_P, C.c_int32, C.POINTER(C.c_float)],
+    "ts_session_enable_general_sd": [_P, C.c_int32],
+    "ts_session_set_successors": [_P, C.c_int32, _I32P],
+    "ts_session_successors": [_P, C.c_int32, _I32P, _I32P],
+    "ts_last_topk": [_P, C.c_int32, _I32P, C.POINTER(C.c_float)],
     "ts_verify_replay": [_P],
     "ts_profile_step": [_P, C.POINTER(C.c_float), _I32P, C.c_int32],
     "ts_commit": [_P, C.POINTER(ts_verify_result)],
@@ -308,6 +314,19 @@ class Session:
         _check(lib().ts_session_create(model.h if model else None, schema.h if schema else None,
                                        store.h if store else None, C.byref(cfg), C.byref(self.h)))
 
+    def enable_general_sd(self, on: bool = True):
+        _check(lib().ts_session_enable_general_sd(self.h, 1 if on else 0))
+
+    def set_successors(self, token: int, ids: Sequence[int]):
+        assert len(ids) == TS_TOPK
+        _check(lib().ts_session_set_successors(self.h, token, _i32(ids)))
+
+    def successors(self, token: int):
+        ids = (C.c_int32 * TS_TOPK)()
+        found = C.c_int32(0)
+        _check(lib().ts_session_successors(self.h, token, ids, C.byref(found)))
+        return list(ids) if found.value else None
+
     def set_ranks(self, ranks: Sequence[int]):
         _check(lib().ts_session_set_ranks(self.h, _i32(ranks), len(ranks)))
 
@@ -441,6 +460,13 @@ def ts_last_hidden(model: Model, row: int):
     out = np.empty(model.cfg.d_model, dtype=np.float32)
     _check(lib().ts_last_hidden(model.h, row, out.ctypes.data_as(C.POINTER(C.c_float))))
     return out
+
+
+def ts_last_topk(model: Model, row: int):
+    ids = (C.c_int32 * TS_TOPK)()
+    vals = (C.c_float * TS_TOPK)()
+    _check(lib().ts_last_topk(model.h, row, ids, vals))
+    return list(ids), list(vals)
 
 
 def ts_verify_replay(model: Model):

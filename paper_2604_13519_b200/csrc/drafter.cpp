@@ -288,4 +288,43 @@ void pack_candidates(const std::vector<std::vector<int32_t>> &cands, int32_t max
   }
 }
 
+void context_match(const std::vector<int32_t> &ctx, int32_t n, std::vector<int32_t> *out) {
+  out->clear();
+  const int32_t len = (int32_t)ctx.size();
+  if (n <= 0) return;
+  for (int32_t L = 7; L >= 5; --L) {
+    if (len <= L) continue;
+    const int32_t *tail = ctx.data() + len - L;
+    for (int32_t m = L; m < len; ++m) {   // m = len would be the suffix matching itself
+      if (std::memcmp(ctx.data() + m - L, tail, sizeof(int32_t) * L) == 0) {
+        out->assign(ctx.begin() + m, ctx.begin() + std::min(len, m + n));
+        return;
+      }
+    }
+  }
+}
+
+// breadth-first: four successors of the pending token; 3, 2, 1, 1 below them; then 2, 1, 1; then a chain of two
+const RecycleSlot kRecycleTree[17] = {{0, 0}, {0, 1}, {0, 2}, {0, 3}, {1, 0}, {1, 1}, {1, 2}, {2, 0}, {2, 1}, {3, 0},
+                                      {4, 0}, {5, 0}, {5, 1}, {6, 0}, {8, 0}, {12, 0}, {16, 0}};
+
+void recycled_tree(int32_t pending, const std::unordered_map<int32_t, std::array<int32_t, TS_TOPK>> &table,
+                   int32_t max_nodes, std::vector<int32_t> *tokens, std::vector<int32_t> *parents) {
+  tokens->clear();
+  parents->clear();
+  int32_t node_of[18], tok_of[18];   // per slot: node number (-1 = left out) and token
+  node_of[0] = 0; tok_of[0] = pending;
+  for (int i = 1; i <= 17; ++i) {
+    node_of[i] = -1; tok_of[i] = -1;
+    const RecycleSlot sl = kRecycleTree[i - 1];
+    if (node_of[sl.parent] < 0 || (int32_t)tokens->size() + 1 >= max_nodes) continue;
+    auto it = table.find(tok_of[sl.parent]);
+    if (it == table.end()) continue;
+    tok_of[i] = it->second[sl.rank];
+    tokens->push_back(tok_of[i]);
+    parents->push_back(node_of[sl.parent]);
+    node_of[i] = (int32_t)tokens->size();
+  }
+}
+
 }  // namespace ts

@@ -4,6 +4,8 @@
 #pragma once
 #include <cstdint>
 #include <string>
+#include <array>
+#include <unordered_map>
 #include <vector>
 
 #include "toolspec.h"
@@ -83,5 +85,19 @@ void suffix_matches(const std::vector<int32_t> &y, const ts_datastore &d, const 
 // node j + 1 at index j.
 void pack_candidates(const std::vector<std::vector<int32_t>> &cands, int32_t max_nodes, std::vector<int32_t> *tokens,
                      std::vector<int32_t> *parents);
+
+// Suffix match inside the context itself (prompt followed by the generated output), as the paper's ablation without
+// schema and retrieval falls back to: L = 7, 6, 5 ids at the end of the context, the earliest earlier occurrence,
+// continuation of at most n ids.
+void context_match(const std::vector<int32_t> &ctx, int32_t n, std::vector<int32_t> *out);
+
+// Static draft tree over recycled successors: node slots in breadth-first order, slot i hangs from slot
+// kRecycleTree[i].parent and carries the rank-th successor of that slot's token (slot 0 = the pending token).  A
+// slot whose parent is missing or whose parent's token has no table entry is left out; nodes are numbered in
+// creation order; nothing is added once the chunk holds max_nodes nodes.
+struct RecycleSlot { int8_t parent, rank; };
+extern const RecycleSlot kRecycleTree[17];
+void recycled_tree(int32_t pending, const std::unordered_map<int32_t, std::array<int32_t, TS_TOPK>> &table,
+                   int32_t max_nodes, std::vector<int32_t> *tokens, std::vector<int32_t> *parents);
 
 }  // namespace ts

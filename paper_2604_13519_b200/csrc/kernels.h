@@ -127,6 +127,10 @@ cudaError_t launch_sample_accept(const SampleArgs &a, cudaStream_t st);
 cudaError_t launch_topk_cosine(const __nv_bfloat16 *H, int N, int d, const float *q_dev, const __nv_bfloat16 *q_planes,
                                int plane_stride, int planes, int K, float *scores, cudaStream_t st);
 
+// Row-wise Top-K (topk.cu): out[r][j] = (column as int bits, value) of the j-th largest entry of row r, lowest column
+// on ties.  cand: scratch of n_rows * ceil(n_cols / 4096) * K pairs.
+cudaError_t launch_topk_rows(const float *x, int n_rows, int n_cols, int K, float2 *cand, float *out, cudaStream_t st);
+
 // After a tree step: move the K/V rows of the accepted path to consecutive cache positions len, len+1, ...
 struct CompactArgs {
   StepIn in;

@@ -6,6 +6,8 @@
 #include <cstdio>
 #include <cstring>
 #include <string>
+#include <array>
+#include <unordered_map>
 #include <vector>
 
 #include "drafter.h"
@@ -58,8 +60,8 @@ struct Layout {
   int n_maps, n_counters, n_phases, max_tiles128, o_tile128_seq, o_tile128_row0;
   // step io (int32 offsets inside d_in / h_in)
   int o_tokens, o_pos, o_rowseq, o_cu, o_len, o_tile_seq, o_tile_row0, o_btab, in_ints;
-  int o_parent, o_anc, o_path, o_uni;
-  uint64_t samp_stats;
+  int o_parent, o_anc, o_path, o_uni, o_topk;
+  uint64_t samp_stats, topk_cand;
   // step out (int32 offsets)
   int o_argmax, o_accept, o_emitted, o_newlen, o_newpend, o_err, out_ints;
   int rows_alloc, pages_per_seq, max_tiles, Nqkv, n_vocab_tiles;
@@ -128,6 +130,7 @@ void make_layout(const ts_model_config &c, Layout *L) {
   L->logits = take(R * V * 4);
   L->amax = take(R * 8);
   L->samp_stats = take(R * 16 * 4);
+  L->topk_cand = take(R * (uint64_t)((c.vocab + 4095) / 4096) * TS_TOPK * 8);
   L->rope = take((uint64_t)c.max_ctx * (hd / 2) * 8);
   int io = 0;
   auto itake = [&](int n) { int r = io; io += (n + 3) / 4 * 4; return r; };
@@ -143,6 +146,7 @@ void make_layout(const ts_model_config &c, Layout *L) {
   L->o_argmax = itake(c.max_rows); L->o_accept = itake(c.max_batch); L->o_emitted = itake(c.max_batch * c.k_max);
   L->o_newlen = itake(c.max_batch); L->o_newpend = itake(c.max_batch); L->o_err = itake(4);
   L->o_path = itake(c.max_batch * c.k_max);
+  L->o_topk = itake(c.max_rows * TS_TOPK * 2);   // (id bits, value) pairs, written by the Top-K kernel
   L->out_ints = io;
   L->d_in = take((uint64_t)L->in_ints * 4);
   L->d_out = take((uint64_t)L->out_ints * 4);
@@ -233,6 +237,9 @@ struct ts_session {
   ts_draft_config cfg{};
   ts::Fsm fsm;
   std::vector<int32_t> y, ranks, pages, last_chunk;
+  std::vector<int32_t> prompt;                                         // kept for the context suffix match
+  bool general_sd = false;                                             // drafts for q_v / q_o: context match, then recycled successors
+  std::unordered_map<int32_t, std::array<int32_t, TS_TOPK>> successors;  // token -> the model's last Top-K after it
   bool have_ranks = false;
   int32_t cache_len = -1, pending = -1;
   bool finished = false;
@@ -501,6 +508,12 @@ ts_status run_step(ts_model *m) {
                          amax, nullptr);
   if (s) return s;
   int32_t *dout = m->d_out();
+  if (m->last_flags & TS_FLAG_WANT_TOPK) {   // per-position Top-K of the logits, for the successor tables
+    CU_TRY(ts::launch_topk_rows((const float *)m->WS(L.logits), M, c.vocab, TS_TOPK, (float2 *)m->WS(L.topk_cand),
+                                (float *)(dout + L.o_topk), m->st));
+    m->launched(5);
+    m->launched(5);
+  }
   if (m->last_sample) {
     ts::SampleArgs sa{};
     sa.in = in; sa.logits = (const float *)m->WS(L.logits); sa.amax = amax;
@@ -624,7 +637,10 @@ ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::ve
     m->last_inv_t = 1.f / temperature;
     std::memcpy(hi + L.o_uni, uniforms, sizeof(float) * M);
   }
-  m->last_fused = !m->last_tree && !m->last_sample && can_fuse && (c.path == 2 || (c.path == 0 && kAutoPrefersFused));
+  if ((flags & TS_FLAG_WANT_TOPK) && c.path == 2)
+    return fail(TS_ERR_UNIMPLEMENTED, "the per-position Top-K needs the one-kernel-per-stage path");
+  m->last_fused = !m->last_tree && !m->last_sample && !(flags & TS_FLAG_WANT_TOPK) && can_fuse &&
+                  (c.path == 2 || (c.path == 0 && kAutoPrefersFused));
   m->last_B = B; m->last_M = M; m->last_tiles = tiles; m->last_tiles128 = tiles128; m->last_flags = flags;
   m->have_step = true;
   const size_t in_bytes = (size_t)(L.o_btab + (size_t)B * L.pages_per_seq) * 4;
@@ -964,6 +980,40 @@ ts_status ts_session_set_ranks(ts_session *s, const int32_t *ranks, int32_t n) {
   return TS_OK;
 }
 
+ts_status ts_session_enable_general_sd(ts_session *s, int32_t on) {
+  if (!s) return fail(TS_ERR_ARG, "null argument");
+  s->general_sd = on != 0;
+  return TS_OK;
+}
+
+ts_status ts_session_set_successors(ts_session *s, int32_t token, const int32_t *ids) {
+  if (!s || !ids || token < 0) return fail(TS_ERR_ARG, "bad argument");
+  std::array<int32_t, TS_TOPK> a;
+  for (int t = 0; t < TS_TOPK; ++t) a[t] = ids[t];
+  s->successors[token] = a;
+  return TS_OK;
+}
+
+ts_status ts_session_successors(const ts_session *s, int32_t token, int32_t *ids, int32_t *found) {
+  if (!s || !ids || !found) return fail(TS_ERR_ARG, "null argument");
+  auto it = s->successors.find(token);
+  *found = it != s->successors.end();
+  if (*found) for (int t = 0; t < TS_TOPK; ++t) ids[t] = it->second[t];
+  return TS_OK;
+}
+
+ts_status ts_last_topk(ts_model *m, int32_t row, int32_t *ids, float *values) {
+  if (!m || !ids) return fail(TS_ERR_ARG, "null argument");
+  if (!m->have_step || !(m->last_flags & TS_FLAG_WANT_TOPK)) return fail(TS_ERR_STATE, "the last step was not asked for the Top-K");
+  if (row < 0 || row >= m->last_M) return fail(TS_ERR_ARG, "row outside the last step");
+  const int32_t *ho = m->h_out() + m->L.o_topk + (size_t)row * TS_TOPK * 2;
+  for (int t = 0; t < TS_TOPK; ++t) {
+    ids[t] = ho[2 * t];
+    if (values) std::memcpy(&values[t], &ho[2 * t + 1], 4);
+  }
+  return TS_OK;
+}
+
 ts_status ts_session_destroy(ts_session *s) {
   if (!s) return TS_OK;
   if (s->m) {
@@ -981,6 +1031,7 @@ ts_status ts_prefill(ts_model *m, ts_session *s, const int32_t *tokens, int32_t 
   if (s->cache_len >= 0) return fail(TS_ERR_STATE, "session already has a context");
   if (s->schema)
     for (int i = 0; i < n; ++i) s->fsm.step(tokens[i]);
+  s->prompt.assign(tokens, tokens + n);
   s->cache_len = 0;
   if (m) {
     std::vector<std::vector<int32_t>> rows(1);
@@ -1063,7 +1114,21 @@ ts_status ts_draft_tree(ts_session *s, int32_t max_nodes, int32_t *out_tokens, i
     if (!cands.empty()) source = 1;
   }
   std::vector<int32_t> toks, par;
-  ts::pack_candidates(cands, max_nodes, &toks, &par);
+  if (cands.empty() && s->general_sd) {
+    // open-ended states: a suffix match inside the context itself, else the static tree over recycled successors
+    std::vector<int32_t> ctx(s->prompt);
+    ctx.insert(ctx.end(), s->y.begin(), s->y.end());
+    std::vector<int32_t> d;
+    ts::context_match(ctx, std::min(s->cfg.n_cap, max_draft), &d);
+    if (!d.empty()) {
+      cands.push_back(d);
+      source = 3;
+    } else {
+      ts::recycled_tree(s->pending, s->successors, max_nodes, &toks, &par);
+      if (!toks.empty()) source = 4;
+    }
+  }
+  if (source != 4) ts::pack_candidates(cands, max_nodes, &toks, &par);
   std::memcpy(out_tokens, toks.data(), toks.size() * sizeof(int32_t));
   std::memcpy(out_parents, par.data(), par.size() * sizeof(int32_t));
   *out_n = (int32_t)toks.size();
@@ -1117,6 +1182,14 @@ ts_status verify_impl(ts_model *m, ts_session *const *ss, int32_t B, const int32
       if (path_out) {
         for (int j = 0; j < TS_K_MAX; ++j)
           path_out[i * TS_K_MAX + j] = j <= r.accept_len ? ho[L.o_path + i * m->c.k_max + j] : -1;
+      }
+      if ((flags & TS_FLAG_WANT_TOPK) && ss[i]->general_sd) {
+        // successor table: what the model ranked highest after each token it was fed in this step (all rows)
+        for (int j = 0; j < r.k; ++j) {
+          std::array<int32_t, TS_TOPK> ids;
+          for (int t = 0; t < TS_TOPK; ++t) ids[t] = ho[L.o_topk + ((row + j) * TS_TOPK + t) * 2];
+          ss[i]->successors[rows[i][j]] = ids;
+        }
       }
       if (draft_parents) {
         // the cache now holds the accepted path's rows at consecutive positions: record what sits there, so that

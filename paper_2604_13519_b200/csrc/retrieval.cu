@@ -4,7 +4,7 @@
 //
 // cosine_scores_kernel: one warp per datastore entry, 16-byte loads of its bf16 row, fp32 dot product and squared
 // norm, the query in shared memory: one pass over N x d x 2 bytes, bound by HBM.
-// topk_slice_kernel / topk_final_kernel: K best per 4096-score slice in shared memory, then the K best of those.
+// The K best scores are then taken by the row Top-K kernels (topk.cu).
 #include "kernels.h"
 
 namespace ts {
@@ -52,76 +52,6 @@ cosine_scores_kernel(const __nv_bfloat16 *H, int N, int d, const float *q_dev, c
   }
 }
 
-// Selection in two levels, both with the same rule (largest score, lowest index on ties): every CTA of the first
-// kernel holds a slice of kSlice scores in shared memory and takes its K best in K rounds; the second kernel (one
-// CTA) takes the K best of the slices' candidates.  cand: [slices][K] (index, score) pairs; out: [K] pairs.
-static constexpr int kSlice = 4096;
-static constexpr int kSelThreads = 256;
-
-__device__ __forceinline__ void block_argmax(float &v, int &idx, float *bv, int *bi) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float ov = __shfl_xor_sync(0xffffffffu, v, o);
-    const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
-    if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
-  }
-  __syncthreads();
-  if (lane == 0) { bv[warp] = v; bi[warp] = idx; }
-  __syncthreads();
-  v = bv[0]; idx = bi[0];
-  for (int w = 1; w < kSelThreads / 32; ++w)
-    if (bv[w] > v || (bv[w] == v && bi[w] < idx)) { v = bv[w]; idx = bi[w]; }
-}
-
-__global__ void __launch_bounds__(kSelThreads)
-topk_slice_kernel(const float *scores, int N, int K, float2 *cand) {
-  __shared__ float s[kSlice];
-  __shared__ float bv[kSelThreads / 32];
-  __shared__ int bi[kSelThreads / 32];
-  const int base = blockIdx.x * kSlice;
-  for (int i = threadIdx.x; i < kSlice; i += blockDim.x) s[i] = base + i < N ? scores[base + i] : -INFINITY;
-  __syncthreads();
-  for (int j = 0; j < K; ++j) {
-    float v = -INFINITY;
-    int idx = 0x7FFFFFFF;
-    for (int i = threadIdx.x; i < kSlice; i += blockDim.x)
-      if (s[i] > v) { v = s[i]; idx = base + i; }        // ascending i: the first of equal scores stays
-    block_argmax(v, idx, bv, bi);
-    if (threadIdx.x == 0) {
-      cand[(size_t)blockIdx.x * K + j] = make_float2(__int_as_float(idx), v);
-      if (idx != 0x7FFFFFFF) s[idx - base] = -INFINITY;  // struck out (a slice with fewer than K entries yields -inf pairs)
-    }
-    __syncthreads();
-  }
-}
-
-__global__ void __launch_bounds__(kSelThreads)
-topk_final_kernel(float2 *cand, int n_cand, int K, float *out) {
-  __shared__ float bv[kSelThreads / 32];
-  __shared__ int bi[kSelThreads / 32];
-  __shared__ int taken_slot;
-  for (int j = 0; j < K; ++j) {
-    float v = -INFINITY;
-    int idx = 0x7FFFFFFF, slot = -1;
-    for (int i = threadIdx.x; i < n_cand; i += blockDim.x) {
-      const float2 c = cand[i];
-      const int ci = __float_as_int(c.x);
-      if (c.y > v || (c.y == v && ci < idx)) { v = c.y; idx = ci; slot = i; }
-    }
-    const int my_idx = idx;
-    block_argmax(v, idx, bv, bi);
-    if (my_idx == idx && slot >= 0) taken_slot = slot;   // indices are unique among live candidates
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      out[2 * j] = __int_as_float(idx);
-      out[2 * j + 1] = v;
-      if (idx != 0x7FFFFFFF) cand[taken_slot] = make_float2(__int_as_float(0x7FFFFFFF), -INFINITY);
-    }
-    __syncthreads();
-  }
-}
-
 cudaError_t launch_topk_cosine(const __nv_bfloat16 *H, int N, int d, const float *q_dev, const __nv_bfloat16 *q_planes,
                                int plane_stride, int planes, int K, float *scores, cudaStream_t st) {
   static bool attr_done = false;
@@ -136,13 +66,8 @@ cudaError_t launch_topk_cosine(const __nv_bfloat16 *H, int N, int d, const float
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   // candidates live behind the K result pairs: scores[N + 2K ...], 2 floats per candidate
-  const int slices = (N + kSlice - 1) / kSlice;
   float2 *cand = reinterpret_cast<float2 *>(scores + N + 2 * K + ((N + 2 * K) & 1));
-  topk_slice_kernel<<<slices, kSelThreads, 0, st>>>(scores, N, K, cand);
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-  topk_final_kernel<<<1, kSelThreads, 0, st>>>(cand, slices * K, K, scores + N);
-  return cudaGetLastError();
+  return launch_topk_rows(scores, 1, N, K, cand, scores + N, st);
 }
 
 }  // namespace ts

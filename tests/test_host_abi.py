@@ -192,3 +192,40 @@ def test_fused_schedule_partition(T, KB, n):
     for tile, lst in per_tile.items():
         assert [c for c, _, _ in lst] == list(range(lst[0][1], lst[0][1] + lst[0][2]))
         assert all(cf == lst[0][1] and ns == lst[0][2] for _, cf, ns in lst)
+
+
+def test_general_sd_drafts_bit_exact_with_oracle():
+    """Context match and recycled-successor trees (host only): the same table and context on both sides."""
+    schema = synth.make_schema(4096, 8, seed=4)
+    rnd = random.Random(31)
+    sc = ts.Schema(schema.vocab, schema.tools)
+    seen = set()
+    for trial in range(60):
+        d = oracle.Drafter(schema, oracle.Datastore(len(schema.tools)), general_sd=True)
+        s = ts.Session(None, sc, None)
+        s.enable_general_sd()
+        alphabet = rnd.choice([3, 50, 4000])
+        prompt = [64 + rnd.randrange(alphabet) for _ in range(rnd.randint(1, 30))]     # no tool call: q_o
+        d.feed_prompt(prompt)
+        ts.ts_prefill(None, s, prompt)
+        for step in range(12):
+            # the same successor lists on both sides, for some of the tokens around
+            for _ in range(rnd.randint(0, 6)):
+                t = 64 + rnd.randrange(alphabet)
+                ids = rnd.sample(range(64, 64 + max(alphabet, 16)), oracle.TOPK)
+                d.successors[t] = ids
+                s.set_successors(t, ids)
+                assert s.successors(t) == ids
+            mn = rnd.choice([1, 2, 7, 18, 64])
+            wt, wp, wsrc = d.draft_tree(mn)
+            gt, gp, gsrc = ts.ts_draft_tree(s, mn)
+            assert (gt, gp, gsrc) == (wt, wp[1:], wsrc), (trial, step, mn)
+            seen.add(wsrc)
+            span = [64 + rnd.randrange(alphabet) for _ in range(rnd.randint(1, 4))]
+            d.commit(span, schema.vocab.eos, 10 ** 6)
+            ts.ts_commit_forced(s, span)
+    assert {0, 3, 4} <= seen
+    # off by default: the same session state drafts nothing in q_o
+    s2 = ts.Session(None, sc, None)
+    ts.ts_prefill(None, s2, [70, 71, 72, 73, 74, 75, 70, 71, 72, 73, 74, 75])
+    assert ts.ts_draft_tree(s2, 16) == ([], [], 0)

@@ -333,3 +333,85 @@ def test_tree_loop_equals_vanilla_greedy_on_a_tiny_model():
     assert out == ref
     assert len(trace) < len(ref)                                     # drafts were accepted
     assert any(len(set(t["parents"])) < len(t["parents"]) for t in trace)       # and some trees did branch
+
+
+# ---- general speculative drafting for q_v / q_o: context match and recycled successors ----------------------
+def test_context_match_equals_brute_force():
+    rnd = random.Random(21)
+    hits = 0
+    for _ in range(300):
+        alphabet = rnd.choice([2, 3, 6])
+        ctx = [rnd.randrange(alphabet) for _ in range(rnd.randint(0, 40))]
+        n = rnd.choice([1, 5, 32])
+        best = None
+        for L in (5, 6, 7):
+            if len(ctx) <= L:
+                continue
+            for m in range(L, len(ctx)):
+                if ctx[m - L:m] == ctx[-L:]:
+                    key = (-L, m)
+                    if best is None or key < best:
+                        best = key
+        want = [] if best is None else ctx[best[1]:best[1] + n]
+        assert oracle.context_match(ctx, n) == want
+        hits += bool(want)
+    assert hits > 30
+    assert oracle.context_match([1, 2, 3, 4, 5], 4) == []            # the suffix matching itself does not count
+
+
+def test_recycled_tree_shape_and_lookup():
+    class Every(dict):                                # a list for every token: 10 t + rank + 1
+        def __contains__(self, t):
+            return True
+
+        def __getitem__(self, t):
+            return [10 * t + r + 1 for r in range(oracle.TOPK)]
+    table = Every()
+    toks, par = oracle.recycled_tree(1, table, 64)
+    assert len(toks) == 17 and par[0] == -1
+    # every node carries the successor of its parent's token at the template's rank, parents come first
+    z = [1] + toks
+    kids = {}
+    for j in range(1, len(z)):
+        assert 0 <= par[j] < j
+        r = kids.setdefault(par[j], 0)
+        assert z[j] == table[z[par[j]]][r]           # children of a node appear in rank order 0, 1, 2, ...
+        kids[par[j]] = r + 1
+    assert kids[0] == 4 and sorted(kids.values(), reverse=True)[:4] == [4, 3, 2, 2]
+    depth = oracle.node_depths(par)
+    assert max(depth) == 5 and depth.count(1) == 4 and depth.count(2) == 7
+    # the budget cuts in slot order; a token without a list prunes its subtree
+    assert oracle.recycled_tree(1, table, 6)[1] == [-1, 0, 0, 0, 0, 1]
+    class AllBut(Every):                              # the first child has no list: its whole subtree goes
+        def __contains__(self, t):
+            return t != table[1][0]
+    toks2, par2 = oracle.recycled_tree(1, AllBut(), 64)
+    assert len(toks2) == 17 - 8                       # slots 5, 6, 7, 12, 13, 14, 16, 17 hang below slot 1
+    assert all(p != 1 for p in par2[1:])
+    assert oracle.recycled_tree(7, {}, 64) == ([], [-1])
+
+
+def test_topk_lowest_against_torch_and_ties():
+    import torch
+    g = torch.Generator().manual_seed(4)
+    x = torch.randn(500, generator=g, dtype=torch.float64)
+    assert oracle.topk_lowest(x, 8) == torch.topk(x, 8).indices.tolist()
+    assert oracle.topk_lowest(torch.tensor([1.0, 3.0, 3.0, 0.0, 3.0]), 4) == [1, 2, 4, 0]
+
+
+def test_general_sd_loop_is_lossless_and_uses_both_sources():
+    from test_oracle_pins import _small_shape, _rand_weights
+    shape = _small_shape(vocab=4096)
+    om = oracle.OracleModel(shape, _rand_weights(shape, seed=12))
+    schema = _schema(seed=5, n_tools=8)
+    v = schema.vocab
+    st = oracle.Datastore(len(schema.tools))          # empty: nothing to retrieve, q_o throughout
+    prompt = synth.make_context(4096, 30, seed=5)[:-1] + [77]        # no tool call: the FSM stays in q_o
+    ref = oracle.vanilla_greedy(om, schema, prompt, v.eos, 48)
+    trace = []
+    out = oracle.speculative_decode_tree(om, schema, st, prompt, v.eos, 48, max_nodes=20, trace=trace,
+                                         general_sd=True)
+    assert out == ref
+    srcs = {t["source"] for t in trace}
+    assert 4 in srcs                                   # recycled trees were drafted once lists existed
+    assert trace[0]["source"] == 0                     # nothing to draft from at the very first step
