@@ -41,6 +41,34 @@ def _model(shape, seqs, path):
                     max_ctx=max(lens) + 2 * k_max, act_split=True, path=path)
 
 
+def _extras_at_full_vocabulary(gm, sess, draft, logits):
+    """The per-position Top-K and the sampling acceptance on the full 151 936-id vocabulary (37 whole 4096-id slices
+    and a ragged one), against the oracle's logits of the same chunk."""
+    k = len(draft) + 1
+    ts.ts_verify(gm, [sess], [draft], flags=ts.TS_FLAG_WANT_TOPK)
+    exact = 0
+    for j in range(k):
+        ids, vals = ts.ts_last_topk(gm, j)
+        want = oracle.topk_lowest(logits[j], ts.TS_TOPK)
+        assert len(set(ids)) == ts.TS_TOPK
+        for r, i in enumerate(ids):
+            assert float(logits[j][i]) >= float(logits[j][want[r]]) - 0.05, f"row {j} rank {r}"
+        exact += ids == want
+    assert exact >= k // 2        # with 151 936 ids the 8 best lie close together: swaps inside the margin are common
+    # sampling acceptance: at a temperature where the greedy token is a coin flip, same uniforms on both sides
+    T = 1.0
+    while T > 1e-3 and float(oracle.target_probs(logits[0], T).max()) < 0.5:
+        T /= 2
+    g = np.random.Generator(np.random.Philox(key=[260413519, 0x8B37]))
+    agree = 0
+    for _ in range(12):
+        u = [min(float(x), 0.99999994) for x in g.random(k).astype(np.float32)]
+        want = oracle.accept_sampled(logits, draft, T, u)
+        r = ts.ts_verify_sampled(gm, [sess], [draft], T, u)[0]
+        agree += (r.accept_len, list(r.emitted[:r.n_emitted])) == want
+    assert agree >= 10
+
+
 def test_8b_full_depth():
     shape = synth.SHAPES["8b"]
     assert shape.n_layers == 36
@@ -98,4 +126,6 @@ def test_8b_full_depth():
             mx, mean = check_step(r, got, refs[i], where=where)
             print(f"{where}: logits max-abs {mx:.3e}, mean-abs {mean:.3e}")
             row0 += k
+        if gm.cfg.path == 1:
+            _extras_at_full_vocabulary(gm, ss[0], drafts[idx[0]], refs[idx[0]]["logits"])
         gm.close()
