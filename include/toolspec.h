@@ -312,6 +312,9 @@ ts_status ts_debug_import_kv(ts_model *m, ts_session *s, int32_t layer, const fl
 ts_status ts_debug_export_kv(ts_model *m, ts_session *s, int32_t layer, float *k, float *v,
                              int32_t n_tokens);
 ts_status ts_debug_set_cache(ts_session *s, int32_t cache_len, int32_t pending);
+/* ts_debug_set_cache, and the session forgets what it generated: output, FSM state (back to q_o), successor lists,
+ * the finished mark.  For replaying a context with another decoding strategy (benchmark traces). */
+ts_status ts_debug_restart(ts_session *s, int32_t cache_len, int32_t pending);
 /* Copy rows [row0, row0+n_rows) of the last step's float32 logits [rows][vocab] to host memory. */
 ts_status ts_read_logits(ts_model *m, int32_t row0, int32_t n_rows, float *host_out);
 /* Copy the first `bytes` bytes of an internal activation buffer of the last step to host memory:

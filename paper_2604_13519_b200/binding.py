@@ -108,6 +108,7 @@ _SIGNATURES = {
     "ts_session_set_successors": [_P, C.c_int32, _I32P],
     "ts_session_successors": [_P, C.c_int32, _I32P, _I32P],
     "ts_last_topk": [_P, C.c_int32, _I32P, C.POINTER(C.c_float)],
+    "ts_debug_restart": [_P, C.c_int32, C.c_int32],
     "ts_verify_replay": [_P],
     "ts_profile_step": [_P, C.POINTER(C.c_float), _I32P, C.c_int32],
     "ts_commit": [_P, C.POINTER(ts_verify_result)],
@@ -344,6 +345,9 @@ class Session:
 
     def set_cache(self, cache_len: int, pending: int):
         _check(lib().ts_debug_set_cache(self.h, cache_len, pending))
+
+    def restart(self, cache_len: int, pending: int):
+        _check(lib().ts_debug_restart(self.h, cache_len, pending))
 
     def import_kv(self, layer: int, k, v):
         """k, v: CPU tensors [n_tokens][n_kv_heads][head_dim] (any float dtype; sent as float32)."""

@@ -1399,6 +1399,17 @@ ts_status ts_debug_set_cache(ts_session *s, int32_t cache_len, int32_t pending) 
   return TS_OK;
 }
 
+ts_status ts_debug_restart(ts_session *s, int32_t cache_len, int32_t pending) {
+  ts_status st = ts_debug_set_cache(s, cache_len, pending);
+  if (st) return st;
+  s->y.clear();
+  s->last_chunk.clear();
+  s->successors.clear();
+  s->finished = false;
+  s->fsm.reset();
+  return TS_OK;
+}
+
 ts_status ts_read_logits(ts_model *m, int32_t row0, int32_t n_rows, float *host_out) {
   if (!m || !host_out) return fail(TS_ERR_ARG, "null argument");
   if (!m->have_step || (m->last_flags & TS_FLAG_SKIP_LM_HEAD)) return fail(TS_ERR_STATE, "last step produced no logits");
