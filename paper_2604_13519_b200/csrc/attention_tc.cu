@@ -196,11 +196,20 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
     if (lane == 0) mbar_arrive(smem_u32(&ctl->s_empty[buf]));
     // a block every row sees whole needs no mask (all but the last blocks of a sequence's last split)
     if (p_base + kAttnBlk - 1 > lim_all) {
+      // bit e of `vis`: position p_base + e is visible to this row (cache positions all, chunk rows by the mask,
+      // nothing at or past the split's end)
+      const int rel0 = p_base - t.len;                 // chunk row of the block's first position (negative: cache)
+      unsigned long long vis;
+      if (rel0 >= 0) vis = rel0 < 64 ? anc >> rel0 : 0ull;
+      else if (rel0 > -64) vis = (anc << (-rel0)) | ((1ull << (-rel0)) - 1ull);
+      else vis = ~0ull;
+      const int n_in = t.pos_end - p_base;             // positions of the block inside the split
+      if (n_in < 64) vis &= n_in > 0 ? (1ull << n_in) - 1ull : 0ull;
+      const uint32_t vlo = (uint32_t)vis, vhi = (uint32_t)(vis >> 32);
 #pragma unroll
-      for (int e = 0; e < 64; ++e) {
-        const int p = p_base + e, rel = p - t.len;   // rel < 64: the chunk has at most 64 rows and p < pos_end below
-        const bool vis = p < t.pos_end && (rel < 0 || ((anc >> (rel & 63)) & 1ull) != 0ull);
-        sc[e] = vis ? sc[e] : -INFINITY;
+      for (int e = 0; e < 32; ++e) {
+        sc[e] = (vlo >> e) & 1u ? sc[e] : -INFINITY;
+        sc[32 + e] = (vhi >> e) & 1u ? sc[32 + e] : -INFINITY;
       }
     }
     float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;

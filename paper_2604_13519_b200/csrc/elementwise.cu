@@ -139,10 +139,8 @@ __global__ void rope_kv_kernel(StepIn in, const float *part, int n_splits, int p
     q[i] = to_half_sat(a);
     q[i + half] = to_half_sat(b);
   } else {
-    // cache slot = cached length + the row's index in its chunk (equal to its position in a chain; in a draft
-    // tree the position is the depth, and siblings still need slots of their own)
     const int seq = in.row_seq[m];
-    const int slot = in.seq_len[seq] + (m - in.cu_rows[seq]);
+    const int slot = in.slot[m];
     const int page = in.block_tab[(size_t)seq * in.pages_per_seq + (slot >> 4)];
     const bool is_k = head < Hq + Hkv;
     const int kh = is_k ? head - Hq : head - Hq - Hkv;

@@ -35,7 +35,9 @@ cudaError_t launch_gemm(int epi, const CUtensorMap &tw, const CUtensorMap &ta, G
 // Per-step inputs resident in device memory (all int32).
 struct StepIn {
   const int32_t *tokens;     // [M] chunk ids, rows of sequence i at cu_rows[i]..cu_rows[i+1]
-  const int32_t *pos;        // [M] absolute position of each row
+  const int32_t *pos;        // [M] absolute (rotary) position of each row
+  const int32_t *slot;       // [M] cache slot the row's K/V go to: cached length + the row's index in its chunk (equal
+                             // to pos in a chain; in a draft tree pos is the depth and siblings need slots of their own)
   const int32_t *row_seq;    // [M] sequence index of each row
   const int32_t *cu_rows;    // [B+1]
   const int32_t *seq_len;    // [B] tokens already in the cache

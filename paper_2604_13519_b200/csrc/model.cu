@@ -60,7 +60,7 @@ struct Layout {
   int n_maps, n_counters, n_phases, max_tiles128, o_tile128_seq, o_tile128_row0;
   // step io (int32 offsets inside d_in / h_in)
   int o_tokens, o_pos, o_rowseq, o_cu, o_len, o_tile_seq, o_tile_row0, o_btab, in_ints;
-  int o_parent, o_anc, o_path, o_uni, o_topk;
+  int o_parent, o_anc, o_path, o_uni, o_topk, o_slot;
   uint64_t samp_stats, topk_cand;
   // step out (int32 offsets)
   int o_argmax, o_accept, o_emitted, o_newlen, o_newpend, o_err, out_ints;
@@ -140,6 +140,7 @@ void make_layout(const ts_model_config &c, Layout *L) {
   L->max_tiles128 = c.max_batch * ((c.k_max * G + 127) / 128);
   L->o_tile128_seq = itake(L->max_tiles128); L->o_tile128_row0 = itake(L->max_tiles128);
   L->o_parent = itake(c.max_rows); L->o_anc = itake(2 * c.max_rows); L->o_uni = itake(c.max_rows);
+  L->o_slot = itake(c.max_rows);
   L->o_btab = itake(c.max_batch * L->pages_per_seq);   // (last: only the used part is copied per step)
   L->in_ints = io;
   io = 0;
@@ -378,7 +379,7 @@ ts_status run_step_fused(ts_model *m) {
   a.V = c.vocab; a.Hq = c.n_q_heads; a.Hkv = c.n_kv_heads; a.hd = c.head_dim; a.eps = c.rms_eps;
   a.in.tokens = di + L.o_tokens; a.in.pos = di + L.o_pos; a.in.row_seq = di + L.o_rowseq; a.in.cu_rows = di + L.o_cu;
   a.in.seq_len = di + L.o_len; a.in.block_tab = di + L.o_btab; a.in.pages_per_seq = L.pages_per_seq;
-  a.in.parent = di + L.o_parent; a.in.anc = (const uint32_t *)(di + L.o_anc);
+  a.in.parent = di + L.o_parent; a.in.anc = (const uint32_t *)(di + L.o_anc); a.in.slot = di + L.o_slot;
   a.in.B = m->last_B; a.in.M = m->last_M;
   a.mc_index = pick_mc_index(m->last_M); a.Mc = kMcOptions[a.mc_index]; a.planes = m->planes;
   a.n_ctas = m->n_sms; a.skip_lm = (m->last_flags & TS_FLAG_SKIP_LM_HEAD) ? 1 : 0;
@@ -426,7 +427,7 @@ ts_status run_step(ts_model *m) {
   int32_t *di = m->d_in();
   in.tokens = di + L.o_tokens; in.pos = di + L.o_pos; in.row_seq = di + L.o_rowseq; in.cu_rows = di + L.o_cu;
   in.seq_len = di + L.o_len; in.block_tab = di + L.o_btab; in.pages_per_seq = L.pages_per_seq;
-  in.parent = di + L.o_parent; in.anc = (const uint32_t *)(di + L.o_anc);
+  in.parent = di + L.o_parent; in.anc = (const uint32_t *)(di + L.o_anc); in.slot = di + L.o_slot;
   in.B = B; in.M = M;
   float *x = (float *)m->WS(L.x);
   __nv_bfloat16 *h = (__nv_bfloat16 *)m->WS(L.h);
@@ -592,6 +593,7 @@ ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::ve
       hi[L.o_tokens + M + j] = rows[i][j];
       hi[L.o_pos + M + j] = s->cache_len + (parents ? depth[j] : j);
       hi[L.o_rowseq + M + j] = i;
+      hi[L.o_slot + M + j] = s->cache_len + j;
       hi[L.o_parent + M + j] = par;
       hi[L.o_anc + 2 * (M + j)] = (int32_t)(uint32_t)(mask & 0xFFFFFFFFull);
       hi[L.o_anc + 2 * (M + j) + 1] = (int32_t)(uint32_t)(mask >> 32);

@@ -82,9 +82,12 @@ TS_HD void split_pages(int n_pages, int n_splits, int split, int *p0, int *p1) {
 
 
 // The same cut in whole 64-position blocks (4 pages), so that only a sequence's last split ends in a partial block.
+// Cut points are rounded up, so a remainder goes to the first splits: the last one, which alone waits for the chunk's
+// own K/V rows and masks its last block, never gets the extra block.
 TS_HD void split_blocks(int n_pages, int n_splits, int split, int *p0, int *p1) {
   const int nb = (n_pages + 3) >> 2;
-  const int b0 = (int)(((int64_t)split * nb) / n_splits), b1 = (int)(((int64_t)(split + 1) * nb) / n_splits);
+  const int b0 = (int)(((int64_t)split * nb + n_splits - 1) / n_splits);
+  const int b1 = (int)(((int64_t)(split + 1) * nb + n_splits - 1) / n_splits);
   *p0 = b0 << 2;
   *p1 = (b1 << 2) < n_pages ? (b1 << 2) : n_pages;
 }
