@@ -150,6 +150,27 @@ def test_ragged_batch():
     gm.close()
 
 
+def test_sixteen_sessions_512_rows():
+    """The largest step of the batched configuration: 16 sessions x k = 32 = 512 rows (four 128-row chunks in every
+    projection, 16 attention row tiles), ragged contexts from a few tokens to two thousand."""
+    shape = synth.SHAPES["8b-2l"]
+    g = np.random.Generator(np.random.Philox(key=[260413519, 0x512]))
+    lens = [int(x) for x in g.integers(3, 2048, size=16)]
+    lens[3], lens[11] = 2047, 16
+    om, gm = make_pair(shape, max_batch=16, k_max=32, max_rows=512, max_ctx=2048 + 64)
+    sess, drafts, refs = [], [], []
+    for i, n in enumerate(lens):
+        cache, s, pending = synthetic_context(shape, om, gm, n, stream=i, pending=200 + i)
+        draft = _rand_draft(shape.vocab, 31, 40 + i)
+        sess.append(s); drafts.append(draft)
+        refs.append(om.verify(pending, draft, cache, want_logits=True))
+    out = ts.ts_verify(gm, sess, drafts)
+    for i, (res, ref) in enumerate(zip(out, refs)):
+        assert res.first_row == 32 * i and res.k == 32
+        check_step(res, gm.read_logits(32 * i, 32), ref, f"seq {i} (ctx {lens[i]})")
+    gm.close()
+
+
 def test_retrieval_heavy_batch():
     """Config-5-like: batch 4, long retrieved drafts (k = 64) from a large store searched through
     the n-gram index; drafts bit-exact with the oracle's linear scan."""
