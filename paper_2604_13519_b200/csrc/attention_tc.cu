@@ -5,8 +5,9 @@
 //   warp 1   tensor memory allocation + tcgen05.mma issue:  S = Q K^T  (Q tile and K block K-major in shared
 //            memory, 128 x 64 fp32 result in tensor memory), then  O_blk = P V  with P read from tensor memory
 //            (fp16) and the V block read MN-major from the same [position][64 elements] image K uses
-//   warps 2..5  one row per thread: running max over the block's 64 scores, P = exp2(S - max) written back to
-//            tensor memory as fp16, O_blk added into registers with the running-softmax rescale
+//   warps 2..5  one row per thread: maximum over the block's 64 scores, P = exp2(S - reference maximum) written back
+//            to tensor memory as fp16.  The output sums stay in tensor memory (every P V adds to them); the
+//            reference maximum follows the running one in steps, and only then is the row of sums multiplied down
 // Each split writes an un-normalised partial output with its (max, sum); attn_combine_kernel merges the splits.
 // Every wait is bounded; on expiry the CTA records an error word and leaves through the normal exit.
 #include <cuda_fp16.h>
@@ -25,7 +26,7 @@ static constexpr int kWorkerWarp0 = 2;
 
 struct __align__(16) AttnCtl {
   uint64_t kv_full[kKvStages], kv_empty[kKvStages], q_full;
-  uint64_t s_full[2], s_empty[2], p_full[2], o_full[2], o_empty[2];
+  uint64_t s_full[2], s_empty[2], p_full[2], pv_done;
   uint32_t tmem_base;
 };
 
@@ -88,7 +89,8 @@ __device__ __forceinline__ AttnUnit attn_unit_info(const AttnTcArgs &a, int u) {
 // tensor-memory columns of the attention phase (they lie over the projection accumulators, which are idle then)
 static constexpr int kColS = 0;      // two score buffers of 64 columns
 static constexpr int kColP = 128;    // two probability buffers of 32 columns (fp16 pairs)
-static constexpr int kColO = 192;    // two output-block buffers of head_dim columns
+static constexpr int kColO = 192;    // the output sums: head_dim columns, accumulated over the unit's blocks
+static constexpr float kRescaleStep = 8.f;   // the reference maximum follows the running one in steps of 2^8
 
 __device__ __forceinline__ void cp_async16z(uint32_t dst, const void *src, bool valid) {
   const int sz = valid ? 16 : 0;
@@ -109,7 +111,7 @@ __device__ __forceinline__ uint32_t pack_h2(float x, float y) {
 }
 
 // Worker side of one unit.  Thread <-> row (tensor-memory lane q*32 + lane): it takes the row maximum over the
-// block's 64 scores, writes the 64 probabilities back as fp16 and keeps the head_dim output sums in registers.
+// block's 64 scores, writes the 64 probabilities back as fp16 and, rarely, rescales the row's output sums.
 // `blk` counts K/V blocks over all units of this CTA (buffer index and barrier parity come from it).
 template <int HD>
 __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *ctl, const AttnUnit &t, uint8_t *sQ, uint32_t tmem_base,
@@ -145,32 +147,13 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
   const int lim_all = min(t.len, t.pos_end) - 1;   // every row sees every position up to here
   const unsigned long long anc = ((unsigned long long)a.in.anc[2 * (t.r_beg + j) + 1] << 32) | a.in.anc[2 * (t.r_beg + j)];
   const float scale = rsqrtf((float)HD) * 1.4426950408889634f;
-  float acc[HD];
-#pragma unroll
-  for (int i = 0; i < HD; ++i) acc[i] = 0.f;
-  float m_run = -INFINITY, l_run = 0.f, f_pending = 0.f;
+  // The output sums stay in tensor memory: every product P V adds to them.  Probabilities are taken against a
+  // reference maximum m_ref that follows the running maximum lazily: only when a block's maximum exceeds it by
+  // more than kRescaleStep (in the log2 domain) is the row of sums multiplied down and m_ref raised, so in most
+  // blocks the softmax thread never touches the sums.  Until then probabilities may reach 2^kRescaleStep: well
+  // inside fp16, and the sums are fp32.
+  float m_ref = -INFINITY, l_run = 0.f;
   bool ok = true;
-
-  auto consume_o = [&](uint32_t bi, float f) {   // acc = acc * f + O_blk
-    const uint32_t buf = bi & 1;
-    if (ok && !mbar_wait_err(smem_u32(&ctl->o_full[buf]), (bi >> 1) & 1, err)) { ok = false; atomicCAS((int *)err, 0, DEV_TIMEOUT_TMEM); }
-    tc_fence_after();
-#pragma unroll
-    for (int i = 0; i < HD / 32; ++i) {
-      uint32_t r0[16], r1[16];
-      tmem_ld16(tq + kColO + buf * HD + i * 32, r0);
-      tmem_ld16(tq + kColO + buf * HD + i * 32 + 16, r1);
-      tmem_wait_ld();
-#pragma unroll
-      for (int e = 0; e < 16; ++e) {
-        acc[i * 32 + e] = acc[i * 32 + e] * f + __uint_as_float(r0[e]);
-        acc[i * 32 + 16 + e] = acc[i * 32 + 16 + e] * f + __uint_as_float(r1[e]);
-      }
-    }
-    tc_fence_before();
-    __syncwarp();
-    if (lane == 0) mbar_arrive(smem_u32(&ctl->o_empty[buf]));
-  };
 
   for (int b = 0; b < t.nblk; ++b, ++blk) {
     const uint32_t buf = blk & 1;
@@ -217,43 +200,80 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
     for (int e = 0; e < 64; e += 4) {
       mx0 = fmaxf(mx0, sc[e]); mx1 = fmaxf(mx1, sc[e + 1]); mx2 = fmaxf(mx2, sc[e + 2]); mx3 = fmaxf(mx3, sc[e + 3]);
     }
-    // running maximum in the log2 domain: scores times log2(e)/sqrt(head_dim), folded into one multiply-add per score
-    const float m_new = fmaxf(m_run, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale);
-    const float ref = (m_new == -INFINITY) ? 0.f : m_new;
-    const float f = ex2_approx(m_run - ref);   // exp2(-inf) = 0 on the first block
-    m_run = m_new;
+    // block maximum in the log2 domain: scores times log2(e)/sqrt(head_dim), folded into one multiply-add per score
+    const float m_blk = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale;
+    const bool raise = m_blk > m_ref + kRescaleStep;   // (also the first finite maximum: m_ref starts at -inf)
+    const float m_old = m_ref;
+    if (raise) m_ref = m_blk;
+    const float ref = (m_ref == -INFINITY) ? 0.f : m_ref;
     float sum0 = 0.f, sum1 = 0.f;
-    // the P buffer is free: the product that read it two blocks ago was seen complete when its O_blk was taken
+    uint32_t pk0[16], pk1[16];
 #pragma unroll
-    for (int g = 0; g < 2; ++g) {
-      uint32_t pk[16];
-#pragma unroll
-      for (int e = 0; e < 16; ++e) {
-        const float e0 = ex2_approx(fmaf(sc[g * 32 + 2 * e], scale, -ref));
-        const float e1 = ex2_approx(fmaf(sc[g * 32 + 2 * e + 1], scale, -ref));
-        sum0 += e0; sum1 += e1;
-        pk[e] = pack_h2(e0, e1);
-      }
-      tmem_st16(tq + kColP + buf * 32 + g * 16, pk);
+    for (int e = 0; e < 16; ++e) {
+      const float e0 = ex2_approx(fmaf(sc[2 * e], scale, -ref));
+      const float e1 = ex2_approx(fmaf(sc[2 * e + 1], scale, -ref));
+      const float e2 = ex2_approx(fmaf(sc[32 + 2 * e], scale, -ref));
+      const float e3 = ex2_approx(fmaf(sc[32 + 2 * e + 1], scale, -ref));
+      sum0 += e0 + e2; sum1 += e1 + e3;
+      pk0[e] = pack_h2(e0, e1);
+      pk1[e] = pack_h2(e2, e3);
     }
-    const float sum = sum0 + sum1;
-    l_run = l_run * f + sum;
+    // the previous product has to be complete before its P buffer's twin is reused and before the sums are touched
+    if (b > 0) {
+      if (ok && !mbar_wait_err(smem_u32(&ctl->pv_done), (uint32_t)(b - 1) & 1u, err)) { ok = false; atomicCAS((int *)err, 0, DEV_TIMEOUT_TMEM); }
+      tc_fence_after();
+    }
+    float f = 1.f;
+    if (b > 0 && __any_sync(0xffffffffu, raise)) {       // tensor-memory accesses are warp-wide: lanes that stay use f = 1
+      if (raise) f = ex2_approx(m_old - ref);            // exp2(-inf) = 0: nothing was summed before the first finite maximum
+#pragma unroll
+      for (int i = 0; i < HD / 32; ++i) {
+        uint32_t r0[16], r1[16];
+        tmem_ld16(tq + kColO + i * 32, r0);
+        tmem_ld16(tq + kColO + i * 32 + 16, r1);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          r0[e] = __float_as_uint(__uint_as_float(r0[e]) * f);
+          r1[e] = __float_as_uint(__uint_as_float(r1[e]) * f);
+        }
+        tmem_st16(tq + kColO + i * 32, r0);
+        tmem_st16(tq + kColO + i * 32 + 16, r1);
+      }
+    }
+    l_run = l_run * f + (sum0 + sum1);
+    tmem_st16(tq + kColP + buf * 32, pk0);
+    tmem_st16(tq + kColP + buf * 32 + 16, pk1);
     tmem_wait_st();
     tc_fence_before();
     __syncwarp();
     if (lane == 0) mbar_arrive(smem_u32(&ctl->p_full[buf]));
-    if (b > 0) consume_o(blk - 1, f_pending);
-    f_pending = f;   // (no CTA-wide barrier per block: a failed wait has set the error word, which ends every other wait)
+    // (no CTA-wide barrier per block: a failed wait has set the error word, which ends every other wait)
   }
-  consume_o(blk - 1, f_pending);
+  if (ok && !mbar_wait_err(smem_u32(&ctl->pv_done), (uint32_t)(t.nblk - 1) & 1u, err)) { ok = false; atomicCAS((int *)err, 0, DEV_TIMEOUT_TMEM); }
+  tc_fence_after();
   if (!worker_all(ok)) return false;
 
-  // ---- partial result of this split: un-normalised output, running max (log2 domain), sum -----------------
-  if (valid) {
-    a.attn_ml[ob] = make_float2(m_run, l_run);
+  // ---- partial result of this split: un-normalised output, its reference maximum (log2 domain), sum -------
+  {
     float4 *dst = reinterpret_cast<float4 *>(a.attn_o + ob * HD);
+    if (valid) a.attn_ml[ob] = make_float2(m_ref, l_run);
 #pragma unroll
-    for (int i = 0; i < HD / 4; ++i) dst[i] = make_float4(acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3]);
+    for (int i = 0; i < HD / 32; ++i) {
+      uint32_t r0[16], r1[16];
+      tmem_ld16(tq + kColO + i * 32, r0);      // (warp-wide: rows past the tile's end read too, and write nothing)
+      tmem_ld16(tq + kColO + i * 32 + 16, r1);
+      tmem_wait_ld();
+      if (valid) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          dst[i * 8 + e] = make_float4(__uint_as_float(r0[4 * e]), __uint_as_float(r0[4 * e + 1]),
+                                       __uint_as_float(r0[4 * e + 2]), __uint_as_float(r0[4 * e + 3]));
+          dst[i * 8 + 4 + e] = make_float4(__uint_as_float(r1[4 * e]), __uint_as_float(r1[4 * e + 1]),
+                                           __uint_as_float(r1[4 * e + 2]), __uint_as_float(r1[4 * e + 3]));
+        }
+      }
+    }
   }
   return true;
 }
@@ -276,10 +296,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
       mbar_init(smem_u32(&ctl->s_full[b]), 1);
       mbar_init(smem_u32(&ctl->s_empty[b]), 4);
       mbar_init(smem_u32(&ctl->p_full[b]), 4);
-      mbar_init(smem_u32(&ctl->o_full[b]), 1);
-      mbar_init(smem_u32(&ctl->o_empty[b]), 4);
     }
     mbar_init(smem_u32(&ctl->q_full), 1);
+    mbar_init(smem_u32(&ctl->pv_done), 1);
     fence_barrier_init();
   }
   if (warp == 1) {
@@ -332,17 +351,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
       const uint32_t idesc_pv = umma_idesc_f16(kAttnRows, HD, 1);
       const uint32_t sQ = smem_u32(smem);
       bool ok = true;
-      auto issue_pv = [&](uint32_t bi) -> bool {   // O_blk = P V for block bi
+      auto issue_pv = [&](uint32_t bi) -> bool {   // O += P V for block bi
         const uint32_t pb = bi & 1, vst = bi % kKvStages;
         if (!mbar_wait_err(smem_u32(&ctl->p_full[pb]), (bi >> 1) & 1, err)) return false;
-        if (!mbar_wait_err(smem_u32(&ctl->o_empty[pb]), ((bi >> 1) & 1) ^ 1, err)) return false;
         tc_fence_after();
         const uint32_t sV = sQ + kQBytes + vst * kKvBytes + kAttnBlk * HD * 2;
 #pragma unroll
         for (int ks = 0; ks < kAttnBlk / 16; ++ks)   // 16 positions per instruction
-          umma_f16_ts(tmem_base + kColO + pb * HD, tmem_base + kColP + pb * 32 + ks * 8,
-                      umma_desc_sw128_mn(sV + ks * 2048, kAttnBlk * 128), idesc_pv, ks > 0 ? 1u : 0u);
-        umma_commit(smem_u32(&ctl->o_full[pb]));
+          umma_f16_ts(tmem_base + kColO, tmem_base + kColP + pb * 32 + ks * 8,
+                      umma_desc_sw128_mn(sV + ks * 2048, kAttnBlk * 128), idesc_pv, (bi | ks) != 0 ? 1u : 0u);
+        umma_commit(smem_u32(&ctl->pv_done));
         umma_commit(smem_u32(&ctl->kv_empty[vst]));
         return true;
       };
