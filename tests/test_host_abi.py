@@ -229,3 +229,15 @@ def test_general_sd_drafts_bit_exact_with_oracle():
     s2 = ts.Session(None, sc, None)
     ts.ts_prefill(None, s2, [70, 71, 72, 73, 74, 75, 70, 71, 72, 73, 74, 75])
     assert ts.ts_draft_tree(s2, 16) == ([], [], 0)
+
+
+def test_bench_tree_shapes_are_valid_trees():
+    """The draft-tree shapes bench.py --tree feeds to ts_verify_tree: parents precede their children, four branches."""
+    import bench
+    for k in range(1, 65):
+        par = bench.tree_parents(k)
+        assert len(par) == k - 1
+        for j, p in enumerate(par):
+            assert 0 <= p <= j                         # node j + 1 hangs from an earlier node
+        assert par.count(0) == min(4, sum(1 for n in (k - 1 - (k - 1) // 2, (k - 1) // 2 - (k - 1) // 4,
+                                                      (k - 1) // 4 - (k - 1) // 8, (k - 1) // 8) if n > 0))
