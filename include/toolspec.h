@@ -250,6 +250,18 @@ ts_status ts_verify_sampled(ts_model *m, ts_session *const *sessions, int32_t B,
                             const int32_t *draft_tokens, const int32_t *draft_offsets, float temperature,
                             const float *uniforms, uint32_t flags, ts_verify_result *out);
 
+/* ts_verify_tree_sampled — the paper's full verification: a draft tree (ts_verify_tree) accepted by speculative
+ * sampling (ts_verify_sampled).  At a node the children are tried in node order against the residual: child c with
+ * token x is accepted with probability r(x) / R, r being the node's p = softmax(logits / T) with the tokens of the
+ * children already refused removed and R its total; if none is accepted (or the node is a leaf) one sample of the
+ * residual is emitted and the step ends.  uniforms: one value in [0, 1) per chunk node, chunk after chunk: value c of
+ * a chunk decides its node c (c >= 1), value 0 draws the sample.  Arguments, result, path and compaction as
+ * ts_verify_tree; errors as ts_verify_tree and ts_verify_sampled. */
+ts_status ts_verify_tree_sampled(ts_model *m, ts_session *const *sessions, int32_t B,
+                                 const int32_t *draft_tokens, const int32_t *draft_parents,
+                                 const int32_t *draft_offsets, float temperature, const float *uniforms,
+                                 uint32_t flags, ts_verify_result *out, int32_t *path_out);
+
 /* Enqueue again the device work of the last ts_verify call on its inputs, which are still resident
  * in device memory; no host<->device copy, no synchronisation.  The step is idempotent because
  * sessions advance only in ts_commit.  For timing the kernels alone. */

@@ -11,5 +11,6 @@ from .drafter import (SchemaFsm, Datastore, Drafter, suffix_match, suffix_matche
 from .loop import prefill, vanilla_greedy, speculative_decode, speculative_decode_tree  # noqa: F401
 from .tree import (verify_tree, forward_tree, accepted_path, ancestor_mask, node_depths,  # noqa: F401
                    pack_candidates)
-from .sampling import target_probs, sample_inverse_cdf, accept_sampled, verify_sampled   # noqa: F401
+from .sampling import (target_probs, sample_inverse_cdf, accept_sampled, verify_sampled,   # noqa: F401
+                       accept_sampled_tree)
 from .retrieval import cosine_scores, topk_cosine   # noqa: F401

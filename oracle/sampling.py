@@ -64,3 +64,34 @@ def verify_sampled(model: OracleModel, pending: int, draft: Sequence[int], cache
     if want_logits:
         res["logits"] = logits
     return res
+
+
+def accept_sampled_tree(logits: torch.Tensor, z: Sequence[int], parents: Sequence[int], temperature: float,
+                        u: Sequence[float]):
+    """Speculative sampling over a draft tree (Appendix A.1's tree + Appendix B.2's acceptance rule).  z: tokens of
+    all k nodes (z[0] = pending), parents[0] = -1.  At node v with target p = softmax(logits_v / T) the children are
+    tried in node order against the residual: child c (token x) is accepted with probability r(x) / R, where r is
+    p with the tokens of the children already refused removed and R its total; u[c] decides child c.  If a child
+    is accepted the walk moves there; if none is (or v is a leaf) one sample of the residual is emitted with u[0]
+    and the step ends.  Each emitted token is then distributed as the model's own, whatever the tree holds.
+    Returns (path of node indices, emitted ids)."""
+    k = len(z)
+    assert logits.shape[0] == k and len(parents) == k and len(u) == k
+    path, emitted, v = [0], [], 0
+    while True:
+        r = target_probs(logits[v], temperature).clone()
+        nxt = None
+        for c in range(v + 1, k):
+            if parents[c] != v:
+                continue
+            x = z[c]
+            if u[c] * float(r.sum()) < float(r[x]):
+                nxt = c
+                break
+            r[x] = 0.0
+        if nxt is None:
+            emitted.append(sample_inverse_cdf(r, u[0]))
+            return path, emitted
+        path.append(nxt)
+        emitted.append(z[nxt])
+        v = nxt

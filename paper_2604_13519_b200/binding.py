@@ -109,6 +109,8 @@ _SIGNATURES = {
     "ts_session_successors": [_P, C.c_int32, _I32P, _I32P],
     "ts_last_topk": [_P, C.c_int32, _I32P, C.POINTER(C.c_float)],
     "ts_debug_restart": [_P, C.c_int32, C.c_int32],
+    "ts_verify_tree_sampled": [_P, C.POINTER(_P), C.c_int32, _I32P, _I32P, _I32P, C.c_float, C.POINTER(C.c_float),
+                               C.c_uint32, C.POINTER(ts_verify_result), _I32P],
     "ts_verify_replay": [_P],
     "ts_profile_step": [_P, C.POINTER(C.c_float), _I32P, C.c_int32],
     "ts_commit": [_P, C.POINTER(ts_verify_result)],
@@ -471,6 +473,27 @@ def ts_last_topk(model: Model, row: int):
     vals = (C.c_float * TS_TOPK)()
     _check(lib().ts_last_topk(model.h, row, ids, vals))
     return list(ids), list(vals)
+
+
+def ts_verify_tree_sampled(model: Model, sessions: Sequence[Session], drafts: Sequence[Sequence[int]],
+                           parents: Sequence[Sequence[int]], temperature: float, uniforms: Sequence[float],
+                           flags: int = 0):
+    """Draft trees accepted by speculative sampling; uniforms: one value per chunk node (value 0 of a chunk draws
+    the sample).  Returns (results, accepted paths)."""
+    B = len(sessions)
+    hs = (_P * B)(*[s.h for s in sessions])
+    flat, par, offs = [], [], [0]
+    for d, p in zip(drafts, parents):
+        flat += list(d)
+        par += list(p)
+        offs.append(len(flat))
+    assert len(uniforms) == len(flat) + B
+    u = (C.c_float * len(uniforms))(*uniforms)
+    out = (ts_verify_result * B)()
+    path = (C.c_int32 * (B * TS_K_MAX))()
+    _check(lib().ts_verify_tree_sampled(model.h, hs, B, _i32(flat), _i32(par), _i32(offs), temperature, u, flags, out,
+                                        path))
+    return list(out), [[path[i * TS_K_MAX + j] for j in range(out[i].accept_len + 1)] for i in range(B)]
 
 
 def ts_verify_replay(model: Model):

@@ -113,9 +113,9 @@ cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t st);
 // Speculative-sampling acceptance (sampling.cu): per-row softmax statistics, accept tests, the step's one sample.
 struct SampleArgs {
   StepIn in;
-  const float *logits;              // [M][V]
+  float *logits;                    // [M][V] (refused tokens are masked for the draw and restored)
   const unsigned long long *amax;   // [M] packed per-row maxima (argmax is still reported)
-  const float *uni;                 // [M] uniforms in [0, 1): row j of a chunk decides draft j + 1, the last row's draws the sample
+  const float *uni;                 // [M] uniforms in [0, 1): row c of a chunk decides node c, the root row's draws the sample
   float *part;                      // [M][16] scratch: per-slice sums of exp((l - max) / T)
   int V;
   float inv_t;                      // 1 / temperature

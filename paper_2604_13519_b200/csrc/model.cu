@@ -517,7 +517,7 @@ ts_status run_step(ts_model *m) {
   }
   if (m->last_sample) {
     ts::SampleArgs sa{};
-    sa.in = in; sa.logits = (const float *)m->WS(L.logits); sa.amax = amax;
+    sa.in = in; sa.logits = (float *)m->WS(L.logits); sa.amax = amax;
     sa.uni = (const float *)(di + L.o_uni); sa.part = (float *)m->WS(L.samp_stats);
     sa.V = c.vocab; sa.inv_t = m->last_inv_t; sa.k_max = c.k_max;
     sa.argmax = dout + L.o_argmax; sa.accept_len = dout + L.o_accept; sa.emitted = dout + L.o_emitted;
@@ -525,18 +525,18 @@ ts_status run_step(ts_model *m) {
     CU_TRY(ts::launch_sample_accept(sa, m->st));
     m->launched(5);
     m->launched(5);
-    return TS_OK;
+  } else {
+    ts::AcceptArgs ac{};
+    ac.in = in; ac.amax = amax;
+    ac.argmax = dout + L.o_argmax; ac.accept_len = dout + L.o_accept; ac.emitted = dout + L.o_emitted;
+    ac.new_len = dout + L.o_newlen; ac.new_pending = dout + L.o_newpend; ac.k_max = c.k_max;
+    ac.path = dout + L.o_path;
+    CU_TRY(ts::launch_accept(ac, m->st));
+    m->launched(5);
   }
-  ts::AcceptArgs ac{};
-  ac.in = in; ac.amax = amax;
-  ac.argmax = dout + L.o_argmax; ac.accept_len = dout + L.o_accept; ac.emitted = dout + L.o_emitted;
-  ac.new_len = dout + L.o_newlen; ac.new_pending = dout + L.o_newpend; ac.k_max = c.k_max;
-  ac.path = dout + L.o_path;
-  CU_TRY(ts::launch_accept(ac, m->st));
-  m->launched(5);
   if (m->last_tree) {   // the accepted path's K/V rows become the next cache positions
     ts::CompactArgs ca{};
-    ca.in = in; ca.accept_len = ac.accept_len; ca.path = ac.path; ca.k_max = c.k_max;
+    ca.in = in; ca.accept_len = dout + L.o_accept; ca.path = dout + L.o_path; ca.k_max = c.k_max;
     ca.kv_pool = (__half *)m->b.kv_pool; ca.layer_stride = L.kv_layer_stride; ca.v_offset = L.kv_v_offset;
     ca.n_layers = c.n_layers; ca.Hkv = c.n_kv_heads; ca.hd = c.head_dim;
     CU_TRY(ts::launch_kv_compact(ca, m->st));
@@ -635,9 +635,20 @@ ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::ve
   m->last_sample = uniforms != nullptr;
   if (m->last_sample) {
     if (c.path == 2) return fail(TS_ERR_UNIMPLEMENTED, "sampling acceptance needs the one-kernel-per-stage path");
-    if (m->last_tree) return fail(TS_ERR_UNIMPLEMENTED, "sampling acceptance over a draft tree");
     m->last_inv_t = 1.f / temperature;
-    std::memcpy(hi + L.o_uni, uniforms, sizeof(float) * M);
+    // the kernel reads uni[node c] for node c and the root's for the draw; a chain's caller gives value j for draft
+    // j + 1 and its chunk's last value for the draw
+    float *un = reinterpret_cast<float *>(hi + L.o_uni);
+    if (m->last_tree) {
+      std::memcpy(un, uniforms, sizeof(float) * M);
+    } else {
+      for (int i = 0, r = 0; i < B; ++i) {
+        const int k = hi[L.o_cu + i + 1] - hi[L.o_cu + i];
+        un[r] = uniforms[r + k - 1];
+        for (int j = 1; j < k; ++j) un[r + j] = uniforms[r + j - 1];
+        r += k;
+      }
+    }
   }
   if ((flags & TS_FLAG_WANT_TOPK) && c.path == 2)
     return fail(TS_ERR_UNIMPLEMENTED, "the per-position Top-K needs the one-kernel-per-stage path");
@@ -1224,6 +1235,24 @@ ts_status ts_verify_sampled(ts_model *m, ts_session *const *ss, int32_t B, const
       if (!(uniforms[r] >= 0.f && uniforms[r] < 1.f)) return fail(TS_ERR_ARG, "uniform %d outside [0, 1)", r);
   }
   return verify_impl(m, ss, B, draft_tokens, nullptr, draft_offsets, flags, out, nullptr, uniforms, temperature);
+}
+
+ts_status ts_verify_tree_sampled(ts_model *m, ts_session *const *ss, int32_t B, const int32_t *draft_tokens,
+                                 const int32_t *draft_parents, const int32_t *draft_offsets, float temperature,
+                                 const float *uniforms, uint32_t flags, ts_verify_result *out, int32_t *path_out) {
+  if (!uniforms) return fail(TS_ERR_ARG, "null uniforms");
+  if (!(temperature > 0.f) || !(temperature < 1e4f)) return fail(TS_ERR_ARG, "temperature must be in (0, 1e4)");
+  if (flags & TS_FLAG_SKIP_LM_HEAD) return fail(TS_ERR_ARG, "sampling acceptance needs the logits");
+  if (!draft_parents && draft_offsets && B >= 1 && draft_offsets[B] > draft_offsets[0])
+    return fail(TS_ERR_ARG, "null draft_parents");
+  if (draft_offsets && B >= 1 && B <= 4096) {
+    const int M = draft_offsets[B] - draft_offsets[0] + B;
+    for (int r = 0; r < M; ++r)
+      if (!(uniforms[r] >= 0.f && uniforms[r] < 1.f)) return fail(TS_ERR_ARG, "uniform %d outside [0, 1)", r);
+  }
+  static const int32_t none = 0;
+  return verify_impl(m, ss, B, draft_tokens, draft_parents ? draft_parents : &none, draft_offsets, flags, out, path_out,
+                     uniforms, temperature);
 }
 
 ts_status ts_verify_tree(ts_model *m, ts_session *const *ss, int32_t B, const int32_t *draft_tokens,

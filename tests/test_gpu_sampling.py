@@ -110,3 +110,52 @@ def test_sampled_batch_and_errors():
     with pytest.raises(ts.TsError):
         ts.ts_verify_sampled(gm, [s0], [d0], 1.0, [0.5, 1.0, 0.1, 0.2])  # a uniform outside [0, 1)
     gm.close()
+
+
+@pytest.mark.parametrize("name,ctx,n_nodes", [("tiny", 40, 12), ("8b-2l", 300, 24)])
+def test_sampled_acceptance_over_a_tree(name, ctx, n_nodes):
+    """ts_verify_tree_sampled against the oracle's walk with the same uniforms: path and emitted ids agree in at
+    least 90% of the trials (a floating-point decision next to its threshold may fall the other way); every result
+    is a root path of the tree followed by one more id; the cache after compaction matches the oracle's rows."""
+    shape = synth.SHAPES[name]
+    om, gm = make_pair(shape, k_max=max(n_nodes, 8), max_ctx=ctx + 64, path=1)
+    cache, s, pending = synthetic_context(shape, om, gm, ctx)
+    c, p, truth = cache.clone(), pending, []
+    for _ in range(4):
+        p = om.greedy_next(p, c)
+        truth.append(p)
+    g = np.random.Generator(np.random.Philox(key=[260413519, 0x5A3C00 + n_nodes]))
+    lg0 = om.forward_chunk([pending], cache.clone())[0]
+    second = [int(i) for i in torch.topk(lg0, 3).indices.tolist() if int(i) != truth[0]][:2]   # likely siblings of the truth
+    junk = lambda n: [int(t) for t in g.integers(64, shape.vocab, size=n)]
+    cands = [[second[0]] + junk(2), truth + junk(2), [second[1]] + junk(1), truth[:2] + junk(3), junk(3)]
+    toks, par = oracle.pack_candidates(cands, n_nodes)
+    z = [pending] + toks
+    logits, k_new, v_new = oracle.forward_tree(om, z, par, cache)
+    T = 1.0
+    while T > 1e-3 and float(oracle.target_probs(logits[0], T)[truth[0]]) < 0.4:
+        T /= 2
+    exact, lens = 0, []
+    for trial in range(40):
+        u = [min(float(x), 0.99999994) for x in g.random(len(z)).astype(np.float32)]
+        want_path, want_em = oracle.accept_sampled_tree(logits, z, par, T, u)
+        res, paths = ts.ts_verify_tree_sampled(gm, [s], [toks], [par[1:]], T, u)
+        r, path = res[0], paths[0]
+        em = list(r.emitted[:r.n_emitted])
+        assert path[0] == 0 and all(par[path[j]] == path[j - 1] for j in range(1, len(path)))
+        assert em[:-1] == [z[c] for c in path[1:]] and r.accept_len == len(path) - 1
+        exact += (path, em) == (want_path, want_em)
+        lens.append(len(want_path) - 1)
+    assert exact >= 36
+    assert 0 < sum(lens) and min(lens) < max(lens)              # walks of different lengths occurred
+    # commit the last trial if it agreed, and compare the compacted cache with the oracle's rows of that path
+    if (path, em) == (want_path, want_em):
+        ts.ts_commit(s, r)
+        n_new = ctx + len(path)
+        for l in range(shape.n_layers):
+            k, v = s.export_kv(l, n_new)
+            for got, want in ((k, k_new[l]), (v, v_new[l])):
+                ref = want[torch.tensor(path)]
+                d = (got[ctx:].double() - ref).abs()
+                assert bool((d <= 1e-2 + 1e-2 * ref.abs()).all())
+    gm.close()

@@ -87,3 +87,46 @@ def test_emitted_tokens_follow_the_model_distribution_whatever_the_draft():
             c, dof = _chi2(second, p1)
             assert dof >= 3 and c < dof + 5 * math.sqrt(2 * dof), (d0, c, dof)
         assert abs(acc0 / n - p0[d0]) < 5 * math.sqrt(p0[d0] * (1 - p0[d0]) / n) + 1e-9   # P(accept) = p(x)
+
+
+def test_tree_rule_on_a_chain_is_the_chain_rule():
+    """With parents j - 1 the tree walk is the chain rule, the uniforms renamed: node c's uniform is the chain's
+    u[c - 1], the tree's u[0] is the chain's sample uniform u[k - 1]."""
+    g = np.random.Generator(np.random.Philox(key=[11, 4]))
+    for _ in range(100):
+        k, V = int(g.integers(1, 7)), 20
+        logits = torch.tensor(g.normal(size=(k, V)) * 2, dtype=F64)
+        draft = [int(x) for x in g.integers(0, V, size=k - 1)]
+        T = float(g.choice([0.3, 1.0]))
+        u = [float(x) for x in g.random(k)]
+        l, em = oracle.accept_sampled(logits, draft, T, u)
+        ut = [u[k - 1]] + u[:k - 1]
+        path, em_t = oracle.accept_sampled_tree(logits, [7] + draft, [-1] + list(range(k - 1)), T, ut)
+        assert path == list(range(l + 1)) and em_t == em
+
+
+def test_tree_sampling_emits_the_model_distribution():
+    """Several candidates at the root and below its first child: the first emitted token follows p_0 and, given
+    that the walk took child 1, the second follows p_1 -- the residual bookkeeping is what makes this true."""
+    g = np.random.Generator(np.random.Philox(key=[11, 5]))
+    V, T, n = 10, 0.9, 40000
+    z = [0, 3, 7, 1, 4, 5]            # root; children of the root: 3, 7, 1 (nodes 1..3); children of node 1: 4, 5
+    parents = [-1, 0, 0, 0, 1, 1]
+    logits = torch.tensor(g.normal(size=(6, V)) * 1.2, dtype=F64)
+    p0 = oracle.target_probs(logits[0], T).numpy()
+    p1 = oracle.target_probs(logits[1], T).numpy()
+    order = [int(i) for i in np.argsort(-p0)]
+    z[1], z[2], z[3] = order[0], order[5], order[2]       # a likely first child, then an unlikely and a likely one
+    first, second, took1 = np.zeros(V), np.zeros(V), 0
+    us = g.random((n, 6))
+    for i in range(n):
+        path, em = oracle.accept_sampled_tree(logits, z, parents, T, [float(x) for x in us[i]])
+        first[em[0]] += 1
+        if len(path) > 1 and path[1] == 1:
+            took1 += 1
+            second[em[1]] += 1
+    c, dof = _chi2(first, p0)
+    assert c < dof + 5 * math.sqrt(2 * dof), (c, dof)
+    c, dof = _chi2(second, p1)
+    assert took1 > 2000 and c < dof + 5 * math.sqrt(2 * dof), (c, dof)
+    assert abs(took1 / n - p0[z[1]]) < 5 * math.sqrt(p0[z[1]] * (1 - p0[z[1]]) / n)   # the first child is taken with p(x)
