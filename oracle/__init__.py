@@ -13,4 +13,4 @@ from .tree import (verify_tree, forward_tree, accepted_path, ancestor_mask, node
                    pack_candidates)
 from .sampling import (target_probs, sample_inverse_cdf, accept_sampled, verify_sampled,   # noqa: F401
                        accept_sampled_tree)
-from .retrieval import cosine_scores, topk_cosine   # noqa: F401
+from .retrieval import cosine_scores, topk_cosine, HiddenStore   # noqa: F401

@@ -216,14 +216,11 @@ def suffix_match(y: Sequence[int], store: Datastore, ranks: Optional[Sequence[in
             e = store.entries[c]
             if len(e) <= L:
                 continue
-            if len(e) > 4096 or ranks is None and len(store.entries) > 2048:
-                m = _first_match_np(e, s)
-            else:
-                m = -1
-                for mm in range(L, len(e)):
-                    if e[mm - L:mm] == s:
-                        m = mm
-                        break
+            m = -1
+            for mm in range(L, len(e)):
+                if e[mm - L:mm] == s:
+                    m = mm
+                    break
             if m >= 0:
                 return e[m:m + n], (L, c, m)
     return [], (0, -1, -1)
@@ -322,19 +319,6 @@ def pack_candidates(candidates: Sequence[Sequence[int]], max_nodes: int):
                 children[u][t] = nxt
             u = nxt
     return tokens, parents
-
-
-def _first_match_np(e: Sequence[int], s: Sequence[int]) -> int:
-    """Same scan as the loop in suffix_match, vectorised (used only for very large stores)."""
-    a = np.asarray(e)
-    L = len(s)
-    if a.shape[0] <= L:
-        return -1
-    ok = np.ones(a.shape[0] - L, dtype=bool)        # window starts 0 .. |e|-L-1  (m = start+L < |e|)
-    for i in range(L):
-        ok &= a[i:i + a.shape[0] - L] == s[i]
-    idx = np.flatnonzero(ok)
-    return int(idx[0]) + L if idx.size else -1
 
 
 class Drafter:

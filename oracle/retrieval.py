@@ -27,3 +27,21 @@ def topk_cosine(H: torch.Tensor, q: torch.Tensor, K: int) -> Tuple[List[int], Li
     s = cosine_scores(H, q)
     order = sorted(range(s.numel()), key=lambda j: (-float(s[j]), j))[:K]
     return order, [float(s[j]) for j in order]
+
+
+class HiddenStore:
+    """The h_j half of the datastore H = {(h_j, y_j)} (Section 4.3): one hidden state per historical invocation, in
+    insertion order, the paper's "hidden representation of the input question at its final token".  States are kept
+    rounded to bf16, the storage type of the GPU datastore (a reading: the paper does not fix a type); the
+    similarity itself is float64."""
+
+    def __init__(self):
+        self.rows: List[torch.Tensor] = []
+
+    def add(self, h: torch.Tensor):
+        self.rows.append(h.to(torch.bfloat16))
+
+    def retrieve(self, h_x: torch.Tensor, K: int) -> Tuple[List[int], List[float]]:
+        """I_k of Eq. 3 for the query state h_x: indices of the K most similar entries, best first (all entries if the
+        store holds fewer than K)."""
+        return topk_cosine(torch.stack(self.rows), h_x, min(K, len(self.rows)))

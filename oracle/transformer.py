@@ -133,7 +133,20 @@ class OracleModel:
     # -- the row arithmetic shared by both drivers ------------------------------------------
     def _layer(self, l: int, x: torch.Tensor, pos: torch.Tensor, k_prev, v_prev, pos_prev,
                probe: Optional[dict] = None, allowed: Optional[torch.Tensor] = None):
+        xs, k_alls, v_alls = self._layer_multi(l, [x], [pos], [k_prev], [v_prev], [pos_prev], probe,
+                                               None if allowed is None else [allowed])
+        return xs[0], k_alls[0], v_alls[0]
+
+    def _layer_multi(self, l: int, xs, poss, k_prevs, v_prevs, pos_prevs, probe: Optional[dict] = None,
+                     alloweds=None):
+        """One decoder layer over several independent sequences (a batched step): sequence i has rows
+        xs[i] at positions poss[i] behind its own cached k_prevs[i], v_prevs[i].  Norms, projections
+        and the MLP act on rows, so they run once over all rows; attention runs per sequence.
+        Returns (new rows, all keys, all values), each a list over the sequences."""
         s, w = self.s, self.w
+        n_rows = [x.shape[0] for x in xs]
+        x = torch.cat(list(xs), dim=0)
+        pos = torch.cat(list(poss))
         T = x.shape[0]
         h = rmsnorm(x, w[f"l{l}.g1"], s.rms_eps)
         q = _wt(h, w[f"l{l}.wq"]).view(T, s.n_q_heads, s.head_dim)
@@ -141,10 +154,18 @@ class OracleModel:
         v = _wt(h, w[f"l{l}.wv"]).view(T, s.n_kv_heads, s.head_dim)
         q = rope(q, pos, s.rope_theta)
         k = rope(k, pos, s.rope_theta)
-        k_all = torch.cat([k_prev, k], dim=0)
-        v_all = torch.cat([v_prev, v], dim=0)
-        pos_all = torch.cat([pos_prev, pos])
-        o = attention(q, k_all, v_all, pos, pos_all, allowed).reshape(T, s.n_q_heads * s.head_dim)
+        o_parts, k_alls, v_alls = [], [], []
+        r0 = 0
+        for i, n in enumerate(n_rows):
+            k_all = torch.cat([k_prevs[i], k[r0:r0 + n]], dim=0)
+            v_all = torch.cat([v_prevs[i], v[r0:r0 + n]], dim=0)
+            pos_all = torch.cat([pos_prevs[i], poss[i]])
+            o_parts.append(attention(q[r0:r0 + n], k_all, v_all, poss[i], pos_all,
+                                     None if alloweds is None else alloweds[i]))
+            k_alls.append(k_all)
+            v_alls.append(v_all)
+            r0 += n
+        o = torch.cat(o_parts, dim=0).reshape(T, s.n_q_heads * s.head_dim)
         x = x + _wt(o, w[f"l{l}.wo"])
         h2 = rmsnorm(x, w[f"l{l}.g2"], s.rms_eps)
         a = swiglu(_wt(h2, w[f"l{l}.wg"]), _wt(h2, w[f"l{l}.wu"]))
@@ -152,7 +173,7 @@ class OracleModel:
         if probe is not None:
             probe[f"l{l}.q"], probe[f"l{l}.k"], probe[f"l{l}.v"] = q, k, v
             probe[f"l{l}.attn"], probe[f"l{l}.act"], probe[f"l{l}.x"] = o, a, x
-        return x, k_all, v_all
+        return list(torch.split(x, n_rows, dim=0)), k_alls, v_alls
 
     def _head(self, x: torch.Tensor) -> torch.Tensor:
         return _wt(rmsnorm(x, self.w["gf"], self.s.rms_eps), self.w["lm_head"])

@@ -182,6 +182,29 @@ def test_incremental_equals_full_recompute():
     assert cache.length == 21
 
 
+def test_batched_layer_equals_one_sequence_at_a_time():
+    """The layer over several sequences at once (what a batched verify step computes) is each sequence's own
+    forward: rows of different sequences never meet.  Checked against separate full recomputes of three sequences
+    of different lengths, split into a cached part and a chunk at different places."""
+    s = _small_shape()
+    m = oracle.OracleModel(s, _rand_weights(s, seed=12))
+    g = torch.Generator().manual_seed(13)
+    seqs = [[int(x) for x in torch.randint(0, s.vocab, (n,), generator=g)] for n in (19, 7, 30)]
+    cuts = [11, 0, 29]                                        # cached tokens per sequence (one empty cache)
+    caches = [m.new_cache() for _ in seqs]
+    for toks, cut, c in zip(seqs, cuts, caches):
+        if cut:
+            m.forward_chunk(toks[:cut], c)
+    xs = [m.w["embed"][torch.tensor(toks[cut:])].to(F64) for toks, cut in zip(seqs, cuts)]
+    poss = [torch.arange(cut, len(toks)) for toks, cut in zip(seqs, cuts)]
+    for l in range(s.n_layers):
+        xs, _, _ = m._layer_multi(l, xs, poss, [c.k[l] for c in caches], [c.v[l] for c in caches],
+                                  [torch.arange(cut) for cut in cuts])
+    for toks, cut, x in zip(seqs, cuts, xs):
+        want = m.forward_full(toks)[cut:]
+        assert torch.allclose(m._head(x), want, rtol=0, atol=1e-10)
+
+
 def test_verify_special_cases(tiny):
     s, w = tiny
     m = oracle.OracleModel(s, w)

@@ -31,6 +31,21 @@ def test_closed_forms_and_ties():
     assert oracle.topk_cosine(H * 3.0, q * 0.5, 5)[0] == idx
 
 
+def test_hidden_store_retrieval_is_torch_topk_over_the_stored_rows():
+    g = torch.Generator().manual_seed(5)
+    hs = torch.randn(37, 64, generator=g, dtype=F64)
+    store = oracle.HiddenStore()
+    for h in hs:
+        store.add(h)
+    q = hs[20] + 0.05 * torch.randn(64, generator=g, dtype=F64)
+    stored = hs.to(torch.bfloat16).to(F64)                       # what the store keeps: bf16-rounded rows
+    ref = torch.topk(F.cosine_similarity(stored, q[None, :], dim=1, eps=0.0), 10)
+    idx, sc = store.retrieve(q, 10)
+    assert idx == ref.indices.tolist() and idx[0] == 20
+    assert torch.allclose(torch.tensor(sc, dtype=F64), ref.values, rtol=0, atol=1e-14)
+    assert len(store.retrieve(q, 100)[0]) == 37                  # K above the store size: every entry, ranked
+
+
 def test_printed_k():
     gold = os.path.join(os.path.dirname(__file__), "golden", "paper_constants.txt")
     vals = dict(line.split("#")[0].split("=", 1) for line in open(gold) if "=" in line.split("#")[0])
