@@ -127,11 +127,27 @@ ts_status ts_schema_add_tool(ts_schema *s, const int32_t *name, int32_t name_len
                              const int32_t *key_tokens, const int32_t *key_offsets, int32_t n_keys);
 ts_status ts_schema_destroy(ts_schema *s);
 
-/* ---- datastore (Section 4.3: historical invocations y_j; hidden states h_j are not stored) ---- */
+/* ---- datastore (Section 4.3: H = {(h_j, y_j)}, historical invocations y_j with the hidden state h_j of the
+ * question that led to each) --------------------------------------------------------------------------------- */
 ts_status ts_datastore_create(int32_t n_tools, ts_datastore **out);
-/* Append one historical invocation (host ids, copied) and the tool it called (-1 = unknown).
- * Not allowed while a session created over this datastore is between ts_draft calls of a step. */
+/* Append one historical invocation y_j (host ids, copied) and the tool it called (-1 = unknown), without a hidden
+ * state.  Not allowed while a session created over this datastore is between ts_draft calls of a step, and not
+ * once hidden states are attached (TS_ERR_STATE: every entry then needs its h_j, see ts_datastore_add_hidden). */
 ts_status ts_datastore_add(ts_datastore *d, const int32_t *tokens, int32_t n, int32_t tool_id);
+/* Give the datastore the memory for its hidden states: hidden_dev is device memory owned by the caller, bf16
+ * [capacity][d_model] row-major, 16-byte aligned, kept alive until the datastore is destroyed or another matrix is
+ * attached; row j belongs to entry j.  The library allocates nothing and writes only rows it is told to.  Rows of
+ * entries that exist already must hold their states (e.g. a store restored from disk); capacity >= entries.
+ * hidden_dev = NULL detaches.  Errors: TS_ERR_ARG. */
+ts_status ts_datastore_attach_hidden(ts_datastore *d, void *hidden_dev, int32_t capacity, int32_t d_model);
+/* Append (h_j, y_j): y_j as ts_datastore_add, and h_j = the final-norm hidden state (the LM head's input) of row
+ * `row` of model m's last step, rounded to bf16, copied device to device into row j of the attached matrix on the
+ * model's stream.  The paper takes the question's hidden state at its final token: after ts_prefill of the
+ * question, that is row 0 of the session's first ts_verify.  Errors: TS_ERR_STATE (no matrix attached, matrix
+ * full, or the last step left no hidden state: it must run the LM head on the one-kernel-per-stage path),
+ * TS_ERR_ARG (row outside the step, width mismatch). */
+ts_status ts_datastore_add_hidden(ts_datastore *d, ts_model *m, int32_t row, const int32_t *tokens, int32_t n,
+                                  int32_t tool_id);
 ts_status ts_datastore_destroy(ts_datastore *d);
 
 /* ---- session: one sequence being decoded -------------------------------------------------------- */
@@ -255,8 +271,9 @@ ts_status ts_verify_sampled(ts_model *m, ts_session *const *sessions, int32_t B,
  * token x is accepted with probability r(x) / R, r being the node's p = softmax(logits / T) with the tokens of the
  * children already refused removed and R its total; if none is accepted (or the node is a leaf) one sample of the
  * residual is emitted and the step ends.  uniforms: one value in [0, 1) per chunk node, chunk after chunk: value c of
- * a chunk decides its node c (c >= 1), value 0 draws the sample.  Arguments, result, path and compaction as
- * ts_verify_tree; errors as ts_verify_tree and ts_verify_sampled. */
+ * a chunk decides its node c (c >= 1), value 0 draws the sample.  The children of a node must carry distinct tokens
+ * (a trie, as ts_draft_tree builds): TS_ERR_ARG otherwise.  Arguments, result, path and compaction as
+ * ts_verify_tree; other errors as ts_verify_tree and ts_verify_sampled. */
 ts_status ts_verify_tree_sampled(ts_model *m, ts_session *const *sessions, int32_t B,
                                  const int32_t *draft_tokens, const int32_t *draft_parents,
                                  const int32_t *draft_offsets, float temperature, const float *uniforms,
@@ -279,10 +296,15 @@ ts_status ts_profile_step(ts_model *m, float *ms_by_class, int32_t *launches_by_
 
 /* ts_commit — y <- y (+) emitted, q <- delta(q, .) applied id by id (bonus token included), cache
  * length and pending token advanced; stops at the first id that finishes the generation (call
- * complete, EOS, or max_new_tokens) and drops the rest.  Host only. */
+ * complete, EOS, or max_new_tokens) and drops the rest.  Host only.  One commit per verification: with
+ * a model behind the session, TS_ERR_STATE if no ts_verify* call has run since the last commit (or since
+ * ts_debug_set_cache / ts_debug_restart). */
 ts_status ts_commit(ts_session *s, const ts_verify_result *r);
 /* Same, with an emitted span chosen by the caller (n >= 1): the cache keeps the pending token and
- * the first n-1 ids, which must be the ids verified in the last step at those rows. */
+ * the first n-1 ids, which must be the ids the last verification was fed at rows 1 .. n-1 (after a tree
+ * step: along the accepted path) -- their K/V rows are what the cache holds there.  TS_ERR_ARG if n
+ * exceeds those rows or an id differs; the last id is free (it becomes the pending token).  A host-only
+ * session (no model) has no cache and takes any span. */
 ts_status ts_commit_forced(ts_session *s, const int32_t *emitted, int32_t n);
 
 typedef struct {
@@ -308,6 +330,16 @@ ts_status ts_session_output(const ts_session *s, int32_t *out, int32_t cap, int3
 #define TS_TOPK_SCRATCH_FLOATS(n, k) ((n) + 2 * (k) + 1 + 2 * (k) * (((n) + 4095) / 4096))
 ts_status ts_topk_cosine(ts_model *m, const void *hidden_dev, int32_t n_entries, const float *query_dev,
                          int32_t row, int32_t K, float *scores_dev, int32_t *out_index, float *out_score);
+/* ts_session_retrieve — the once-per-query part of Algorithm 1: compute h_x, retrieve the Top-K index set I_k (Eq. 3)
+ * from the session's datastore, and make it the candidate order of the suffix match.  h_x is the final-norm hidden
+ * state of row `row` of model m's last step (row 0 of the session's first step = the question's last token); the
+ * similarity runs over the hidden states attached to the datastore (ts_topk_cosine over rows [0, entries)); the K
+ * indices, best first, are installed as by ts_session_set_ranks and also written to out_index (host, K entries;
+ * out_score may be NULL).  K is lowered to the number of entries.  scores_dev: device scratch as in ts_topk_cosine.
+ * Errors: TS_ERR_STATE (no datastore, no hidden states attached, empty datastore, no hidden state in the last
+ * step), TS_ERR_ARG. */
+ts_status ts_session_retrieve(ts_model *m, ts_session *s, int32_t row, int32_t K, float *scores_dev,
+                              int32_t *out_index, float *out_score, int32_t *out_k);
 /* The final-norm hidden state (the LM head's input) of row `row` of the last step, as fp32 [d_model] on the host:
  * what a caller stores per question to build the datastore's hidden states.  TS_ERR_STATE if the last step skipped
  * the LM head or ran as the persistent kernel. */
@@ -332,7 +364,8 @@ ts_status ts_read_logits(ts_model *m, int32_t row0, int32_t n_rows, float *host_
 /* Copy the first `bytes` bytes of an internal activation buffer of the last step to host memory:
  * 0 residual stream x (float32 [rows_alloc][d_model]); 1 projection input activations (bf16
  * [planes][rows_alloc][d_model]; normalised with separate kernels, x times gain before the
- * row scale with the persistent kernel); 2 rotated queries (fp16 [rows_alloc][n_q_heads*head_dim]);
+ * row scale with the persistent kernel); 2 rotated queries (fp16 [rows_alloc][n_q_heads*head_dim], rounded values;
+ * the rounding remainders the attention kernel adds to them are kept beside them and are not returned);
  * 3 attention output (bf16 [planes][rows_alloc][n_q_heads*head_dim]); 4 SwiGLU output (bf16
  * [planes][rows_alloc][d_ffn]).  rows_alloc = max_rows rounded up to 128; planes = 1 + act_split. */
 ts_status ts_debug_read_buffer(ts_model *m, int32_t which, void *host_out, uint64_t bytes);
@@ -349,6 +382,12 @@ ts_status ts_debug_phase_clocks(ts_model *m, uint64_t *out, int32_t cap, int32_t
  * Host only; for testing the index arithmetic without a GPU. */
 ts_status ts_debug_schedule(int32_t n_tiles, int32_t n_kblocks, int32_t n_ctas, int32_t cta, int32_t cap,
                             int32_t *segments, int32_t *n_segments);
+/* Make the NEXT step (ts_verify*, ts_prefill chunk) report `code` (> 0) in its device status word, as a bounded
+ * device-side wait that expired would: the word is written on the model's stream after the step's last kernel and
+ * before the results are read back, so no kernel sees it and nothing is left waiting.  That step then fails with
+ * TS_ERR_DEVICE_TIMEOUT, the library clears the word and the persistent kernel's counters, and later steps run
+ * normally.  For testing the host's handling of a device timeout without making a GPU wait. */
+ts_status ts_debug_inject_device_error(ts_model *m, int32_t code);
 /* Counters: kernels launched since ts_init_model, bytes copied host->device and device->host by
  * ts_verify since then. */
 ts_status ts_model_counters(const ts_model *m, int64_t *launches, int64_t *h2d_bytes,
@@ -362,9 +401,11 @@ ts_status ts_model_counters(const ts_model *m, int64_t *launches, int64_t *h2d_b
  * callback that runs where cudaMalloc is forbidden, or a process working under a fixed memory
  * budget.  Such a caller cannot size and allocate the workspace that ts_init_model needs.
  * ts_attention_static runs the attention stage of the verify step (rows of the chunk against the
- * paged cache plus the chunk itself, causal inside the chunk; the same two kernels ts_verify uses)
- * with all of its scratch memory (per-split partial outputs, their running max / sum, the
- * row-tile table) in a fixed array of TS_STATIC_ATTN_SCRATCH_MIB MiB (plus about 0.5 MiB of
+ * paged cache plus the chunk itself, causal inside the chunk) as two kernels of its own -- a split-KV
+ * kernel on mma.sync tensor-core instructions and a merge kernel; ts_verify on a B200 runs a
+ * tensor-memory kernel instead, so results agree to rounding, not bit for bit -- with all of its
+ * scratch memory (per-split partial outputs, their running max / sum, the row-tile table, which a
+ * third small kernel builds from cu_rows on the device) in a fixed array of TS_STATIC_ATTN_SCRATCH_MIB MiB (plus about 0.5 MiB of
  * bookkeeping) that is part of the library image.  Every GPU on which the library is loaded
  * holds that array until the process exits.  The call itself allocates nothing, on the host
  * heap or on the device.
@@ -377,6 +418,8 @@ ts_status ts_model_counters(const ts_model *m, int64_t *launches, int64_t *h2d_b
  *   block_table  int32 [batch][pages_per_seq]: page ids of each sequence, in position order
  *   cu_rows      int32 [batch+1] row offsets (cu_rows[0] = 0), on the device and on the host
  *   seq_len      int32 [batch] tokens in the cache before the chunk, on the device and on the host
+ *                (the host copies are only checked against the limits; the kernels read the device
+ *                copies, which must hold the same values)
  *   out          bf16 [planes][out_rows][n_q_heads*head_dim]: plane 0 the rounded result, plane 1
  *                (planes = 2) the rounding remainder, as the output projection consumes them
  * Limits: head_dim 64 or 128; at most TS_K_MAX rows per sequence; rows * n_q_heads * head_dim * 4
@@ -384,7 +427,8 @@ ts_status ts_model_counters(const ts_model *m, int64_t *launches, int64_t *h2d_b
  * at most 512 row tiles of 64 packed rows.  Beyond them the call fails with TS_ERR_K_TOO_LARGE
  * and a message naming the limit; nothing is launched.
  * First use: the first call on each device looks up the array's device address (that device
- * must be current) and keeps it; make that first call outside any stream capture.
+ * must be current) and keeps it, so it must not be made while a stream is being captured.  No
+ * statement is made about capturing later calls.
  * Sharing: every call on a device uses the same array, which keeps whatever the previous call
  * left there.  No part of it has to start at zero: each call writes every word it later reads.
  * Two calls whose kernels overlap on the GPU (different streams, no ordering between them) race

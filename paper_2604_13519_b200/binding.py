@@ -90,6 +90,9 @@ _SIGNATURES = {
     "ts_schema_destroy": [_P],
     "ts_datastore_create": [C.c_int32, C.POINTER(_P)],
     "ts_datastore_add": [_P, _I32P, C.c_int32, C.c_int32],
+    "ts_datastore_attach_hidden": [_P, _P, C.c_int32, C.c_int32],
+    "ts_datastore_add_hidden": [_P, _P, C.c_int32, _I32P, C.c_int32, C.c_int32],
+    "ts_session_retrieve": [_P, _P, C.c_int32, C.c_int32, _P, _I32P, C.POINTER(C.c_float), _I32P],
     "ts_datastore_destroy": [_P],
     "ts_session_create": [_P, _P, _P, C.POINTER(ts_draft_config), C.POINTER(_P)],
     "ts_session_set_ranks": [_P, _I32P, C.c_int32],
@@ -122,6 +125,7 @@ _SIGNATURES = {
     "ts_debug_set_cache": [_P, C.c_int32, C.c_int32],
     "ts_read_logits": [_P, C.c_int32, C.c_int32, C.POINTER(C.c_float)],
     "ts_debug_read_buffer": [_P, C.c_int32, _P, C.c_uint64],
+    "ts_debug_inject_device_error": [_P, C.c_int32],
     "ts_model_counters": [_P, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64)],
     "ts_attention_static": [C.POINTER(ts_attention_args), _P],
     "ts_debug_phase_clocks": [_P, C.POINTER(C.c_uint64), C.c_int32, _I32P],
@@ -199,6 +203,20 @@ class Datastore:
 
     def add(self, tokens: Sequence[int], tool_id: int):
         _check(lib().ts_datastore_add(self.h, _i32(tokens), len(tokens), tool_id))
+        self.n += 1
+
+    def attach_hidden(self, hidden):
+        """hidden: CUDA bf16 tensor [capacity][d_model], owned by the caller (kept referenced here)."""
+        self.hidden = hidden
+        if hidden is None:
+            _check(lib().ts_datastore_attach_hidden(self.h, None, 0, 0))
+        else:
+            assert hidden.is_cuda and hidden.is_contiguous() and hidden.element_size() == 2
+            _check(lib().ts_datastore_attach_hidden(self.h, _P(hidden.data_ptr()), hidden.shape[0], hidden.shape[1]))
+
+    def add_hidden(self, model, row: int, tokens: Sequence[int], tool_id: int):
+        """Append (h_j, y_j): h_j = final-norm hidden state of `row` of the model's last step."""
+        _check(lib().ts_datastore_add_hidden(self.h, model.h, row, _i32(tokens), len(tokens), tool_id))
         self.n += 1
 
     def __del__(self):
@@ -290,6 +308,10 @@ class Model:
         buf = (C.c_uint64 * 4096)()
         _check(lib().ts_debug_phase_clocks(self.h, buf, 4096, C.byref(n)))
         return np.array(buf[:3 * n.value], dtype=np.uint64).reshape(3, n.value)
+
+    def inject_device_error(self, code: int):
+        """Test support: the next step reports `code` in its device status word (see toolspec.h)."""
+        _check(lib().ts_debug_inject_device_error(self.h, code))
 
     def counters(self):
         a, b, c = C.c_int64(), C.c_int64(), C.c_int64()
@@ -461,6 +483,20 @@ def ts_topk_cosine(model: Model, hidden, K: int, query=None, row: int = 0):
     return list(idx), list(sc)
 
 
+def ts_session_retrieve(model: Model, session: Session, K: int, row: int = 0):
+    """Algorithm 1's once-per-query step: h_x (row of the last step) -> Top-K over the datastore's hidden states ->
+    installed as the session's candidate order.  Returns (indices, scores), best first."""
+    torch = model.torch
+    N = session.store.n
+    k = max(1, min(K, N, 64))
+    scratch = torch.empty(N + 2 * k + 1 + 2 * k * ((N + 4095) // 4096), dtype=torch.float32, device=model.device)
+    idx = (C.c_int32 * 64)()
+    sc = (C.c_float * 64)()
+    nk = C.c_int32(0)
+    _check(lib().ts_session_retrieve(model.h, session.h, row, K, _P(scratch.data_ptr()), idx, sc, C.byref(nk)))
+    return list(idx[:nk.value]), list(sc[:nk.value])
+
+
 def ts_last_hidden(model: Model, row: int):
     import numpy as np
     out = np.empty(model.cfg.d_model, dtype=np.float32)
@@ -520,10 +556,12 @@ def ts_commit_forced(session: Session, emitted: Sequence[int]):
 
 
 def ts_attention_static(q, k_pages, v_pages, block_table, cu_rows: Sequence[int], seq_len: Sequence[int],
-                        n_q_heads: int, n_kv_heads: int, head_dim: int, out, stream=None):
+                        n_q_heads: int, n_kv_heads: int, head_dim: int, out, stream=None, cu_rows_dev=None,
+                        seq_len_dev=None):
     """Attention stage of the verify step with library-resident scratch (no device allocation in the
     call).  q, k_pages, v_pages: CUDA fp16 tensors; block_table: CUDA int32 [batch][pages_per_seq];
-    cu_rows / seq_len: Python ints (uploaded here as the device copies the call also needs);
+    cu_rows / seq_len: Python ints; their device copies (int32 CUDA tensors) are taken from cu_rows_dev /
+    seq_len_dev, or made here (an allocation by this wrapper, not by the library call) when those are None;
     out: CUDA bf16 tensor [planes][out_rows][n_q_heads*head_dim], written in place."""
     import torch
     B = len(seq_len)
@@ -532,8 +570,8 @@ def ts_attention_static(q, k_pages, v_pages, block_table, cu_rows: Sequence[int]
     a.batch, a.pages_per_seq = B, block_table.shape[1]
     a.planes, a.out_rows = out.shape[0], out.shape[1]
     h_cu, h_len = _i32(cu_rows), _i32(seq_len)
-    d_cu = torch.tensor(list(cu_rows), dtype=torch.int32, device=q.device)
-    d_len = torch.tensor(list(seq_len), dtype=torch.int32, device=q.device)
+    d_cu = cu_rows_dev if cu_rows_dev is not None else torch.tensor(list(cu_rows), dtype=torch.int32, device=q.device)
+    d_len = seq_len_dev if seq_len_dev is not None else torch.tensor(list(seq_len), dtype=torch.int32, device=q.device)
     a.cu_rows_host, a.seq_len_host = h_cu, h_len
     a.cu_rows, a.seq_len, a.block_table = d_cu.data_ptr(), d_len.data_ptr(), block_table.data_ptr()
     a.q, a.k_pages, a.v_pages, a.out = q.data_ptr(), k_pages.data_ptr(), v_pages.data_ptr(), out.data_ptr()

@@ -64,6 +64,9 @@ attn_split_kernel(const AttnArgs a) {
   extern __shared__ __align__(128) uint8_t sm[];
   uint8_t *sQ = sm, *sK = sm + TILE, *sV = sm + 3 * TILE;   // K and V: two stages each
 
+  // Everything this kernel reads (the row-tile table included) may come from the kernel before it.
+  pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
+  pdl_wait();
   const int split = blockIdx.x, kh = blockIdx.y, tile = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = a.Hq / a.Hkv;
@@ -80,9 +83,6 @@ attn_split_kernel(const AttnArgs a) {
   const int b0 = split * bps;
   const int b1 = min(min(nblk, b0 + bps), (len + j_max + 1 + kBlk - 1) / kBlk);
   const int32_t *btab = a.in.block_tab + (size_t)seq * a.in.pages_per_seq;
-
-  pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
-  pdl_wait();
 
   // this thread's two rows of the warp's 16-row tile
   const int rl = warp * 16 + (lane >> 2), rh = rl + 8;
@@ -286,15 +286,16 @@ static cudaError_t launch_attn_pdl(K kernel, dim3 grid, dim3 block, size_t smem,
 }
 
 cudaError_t launch_attention_split(const AttnArgs &a, cudaStream_t st) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce once;
+  int dev_ = -1;
+  if (once.needed(&dev_)) {
     cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          5 * kBlk * 128 * 2);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              5 * kBlk * 64 * 2);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    once.done(dev_);
   }
   const dim3 grid(a.n_splits, a.Hkv, a.n_row_tiles_total);
   const size_t smem = (size_t)5 * kBlk * a.hd * 2;

@@ -5,7 +5,8 @@
 //
 // The array's name is a host-side stand-in in host code: the device address is looked up once per
 // device with cudaGetSymbolAddress (with that device current) and only that address is handed to
-// the kernels and to the copy that uploads the row-tile table.
+// the kernels.  Nothing is copied from host memory: the row-tile table is built on the device, from
+// the caller's device copy of the row offsets, by a small kernel ahead of the attention kernels.
 #include <algorithm>
 #include <mutex>
 
@@ -28,6 +29,22 @@ constexpr int kMaxAttnSplits = ts::kAttnMaxSplits;
 
 static __device__ __align__(256) unsigned char g_attn_scratch[kScratchBytes];
 
+// Row-tile table of the attention kernel: tile t covers packed rows [row0, row0 + 64) of sequence seq; a
+// sequence of k rows and G query heads per kv head has ceil(k * G / 64) tiles.  One thread: a few hundred
+// entries at most.  Entries past max_tiles are not written (the host has checked the count already).
+__global__ void static_tile_table_kernel(const int32_t *cu_rows, int batch, int G, int max_tiles, int32_t *tile_seq,
+                                         int32_t *tile_row0) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  int t = 0;
+  for (int i = 0; i < batch; ++i) {
+    const int k = cu_rows[i + 1] - cu_rows[i];
+    for (int r0 = 0; r0 < k * G && t < max_tiles; r0 += 64, ++t) {
+      tile_seq[t] = i;
+      tile_row0[t] = r0;
+    }
+  }
+}
+
 std::mutex g_mu;
 unsigned char *g_dev_ptr[kMaxDevices];   // device address of g_attn_scratch, per device
 int g_sms[kMaxDevices];
@@ -47,7 +64,6 @@ extern "C" ts_status ts_attention_static(const ts_attention_args *a, void *strea
   if (a->planes != 1 && a->planes != 2) return set_error(TS_ERR_ARG, "planes must be 1 or 2");
   const int G = a->n_q_heads / a->n_kv_heads;
   int tiles = 0, max_total = 0;
-  int32_t tile_tab[2 * kMaxTiles] = {};   // [0, kMaxTiles): sequence of each 64-row tile; then its first packed row
   if (a->cu_rows_host[0] != 0) return set_error(TS_ERR_ARG, "cu_rows must start at 0");
   for (int i = 0; i < a->batch; ++i) {
     const int k = a->cu_rows_host[i + 1] - a->cu_rows_host[i];
@@ -56,10 +72,7 @@ extern "C" ts_status ts_attention_static(const ts_attention_args *a, void *strea
     const long long total = (long long)a->seq_len_host[i] + k;
     if ((total + TS_PAGE_SIZE - 1) / TS_PAGE_SIZE > a->pages_per_seq)
       return set_error(TS_ERR_ARG, "sequence %d needs more pages than pages_per_seq", i);
-    for (int r0 = 0; r0 < k * G; r0 += 64) {
-      if (tiles < kMaxTiles) { tile_tab[tiles] = i; tile_tab[kMaxTiles + tiles] = r0; }
-      ++tiles;
-    }
+    tiles += (k * G + 63) / 64;
     max_total = total > max_total ? (int)total : max_total;
   }
   const int M = a->cu_rows_host[a->batch];
@@ -102,9 +115,11 @@ extern "C" ts_status ts_attention_static(const ts_attention_args *a, void *strea
   s = (int)std::min<size_t>((size_t)s, kPartOBytes / per_split);
 
   cudaStream_t st = (cudaStream_t)stream;
-  // the table is in pageable host memory, so the copy has left tile_tab when the call returns
-  e = cudaMemcpyAsync(base + kPartOBytes + kPartMlBytes, tile_tab, kTileBytes, cudaMemcpyHostToDevice, st);
-  if (e != cudaSuccess) return set_error(TS_ERR_CUDA, "tile-table upload: %s", cudaGetErrorString(e));
+  int32_t *tile_seq = reinterpret_cast<int32_t *>(base + kPartOBytes + kPartMlBytes);
+  static_tile_table_kernel<<<1, 32, 0, st>>>((const int32_t *)a->cu_rows, a->batch, G, kMaxTiles, tile_seq,
+                                             tile_seq + kMaxTiles);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return set_error(TS_ERR_CUDA, "tile-table launch: %s", cudaGetErrorString(e));
 
   ts::AttnArgs aa{};
   aa.in.cu_rows = a->cu_rows; aa.in.seq_len = a->seq_len; aa.in.block_tab = a->block_table;
@@ -114,8 +129,8 @@ extern "C" ts_status ts_attention_static(const ts_attention_args *a, void *strea
   aa.n_splits = s; aa.n_row_tiles_total = tiles;
   aa.part_o = reinterpret_cast<float *>(base);
   aa.part_ml = reinterpret_cast<float2 *>(base + kPartOBytes);
-  aa.tile_seq = reinterpret_cast<const int32_t *>(base + kPartOBytes + kPartMlBytes);
-  aa.tile_row0 = aa.tile_seq + kMaxTiles;
+  aa.tile_seq = tile_seq;
+  aa.tile_row0 = tile_seq + kMaxTiles;
   aa.out = (__nv_bfloat16 *)a->out; aa.out_rows = a->out_rows; aa.planes = a->planes;
   e = ts::launch_attention_split(aa, st);
   if (e != cudaSuccess) return set_error(TS_ERR_CUDA, "attention launch: %s", cudaGetErrorString(e));

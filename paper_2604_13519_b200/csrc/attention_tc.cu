@@ -1,6 +1,6 @@
 // Paged grouped-query attention of the verify chunk on the 5th-generation tensor cores, as a kernel of its own.
 //
-// One CTA = one unit: (128-row tile of packed (position, query head) rows, kv head, split of the KV positions).
+// One CTA = one unit: (128-row tile of packed (position, query head) rows, kv head, leaf of the KV positions).
 //   warp 0   K/V producer: TMA loads of 64-position blocks straight from the pages (5-d tensor map over the pool)
 //   warp 1   tensor memory allocation + tcgen05.mma issue:  S = Q K^T  (Q tile and K block K-major in shared
 //            memory, 128 x 64 fp32 result in tensor memory), then  O_blk = P V  with P read from tensor memory
@@ -8,7 +8,7 @@
 //   warps 2..5  one row per thread: maximum over the block's 64 scores, P = exp2(S - reference maximum) written back
 //            to tensor memory as fp16.  The output sums stay in tensor memory (every P V adds to them); the
 //            reference maximum follows the running one in steps, and only then is the row of sums multiplied down
-// Each split writes an un-normalised partial output with its (max, sum); attn_combine_kernel merges the splits.
+// Each leaf writes an un-normalised partial output with its (max, sum); attn_merge_kernel adds a row's leaves.
 // Every wait is bounded; on expiry the CTA records an error word and leaves through the normal exit.
 #include <cuda_fp16.h>
 
@@ -59,16 +59,20 @@ __device__ __forceinline__ bool mbar_wait_err(uint32_t bar, uint32_t parity, con
 }
 
 struct AttnUnit {
-  int tile, kh, split;
+  int tile, kh, leaf;
   int seq, row0, rows_here, r_beg, len, G;
   int pos_beg, pos_end, nblk;
 };
 
+// CTA u works on pair u / Hkv (a row tile and one leaf of its sequence) for kv head u % Hkv.  The leaf's positions
+// are [leaf * leaf_len, (leaf + 1) * leaf_len), cut off at the end of the chunk: absolute positions, so the blocks a
+// row meets, and their order, do not depend on where the chunk starts or how long it is.
 __device__ __forceinline__ AttnUnit attn_unit_info(const AttnTcArgs &a, int u) {
   AttnUnit t;
-  t.split = u % a.attn_splits;
-  t.kh = (u / a.attn_splits) % a.Hkv;
-  t.tile = u / (a.attn_splits * a.Hkv);
+  const int pair = u / a.Hkv;
+  t.kh = u - pair * a.Hkv;
+  t.tile = a.unit_tile[pair];
+  t.leaf = a.unit_leaf[pair];
   t.G = a.Hq / a.Hkv;
   t.seq = a.tile_seq[t.tile];
   t.row0 = a.tile_row0[t.tile];
@@ -76,12 +80,8 @@ __device__ __forceinline__ AttnUnit attn_unit_info(const AttnTcArgs &a, int u) {
   const int k_i = a.in.cu_rows[t.seq + 1] - t.r_beg;
   t.len = a.in.seq_len[t.seq];
   t.rows_here = min(kAttnRows, k_i * t.G - t.row0);
-  const int total = t.len + k_i;
-  const int j_max = (t.row0 + t.rows_here - 1) / t.G;
-  int p0, p1;
-  split_blocks((total + 15) >> 4, a.attn_splits, t.split, &p0, &p1);
-  t.pos_beg = p0 << 4;
-  t.pos_end = min(min(p1 << 4, total), t.len + j_max + 1);   // nothing beyond the last row's own position is visible
+  t.pos_beg = t.leaf * a.leaf_len;
+  t.pos_end = min(t.pos_beg + a.leaf_len, t.len + k_i);
   t.nblk = t.pos_end > t.pos_beg ? (t.pos_end - t.pos_beg + kAttnBlk - 1) / kAttnBlk : 0;
   return t;
 }
@@ -121,20 +121,22 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
   const int pr = t.row0 + row;        // packed row of the sequence
   const bool valid = row < t.rows_here;
   const int j = valid ? pr / t.G : 0, gq = valid ? pr % t.G : 0;
-  const size_t ob = ((size_t)(t.r_beg + j) * a.Hq + t.kh * t.G + gq) * a.attn_splits + t.split;
-  if (t.nblk == 0) {   // nothing visible in this split: mark it empty
+  const size_t ob = ((size_t)(t.r_beg + j) * a.Hq + t.kh * t.G + gq) * a.n_slots + t.leaf;
+  if (t.nblk == 0) {   // no position in this leaf: mark it empty
     if (valid) a.attn_ml[ob] = make_float2(-INFINITY, 0.f);
     return true;
   }
-  // ---- stage Q: [128 rows][64 elements] images with the 128-byte swizzle, one per 64-element half ----------
+  // ---- stage Q: [128 rows][64 elements] images with the 128-byte swizzle, one per 64-element half, first of the
+  // values, then of their rounding remainders -------------------------------------------------------------
   for (int idx = wtid; idx < kAttnRows * CH; idx += kWorkers) {
     const int r = idx / CH, c = idx % CH;
     const int prr = t.row0 + r;
     const bool v = r < t.rows_here;
     const int jj = v ? prr / t.G : 0, gg = v ? prr % t.G : 0;
-    const __half *src = a.q + ((size_t)(t.r_beg + jj) * a.Hq + t.kh * t.G + gg) * HD + c * 8;
+    const size_t so = ((size_t)(t.r_beg + jj) * a.Hq + t.kh * t.G + gg) * HD + c * 8;
     const uint32_t dst = smem_u32(sQ) + (c >> 3) * (kAttnRows * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4);
-    cp_async16z(dst, src, v);
+    cp_async16z(dst, a.q + so, v);
+    cp_async16z(dst + kAttnRows * HD * 2, a.q_lo + so, v);
   }
   cp_commit_wait_all();
   fence_proxy_async_all();   // generic-proxy writes -> tcgen05 (async proxy) reads
@@ -282,7 +284,7 @@ template <int HD>
 __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_constant__ AttnTcArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  constexpr uint32_t kQBytes = kAttnRows * HD * 2, kKvBytes = 2u * kAttnBlk * HD * 2, kHalves = HD / 64;
+  constexpr uint32_t kQBytes = 2u * kAttnRows * HD * 2, kKvBytes = 2u * kAttnBlk * HD * 2, kHalves = HD / 64;   // Q: two planes
   AttnCtl *ctl = reinterpret_cast<AttnCtl *>(smem + kQBytes + kKvStages * kKvBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int *err = a.err;
@@ -371,12 +373,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         if (!mbar_wait_err(smem_u32(&ctl->s_empty[st]), ((b >> 1) & 1) ^ 1, err)) { ok = false; break; }
         tc_fence_after();
         const uint32_t sK = sQ + kQBytes + kst * kKvBytes;
+        // S = Q K^T + Q_lo K^T: the remainder plane of the queries goes through the same keys into the same sums
 #pragma unroll
-        for (int hh = 0; hh < (int)kHalves; ++hh) {
-          const uint64_t dq = umma_desc_sw128(sQ + hh * (kAttnRows * 128)), dk = umma_desc_sw128(sK + hh * (kAttnBlk * 128));
+        for (int pl = 0; pl < 2; ++pl) {
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk)
-            umma_bf16(tmem_base + kColS + st * 64, dq + 2 * kk, dk + 2 * kk, idesc_qk, (hh | kk) != 0 ? 1u : 0u);
+          for (int hh = 0; hh < (int)kHalves; ++hh) {
+            const uint64_t dq = umma_desc_sw128(sQ + pl * (kAttnRows * HD * 2) + hh * (kAttnRows * 128));
+            const uint64_t dk = umma_desc_sw128(sK + hh * (kAttnBlk * 128));
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              umma_bf16(tmem_base + kColS + st * 64, dq + 2 * kk, dk + 2 * kk, idesc_qk, (pl | hh | kk) != 0 ? 1u : 0u);
+          }
         }
         umma_commit(smem_u32(&ctl->s_full[st]));
         if (b > 0) ok = issue_pv(b - 1);
@@ -398,21 +405,84 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
   }
 }
 
+// grid = (M, Hq), hd threads: add the leaves of one (row, query head) and emit the normalised row as bf16 (hi[, lo]).
+// The row's sequence has n_leaves = ceil((cached length + chunk rows) / leaf_len) leaves, all of them written (a
+// leaf the row cannot see carries sum 0 and gets weight 0).  Lane s of each warp turns leaf s's (max, sum) into a
+// weight; every thread loads its output element of all leaves at once (one round trip to L2) and adds them in leaf
+// order.  NS = compile-time bound on the number of leaves.
+template <int NS>
+__global__ void attn_merge_kernel(const AttnTcArgs a) {
+  pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
+  pdl_wait();
+  const int m = blockIdx.x, h = blockIdx.y, d = threadIdx.x, lane = threadIdx.x & 31;
+  const int seq = a.in.row_seq[m];
+  const int total = a.in.seq_len[seq] + (a.in.cu_rows[seq + 1] - a.in.cu_rows[seq]);
+  const int nl = (total + a.leaf_len - 1) / a.leaf_len;
+  const size_t base = ((size_t)m * a.Hq + h) * a.n_slots;
+  const float2 ml = lane < nl ? a.attn_ml[base + lane] : make_float2(-INFINITY, 0.f);
+  float t[NS];
+#pragma unroll
+  for (int s = 0; s < NS; ++s) t[s] = (s < nl) ? a.attn_o[(base + s) * a.hd + d] : 0.f;
+  float mx = ml.y > 0.f ? ml.x : -INFINITY;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  float w = ml.y > 0.f ? exp2f(ml.x - mx) : 0.f;
+  // the denominator: leaf by leaf in leaf order (a shuffle tree would pair lanes differently as leaves are added)
+  float den = 0.f, num = 0.f;
+#pragma unroll
+  for (int s = 0; s < NS; ++s) {
+    const float ws = __shfl_sync(0xffffffffu, w, s);
+    const float ls = __shfl_sync(0xffffffffu, ml.y, s);
+    if (ws != 0.f) { den += ws * ls; num += ws * t[s]; }
+  }
+  num *= 1.f / den;
+  __nv_bfloat16 hi, lo;
+  split_bf16(num, hi, lo);
+  const size_t col = (size_t)h * a.hd + d;
+  const size_t ld = (size_t)a.Hq * a.hd;
+  a.out[(size_t)m * ld + col] = hi;
+  if (a.planes == 2) a.out[((size_t)a.out_rows + m) * ld + col] = lo;
+}
+
+template <typename K>
+static cudaError_t launch_merge_pdl(K kernel, const AttnTcArgs &a, cudaStream_t st) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(a.in.M, a.Hq);
+  cfg.blockDim = dim3(a.hd);
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, a);
+}
+
+cudaError_t launch_attention_tc_merge(const AttnTcArgs &a, cudaStream_t st) {
+  if (a.n_slots < 1 || a.n_slots > kAttnMaxSplits) return cudaErrorInvalidValue;
+  if (a.n_slots <= 2) return launch_merge_pdl(attn_merge_kernel<2>, a, st);
+  if (a.n_slots <= 4) return launch_merge_pdl(attn_merge_kernel<4>, a, st);
+  if (a.n_slots <= 8) return launch_merge_pdl(attn_merge_kernel<8>, a, st);
+  if (a.n_slots <= 16) return launch_merge_pdl(attn_merge_kernel<16>, a, st);
+  return launch_merge_pdl(attn_merge_kernel<32>, a, st);
+}
+
 static size_t attn_tc_smem(int hd) {
-  return 1024 + (size_t)kAttnRows * hd * 2 + (size_t)kKvStages * 2 * kAttnBlk * hd * 2 + sizeof(AttnCtl) + 64;
+  return 1024 + (size_t)2 * kAttnRows * hd * 2 + (size_t)kKvStages * 2 * kAttnBlk * hd * 2 + sizeof(AttnCtl) + 64;
 }
 
 cudaError_t launch_attention_tc(const AttnTcArgs &a, cudaStream_t st) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce once;
+  int dev_ = -1;
+  if (once.needed(&dev_)) {
     cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_tc_smem(128));
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_tc_smem(64));
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    once.done(dev_);
   }
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(a.n_tiles * a.Hkv * a.attn_splits);
+  cfg.gridDim = dim3(a.n_units * a.Hkv);
   cfg.blockDim = dim3(kTcThreads);
   cfg.dynamicSmemBytes = attn_tc_smem(a.hd);
   cfg.stream = st;

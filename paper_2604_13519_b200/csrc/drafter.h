@@ -39,6 +39,10 @@ struct ts_datastore {
   std::vector<int64_t> offset{0};    // entry e = tokens[offset[e] .. offset[e+1])
   std::vector<int32_t> tool_of;
   std::vector<int64_t> freq;         // per tool
+  // hidden states h_j of the entries (Section 4.3: H = {(h_j, y_j)}): a caller-owned device matrix, bf16
+  // [hidden_capacity][hidden_width] row-major, row j = entry j; null until attached
+  void *hidden_dev = nullptr;
+  int32_t hidden_capacity = 0, hidden_width = 0;
   // index over every position m with a 5-gram ending at m and a non-empty continuation
   struct Posting { uint64_t key; int32_t entry; int32_t m; };
   mutable std::vector<Posting> index;

@@ -114,7 +114,7 @@ __device__ __forceinline__ __half to_half_sat(float x) {
 // grid = (M, Hq + 2*Hkv); one CTA of hd/2 threads per (row, head).  Thread i handles the rotary pair
 // (i, i + hd/2) of q or k heads, or elements (i, i + hd/2) of a v head.
 __global__ void rope_kv_kernel(StepIn in, const float *part, int n_splits, int part_rows, int Hq, int Hkv, int hd,
-                               const float2 *rope_tab, __half *q_out, __half *k_pages, __half *v_pages) {
+                               const float2 *rope_tab, __half *q_out, __half *q_lo_out, __half *k_pages, __half *v_pages) {
   pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
   pdl_wait();
   const int m = blockIdx.x, head = blockIdx.y, i = threadIdx.x, half = hd >> 1;
@@ -135,9 +135,16 @@ __global__ void rope_kv_kernel(StepIn in, const float *part, int n_splits, int p
     a = ra; b = rb;
   }
   if (head < Hq) {
-    __half *q = q_out + ((size_t)m * Hq + head) * hd;
-    q[i] = to_half_sat(a);
-    q[i + half] = to_half_sat(b);
+    // the query as an fp16 pair (value, rounding remainder): the score product adds both, so the 11 bits of fp16
+    // do not limit the scores (the remainder of a saturated value is dropped)
+    const size_t qo = ((size_t)m * Hq + head) * hd;
+    const __half ha = to_half_sat(a), hb = to_half_sat(b);
+    q_out[qo + i] = ha;
+    q_out[qo + i + half] = hb;
+    if (q_lo_out) {
+      q_lo_out[qo + i] = __float2half_rn(fabsf(a) <= 65504.f ? a - __half2float(ha) : 0.f);
+      q_lo_out[qo + i + half] = __float2half_rn(fabsf(b) <= 65504.f ? b - __half2float(hb) : 0.f);
+    }
   } else {
     const int seq = in.row_seq[m];
     const int slot = in.slot[m];
@@ -151,10 +158,10 @@ __global__ void rope_kv_kernel(StepIn in, const float *part, int n_splits, int p
 }
 
 cudaError_t launch_rope_kv(const StepIn &in, const float *part, int n_splits, int part_rows, int Hq, int Hkv,
-                           int hd, const float2 *rope_tab, __half *q_out, __half *k_pages, __half *v_pages,
-                           cudaStream_t st) {
+                           int hd, const float2 *rope_tab, __half *q_out, __half *q_lo_out, __half *k_pages,
+                           __half *v_pages, cudaStream_t st) {
   return launch_pdl(rope_kv_kernel, dim3(in.M, Hq + 2 * Hkv), dim3(hd / 2), 0, st, in, part, n_splits,
-                    part_rows, Hq, Hkv, hd, rope_tab, q_out, k_pages, v_pages);
+                    part_rows, Hq, Hkv, hd, rope_tab, q_out, q_lo_out, k_pages, v_pages);
 }
 
 // One CTA per source row; thread i moves 16 bytes.  Block (tile, kb) of the stored matrix starts at row

@@ -299,10 +299,8 @@ __device__ __forceinline__ AttnUnit attn_unit_info(const FusedArgs &a, int u) {
   t.rows_here = min(kAttnRows, k_i * t.G - t.row0);
   const int total = t.len + k_i;
   const int j_max = (t.row0 + t.rows_here - 1) / t.G;
-  int p0, p1;
-  split_pages((total + 15) >> 4, a.attn_splits, t.split, &p0, &p1);
-  t.pos_beg = p0 << 4;
-  t.pos_end = min(min(p1 << 4, total), t.len + j_max + 1);   // nothing beyond the last row's own position is visible
+  // (nothing beyond the last row's own position is visible)
+  split_positions(t.len, min(total, t.len + j_max + 1), a.attn_splits, t.split, 4, &t.pos_beg, &t.pos_end);
   t.nblk = t.pos_end > t.pos_beg ? (t.pos_end - t.pos_beg + kAttnBlk - 1) / kAttnBlk : 0;
   return t;
 }
@@ -1002,11 +1000,12 @@ int fused_ring_stages(int planes, int Mc, int hd, size_t smem_limit) {
 }
 
 cudaError_t launch_fused(FusedArgs a, size_t smem_limit, cudaStream_t st) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce once;
+  int dev_ = -1;
+  if (once.needed(&dev_)) {
     cudaError_t e = cudaFuncSetAttribute(fused_verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_limit);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    once.done(dev_);
   }
   a.ring = fused_ring_stages(a.planes, a.Mc, a.hd, smem_limit);
   if (a.ring < 2) return cudaErrorInvalidConfiguration;

@@ -237,12 +237,13 @@ int gemm_pick_stages(int planes, int Mc, size_t smem_budget) {
 template <int EPI>
 static cudaError_t launch_one(const CUtensorMap &tw, const CUtensorMap &ta, const GemmArgs &g, dim3 grid,
                               size_t smem, cudaStream_t st, bool pdl) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce once;
+  int dev_ = -1;
+  if (once.needed(&dev_)) {
     cudaError_t e = cudaFuncSetAttribute(gemm_ws_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          227 * 1024);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    once.done(dev_);
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = grid;

@@ -6,9 +6,24 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "common.cuh"
 
 namespace ts {
+
+// A function attribute (the opt-in to large dynamic shared memory) is set per DEVICE, so "done once" has to be kept
+// per device ordinal: bit d of the mask = done on device d.  Setting an attribute twice is harmless, so a race
+// between two threads on their first launch costs a repeated call and nothing else.
+struct PerDeviceOnce {
+  std::atomic<uint64_t> mask{0};
+  // true if the caller still has to do the set-up on the current device; *dev receives its ordinal (-1 = unknown)
+  bool needed(int *dev) {
+    if (cudaGetDevice(dev) != cudaSuccess || *dev < 0 || *dev >= 64) { *dev = -1; return true; }
+    return !((mask.load(std::memory_order_acquire) >> *dev) & 1ull);
+  }
+  void done(int dev) { if (dev >= 0) mask.fetch_or(1ull << dev, std::memory_order_release); }
+};
 
 enum : int { EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_LOGITS = 2 };
 
@@ -56,10 +71,11 @@ cudaError_t launch_embed_norm(const StepIn &in, const __nv_bfloat16 *embed, cons
 // x[m] += sum_s part[s][m]; h = rmsnorm(x) * gain -> bf16 (hi[, lo])
 cudaError_t launch_add_norm(int M, int d, const float *part, int n_splits, int part_rows, const float *gain,
                             float eps, float *x, __nv_bfloat16 *h, int h_rows, int planes, cudaStream_t st);
-// qkv = sum of split-K partials; rotary on q and k; q -> fp16 [M][Hq][hd]; k, v -> fp16 pages
+// qkv = sum of split-K partials; rotary on q and k; q -> fp16 [M][Hq][hd] (and, if q_lo_out is given, the rounding
+// remainder of every element as a second fp16 array of the same shape); k, v -> fp16 pages
 cudaError_t launch_rope_kv(const StepIn &in, const float *part, int n_splits, int part_rows, int Hq, int Hkv,
-                           int hd, const float2 *rope_tab, __half *q_out, __half *k_pages, __half *v_pages,
-                           cudaStream_t st);
+                           int hd, const float2 *rope_tab, __half *q_out, __half *q_lo_out, __half *k_pages,
+                           __half *v_pages, cudaStream_t st);
 
 constexpr int kAttnMaxSplits = 32;   // KV splits per (row tile, kv head): one lane of the merge kernel each
 
@@ -81,20 +97,32 @@ struct AttnArgs {
 cudaError_t launch_attention_split(const AttnArgs &a, cudaStream_t st);
 cudaError_t launch_attention_combine(const AttnArgs &a, cudaStream_t st);
 
-// tcgen05 attention as a kernel of its own (attention_tc.cu): one CTA per (128-row tile, kv head, split)
+// tcgen05 attention as a kernel of its own (attention_tc.cu): one CTA per (128-row tile, leaf, kv head).
+// A leaf is a run of leaf_len KV positions starting at an absolute multiple of leaf_len (a model constant, a
+// multiple of 64): leaf L of a sequence holds positions [L * leaf_len, (L + 1) * leaf_len), whatever the cached
+// length or the chunk length.  Every leaf yields one partial result per row, and the merge adds a row's leaves in
+// leaf order, so the bits of a row's attention output are a function of its position and its prefix only: the same
+// token gets the same logits whether it is verified alone (vanilla decoding) or as row j of a chunk.
 struct AttnTcArgs {
   StepIn in;
   int Hq, Hkv, hd, layer;
-  int n_tiles, attn_splits;
-  const int32_t *tile_seq;       // [n_tiles] sequence of each 128-row tile of packed rows
-  const int32_t *tile_row0;      // [n_tiles] first packed row of the tile
-  const __half *q;               // [M][Hq][hd] rotated queries
+  int leaf_len;                  // KV positions per leaf
+  int n_units;                   // (tile, leaf) pairs of this step; the grid is n_units * Hkv CTAs
+  int n_slots;                   // partial results kept per (row, query head): the most leaves any sequence has
+  const int32_t *unit_tile;      // [n_units] tile of each pair
+  const int32_t *unit_leaf;      // [n_units] leaf of each pair
+  const int32_t *tile_seq;       // [tiles] sequence of each 128-row tile of packed rows
+  const int32_t *tile_row0;      // [tiles] first packed row of the tile
+  const __half *q, *q_lo;        // [M][Hq][hd] rotated queries as an fp16 pair: value and rounding remainder
   const CUtensorMap *map_kv;     // device copy of the 5-d map over the paged KV pool
-  float *attn_o;                 // [M*Hq][splits][hd] unnormalised partial outputs
-  float2 *attn_ml;               // [M*Hq][splits] (running max in the log2 domain, sum)
+  float *attn_o;                 // [M*Hq][n_slots][hd] unnormalised partial outputs
+  float2 *attn_ml;               // [M*Hq][n_slots] (reference maximum in the log2 domain, sum)
+  __nv_bfloat16 *out;            // [planes][out_rows][Hq*hd] merged, normalised rows as bf16 (hi[, lo])
+  int out_rows, planes;
   int *err;                      // device status word
 };
 cudaError_t launch_attention_tc(const AttnTcArgs &a, cudaStream_t st);
+cudaError_t launch_attention_tc_merge(const AttnTcArgs &a, cudaStream_t st);
 
 // per-row argmax over the LM-head tiles, longest accepted prefix per sequence, new lengths
 struct AcceptArgs {

@@ -58,6 +58,7 @@ struct Layout {
   // fused single-kernel path
   uint64_t maps, slab, ss_part, sync, phase_t;
   int n_maps, n_counters, n_phases, max_tiles128, o_tile128_seq, o_tile128_row0;
+  int leaf_len, max_units, o_unit_tile, o_unit_leaf;   // attention leaves (see AttnTcArgs)
   // step io (int32 offsets inside d_in / h_in)
   int o_tokens, o_pos, o_rowseq, o_cu, o_len, o_tile_seq, o_tile_row0, o_btab, in_ints;
   int o_parent, o_anc, o_path, o_uni, o_topk, o_slot;
@@ -122,7 +123,7 @@ void make_layout(const ts_model_config &c, Layout *L) {
   L->h = take(planes * R * d * 2);
   const uint64_t part_cols = std::max<uint64_t>(L->Nqkv, d);
   L->part = take((uint64_t)kMaxSplits * R * part_cols * 4);
-  L->q = take(R * Nq * 2);
+  L->q = take(2 * R * Nq * 2);   // rotated queries, fp16: values [R][Nq], then their rounding remainders [R][Nq]
   L->attn_o = take(R * c.n_q_heads * kMaxAttnSplits * hd * 4);
   L->attn_ml = take(R * c.n_q_heads * kMaxAttnSplits * 8);
   L->attn = take(planes * R * Nq * 2);
@@ -139,6 +140,12 @@ void make_layout(const ts_model_config &c, Layout *L) {
   L->o_tile_seq = itake(L->max_tiles); L->o_tile_row0 = itake(L->max_tiles);
   L->max_tiles128 = c.max_batch * ((c.k_max * G + 127) / 128);
   L->o_tile128_seq = itake(L->max_tiles128); L->o_tile128_row0 = itake(L->max_tiles128);
+  // attention leaf: the smallest power-of-two number of 64-position blocks with at most kMaxAttnSplits leaves in
+  // max_ctx positions.  A constant of the model, NOT of the step: a row's bits must not depend on the step's shape.
+  L->leaf_len = 64;
+  while ((int64_t)L->leaf_len * kMaxAttnSplits < c.max_ctx) L->leaf_len *= 2;
+  L->max_units = L->max_tiles128 * kMaxAttnSplits;
+  L->o_unit_tile = itake(L->max_units); L->o_unit_leaf = itake(L->max_units);
   L->o_parent = itake(c.max_rows); L->o_anc = itake(2 * c.max_rows); L->o_uni = itake(c.max_rows);
   L->o_slot = itake(c.max_rows);
   L->o_btab = itake(c.max_batch * L->pages_per_seq);   // (last: only the used part is copied per step)
@@ -195,11 +202,12 @@ struct ts_model {
   std::vector<int32_t> free_pages;
   std::vector<ts_session *> sessions;   // live sessions over this model (detached on destroy)
   // last staged step
-  int last_B = 0, last_M = 0, last_tiles = 0, last_tiles128 = 0;
+  int last_B = 0, last_M = 0, last_tiles = 0, last_tiles128 = 0, last_units = 0, last_slots = 1;
   uint32_t last_flags = 0;
   bool have_step = false;
   int64_t launches = 0, h2d = 0, d2h = 0;
   bool use_pdl = true;
+  int32_t inject_err = 0;                      // test support: status code the next step is made to report
   bool fused_ok = false, last_fused = false;   // device can run the fused kernel; the staged step uses it
   bool last_tree = false;                      // the staged step verifies a draft tree (not a chain)
   bool last_sample = false;                    // the staged step accepts by speculative sampling
@@ -304,49 +312,6 @@ int pick_splits(const ts_model *m, int n_tiles, int m_chunks, int n_kblocks, boo
   return best;
 }
 
-// KV splits per (row tile, kv head) of the tensor-memory attention kernel.  A unit (one CTA) costs a fixed part plus
-// a part per 64-position block; a step's units are spread over the SMs by the hardware scheduler, so the kernel
-// takes about max(longest unit, all units / slots, waves x shortest unit), and the merge kernel adds a little per
-// split.  One eighth of the SMs is left out of the slots: the kernels that follow launch early and park their
-// prologues (weight prefetch) there, and measured on the 8B step 128 units beat 136 and 144 on 148 SMs.
-int pick_attn_splits(const ts_model *m) {
-  const ts_model_config &c = m->c;
-  const Layout &L = m->L;
-  const int32_t *hi = m->h_in();
-  const int G = c.n_q_heads / c.n_kv_heads;
-  const double c_unit = 5.0, c_blk = 0.9, c_merge = 0.03;   // microseconds, measured on the 8B shape
-  const int slots = std::max(1, m->n_sms - m->n_sms / 8);
-  double est[kMaxAttnSplits + 1], best = 1e30;
-  long n_units[kMaxAttnSplits + 1];
-  for (int s = 1; s <= kMaxAttnSplits; ++s) {
-    double longest = 0.0, total = 0.0, shortest = 1e30;
-    long units = 0;
-    for (int i = 0; i < m->last_B; ++i) {
-      const int k = hi[L.o_cu + i + 1] - hi[L.o_cu + i];
-      const int blocks = (hi[L.o_len + i] + k + 63) / 64;
-      const int tiles = (k * G + 127) / 128;
-      const int live = std::min(s, blocks);                       // splits that hold at least one block
-      const double unit = c_unit + c_blk * ((blocks + live - 1) / live);
-      longest = std::max(longest, unit);
-      shortest = std::min(shortest, unit);
-      total += (double)tiles * c.n_kv_heads * (live * unit + (s - live) * c_unit);
-      units += (long)tiles * c.n_kv_heads * s;
-    }
-    const double waves = (double)((units + slots - 1) / slots);
-    est[s] = std::max(std::max(longest, total / slots), waves * shortest) + c_merge * s;
-    n_units[s] = units;
-    best = std::min(best, est[s]);
-  }
-  // among the counts within 3% of the best estimate: the largest that still runs as one wave (more CTAs stream
-  // more bytes at once), else the smallest
-  int pick = 0;
-  for (int s = kMaxAttnSplits; s >= 1 && !pick; --s)
-    if (est[s] <= 1.03 * best && n_units[s] <= slots) pick = s;
-  for (int s = 1; s <= kMaxAttnSplits && !pick; ++s)
-    if (est[s] <= 1.03 * best) pick = s;
-  return std::max(1, pick);
-}
-
 struct GemmPlan { int splits, kb_per_split; };
 
 ts_status run_gemm(ts_model *m, int epi, const CUtensorMap &tw, const CUtensorMap *ta4, int N, int K, int M,
@@ -386,12 +351,14 @@ ts_status run_step_fused(ts_model *m) {
   a.k_max = c.k_max;
   a.n_attn_tiles = m->last_tiles128;
   {
+    // (from the cached lengths and the model's k_max, not from this step's k, so that the cut does not change with the
+    // number of rows verified)
     int max_total = 0;
     const int32_t *hi = m->h_in();
-    for (int i = 0; i < m->last_B; ++i)
-      max_total = std::max(max_total, hi[L.o_len + i] + (hi[L.o_cu + i + 1] - hi[L.o_cu + i]));
+    for (int i = 0; i < m->last_B; ++i) max_total = std::max(max_total, hi[L.o_len + i] + c.k_max);
     const int nblk = (max_total + 63) / 64;
-    const int s = m->n_sms / std::max(1, c.n_kv_heads * m->last_tiles128);
+    const int G = c.n_q_heads / c.n_kv_heads;
+    const int s = m->n_sms / std::max(1, c.n_kv_heads * m->last_B * ((c.k_max * G + 127) / 128));
     a.attn_splits = std::max(1, std::min(std::min(s, kMaxAttnSplits), nblk));
   }
   a.tile_seq = di + L.o_tile128_seq; a.tile_row0 = di + L.o_tile128_row0;
@@ -457,12 +424,12 @@ ts_status run_step(ts_model *m) {
 
   ts::AttnTcArgs at{};
   at.in = in; at.Hq = c.n_q_heads; at.Hkv = c.n_kv_heads; at.hd = c.head_dim;
-  at.n_tiles = m->last_tiles128;
+  at.leaf_len = L.leaf_len; at.n_units = m->last_units; at.n_slots = m->last_slots;
+  at.unit_tile = di + L.o_unit_tile; at.unit_leaf = di + L.o_unit_leaf;
   at.tile_seq = di + L.o_tile128_seq; at.tile_row0 = di + L.o_tile128_row0;
-  at.q = q; at.map_kv = (const CUtensorMap *)m->WS(L.maps) + (L.n_maps - 1);
+  at.q = q; at.q_lo = q + (size_t)R * Nq; at.map_kv = (const CUtensorMap *)m->WS(L.maps) + (L.n_maps - 1);
   at.attn_o = aa.part_o; at.attn_ml = aa.part_ml; at.err = m->d_out() + L.o_err;
-  if (m->fused_ok) aa.n_splits = pick_attn_splits(m);
-  at.attn_splits = aa.n_splits;
+  at.out = attn; at.out_rows = R; at.planes = m->planes;
   CU_TRY(ts::launch_embed_norm(in, (const __nv_bfloat16 *)m->W(L.embed), (const float *)m->W(L.g1[0]), c.rms_eps,
                                d, x, h, R, m->planes, (unsigned long long *)m->WS(L.amax), m->st));
   m->launched(3);
@@ -476,17 +443,19 @@ ts_status run_step(ts_model *m) {
     ts_status s = run_gemm(m, ts::EPI_PARTIAL, m->tm_qkv[l], m->tm_h, L.Nqkv, d, M, part, nullptr, nullptr, &plan);
     if (s) return s;
     CU_TRY(ts::launch_rope_kv(in, part, plan.splits, R, c.n_q_heads, c.n_kv_heads, c.head_dim, rope, q,
-                              m->k_pages(l), m->v_pages(l), m->st));
+                              q + (size_t)R * Nq, m->k_pages(l), m->v_pages(l), m->st));
     m->launched(4);
     aa.k_pages = m->k_pages(l); aa.v_pages = m->v_pages(l);
     if (m->fused_ok) {   // tensor-memory attention (needs the same device features as the persistent kernel)
       at.layer = l;
       CU_TRY(ts::launch_attention_tc(at, m->st));
+      m->launched(1);
+      CU_TRY(ts::launch_attention_tc_merge(at, m->st));
     } else {
       CU_TRY(ts::launch_attention_split(aa, m->st));
+      m->launched(1);
+      CU_TRY(ts::launch_attention_combine(aa, m->st));
     }
-    m->launched(1);
-    CU_TRY(ts::launch_attention_combine(aa, m->st));
     m->launched(2);
     s = run_gemm(m, ts::EPI_PARTIAL, m->tm_o[l], m->tm_attn, d, Nq, M, part, nullptr, nullptr, &plan);
     if (s) return s;
@@ -588,6 +557,12 @@ ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::ve
           return fail(TS_ERR_ARG, "sequence %d: parent of row %d must be an earlier row (-1 only for row 0)", i, j);
         depth[j] = j == 0 ? 0 : depth[par] + 1;
         anc[j] = (j == 0 ? 0ull : anc[par]) | (1ull << j);
+        // the residual walk of speculative sampling removes a refused child's token from the distribution: two
+        // children of one node carrying the same token would remove it twice
+        if (uniforms)
+          for (int e = 1; e < j; ++e)
+            if ((*parents)[i][e] == par && rows[i][e] == rows[i][j])
+              return fail(TS_ERR_ARG, "sequence %d: rows %d and %d are children of row %d with the same token", i, e, j, par);
       }
       const uint64_t mask = parents ? anc[j] : (j >= 63 ? ~0ull : ((2ull << j) - 1ull));
       hi[L.o_tokens + M + j] = rows[i][j];
@@ -618,12 +593,31 @@ ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::ve
       return hi[L.o_len + a] + (hi[L.o_cu + a + 1] - hi[L.o_cu + a]) > hi[L.o_len + b] + (hi[L.o_cu + b + 1] - hi[L.o_cu + b]);
     });
     int t = 0;
-    for (int i : order)
-      for (int r0 = 0; r0 < (hi[L.o_cu + i + 1] - hi[L.o_cu + i]) * G; r0 += 128) {
+    // (tile, leaf) pairs of the attention kernel: leaf L of a sequence is the absolute positions [L, L + 1) * leaf_len
+    struct Unit { int tile, leaf, nblk; };
+    std::vector<Unit> units;
+    int slots = 1;
+    for (int i : order) {
+      const int k = hi[L.o_cu + i + 1] - hi[L.o_cu + i], total = hi[L.o_len + i] + k;
+      const int n_leaves = (total + L.leaf_len - 1) / L.leaf_len;
+      slots = std::max(slots, n_leaves);
+      for (int r0 = 0; r0 < k * G; r0 += 128) {
         hi[L.o_tile128_seq + t] = i;
         hi[L.o_tile128_row0 + t] = r0;
+        for (int lf = 0; lf < n_leaves; ++lf)
+          units.push_back({t, lf, (std::min(total, (lf + 1) * L.leaf_len) - lf * L.leaf_len + 63) / 64});
         ++t;
       }
+    }
+    // whole leaves first, the shorter last leaves at the end, where they fill the tail of the last wave
+    std::stable_sort(units.begin(), units.end(), [](const Unit &a, const Unit &b) { return a.nblk > b.nblk; });
+    if ((int)units.size() > L.max_units) return fail(TS_ERR_ARG, "internal: %zu attention units exceed %d", units.size(), L.max_units);
+    for (size_t u = 0; u < units.size(); ++u) {
+      hi[L.o_unit_tile + u] = units[u].tile;
+      hi[L.o_unit_leaf + u] = units[u].leaf;
+    }
+    m->last_units = (int)units.size();
+    m->last_slots = slots;
   }
   const bool can_fuse = m->fused_ok && M <= kFusedMaxRows;
   if (c.path == 2 && !can_fuse)
@@ -661,6 +655,13 @@ ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::ve
   m->h2d += (int64_t)in_bytes;
   ts_status st = run_step(m);
   if (st) return st;
+  if (m->inject_err) {
+    // test support (ts_debug_inject_device_error): after the step's last kernel, write the status word an expired
+    // device-side wait would have left; the code below must then treat the step as failed
+    m->h_out()[L.o_err + 1] = m->inject_err;
+    m->inject_err = 0;
+    CU_TRY(cudaMemcpyAsync(m->d_out() + L.o_err, m->h_out() + L.o_err + 1, 4, cudaMemcpyHostToDevice, m->st));
+  }
   const size_t out_bytes = (size_t)L.out_ints * 4;
   CU_TRY(cudaMemcpyAsync(m->h_out(), m->d_out(), out_bytes, cudaMemcpyDeviceToHost, m->st));
   m->d2h += (int64_t)out_bytes;
@@ -959,8 +960,39 @@ ts_status ts_datastore_create(int32_t n_tools, ts_datastore **out) {
   return TS_OK;
 }
 
+ts_status ts_datastore_attach_hidden(ts_datastore *d, void *hidden_dev, int32_t capacity, int32_t d_model) {
+  if (!d) return fail(TS_ERR_ARG, "null argument");
+  if (!hidden_dev) { d->hidden_dev = nullptr; d->hidden_capacity = d->hidden_width = 0; return TS_OK; }
+  if (capacity < d->n_entries() || capacity < 1) return fail(TS_ERR_ARG, "capacity %d below the %d entries held", capacity, d->n_entries());
+  if (d_model < 8 || d_model % 8) return fail(TS_ERR_ARG, "d_model must be a positive multiple of 8");
+  if ((uintptr_t)hidden_dev & 15) return fail(TS_ERR_ARG, "hidden-state matrix must be 16-byte aligned");
+  d->hidden_dev = hidden_dev; d->hidden_capacity = capacity; d->hidden_width = d_model;
+  return TS_OK;
+}
+
+ts_status ts_datastore_add_hidden(ts_datastore *d, ts_model *m, int32_t row, const int32_t *tokens, int32_t n,
+                                  int32_t tool_id) {
+  if (!d || !m || (!tokens && n > 0) || n < 0) return fail(TS_ERR_ARG, "bad argument");
+  if (!d->hidden_dev) return fail(TS_ERR_STATE, "no hidden-state matrix attached (ts_datastore_attach_hidden)");
+  if (d->n_entries() >= d->hidden_capacity) return fail(TS_ERR_STATE, "hidden-state matrix is full (%d rows)", d->hidden_capacity);
+  if (d->hidden_width != m->c.d_model) return fail(TS_ERR_ARG, "hidden states are %d wide, the model %d", d->hidden_width, m->c.d_model);
+  if (!m->have_step || (m->last_flags & TS_FLAG_SKIP_LM_HEAD) || m->last_fused)
+    return fail(TS_ERR_STATE, "the last step left no final hidden state (it must run the LM head on the one-kernel-per-stage path)");
+  if (row < 0 || row >= m->last_M) return fail(TS_ERR_ARG, "row outside the last step");
+  // the first activation plane of the LM head's input IS the hidden state rounded to bf16
+  const size_t wbytes = (size_t)m->c.d_model * 2;
+  CU_TRY(cudaMemcpyAsync((uint8_t *)d->hidden_dev + (size_t)d->n_entries() * wbytes, m->WS(m->L.h) + (size_t)row * wbytes,
+                         wbytes, cudaMemcpyDeviceToDevice, m->st));
+  d->tokens.insert(d->tokens.end(), tokens, tokens + n);
+  d->offset.push_back((int64_t)d->tokens.size());
+  d->tool_of.push_back(tool_id);
+  if (tool_id >= 0 && tool_id < (int32_t)d->freq.size()) ++d->freq[tool_id];
+  return TS_OK;
+}
+
 ts_status ts_datastore_add(ts_datastore *d, const int32_t *tokens, int32_t n, int32_t tool_id) {
   if (!d || (!tokens && n > 0) || n < 0) return fail(TS_ERR_ARG, "bad argument");
+  if (d->hidden_dev) return fail(TS_ERR_STATE, "hidden states are attached: add entries with ts_datastore_add_hidden");
   d->tokens.insert(d->tokens.end(), tokens, tokens + n);
   d->offset.push_back((int64_t)d->tokens.size());
   d->tool_of.push_back(tool_id);
@@ -1176,6 +1208,7 @@ ts_status verify_impl(ts_model *m, ts_session *const *ss, int32_t B, const int32
       for (int j = 0; j < n; ++j) parents[i].push_back(draft_parents[draft_offsets[i] + j]);
     }
   }
+  for (int i = 0; i < B; ++i) ss[i]->last_chunk.clear();   // this step overwrites the rows of the previous one
   ts_status st = stage_and_run(m, ss, B, rows, flags, draft_parents ? &parents : nullptr, uniforms, temperature);
   if (st) return st;
   const Layout &L = m->L;
@@ -1187,6 +1220,7 @@ ts_status verify_impl(ts_model *m, ts_session *const *ss, int32_t B, const int32
     r.k = (int32_t)rows[i].size();
     r.first_row = row;
     ss[i]->last_chunk = rows[i];
+    if (flags & TS_FLAG_SKIP_LM_HEAD) ss[i]->last_chunk.clear();   // no acceptance ran: nothing to commit
     if (!(flags & TS_FLAG_SKIP_LM_HEAD)) {
       r.accept_len = ho[L.o_accept + i];
       r.n_emitted = r.accept_len + 1;
@@ -1340,6 +1374,21 @@ ts_status ts_commit_forced(ts_session *s, const int32_t *emitted, int32_t n) {
   if (!s || !emitted || n < 1) return fail(TS_ERR_ARG, "bad argument");
   if (s->finished) return fail(TS_ERR_STATE, "session is finished");
   if (s->cache_len < 0) return fail(TS_ERR_STATE, "session has no context");
+  if (s->m) {
+    // The cache keeps the pending token and the first n - 1 emitted ids: the K/V rows at those positions were
+    // written by the last verification (after a tree step: the accepted path, moved to consecutive slots), so the
+    // ids must be the ones that step was fed there.  One commit per verification.
+    if (s->last_chunk.empty())
+      return fail(TS_ERR_STATE, "nothing to commit: no verification since the last commit (or since the context was set)");
+    if (n > (int)s->last_chunk.size())
+      return fail(TS_ERR_ARG, "%d ids to commit, but the last verification holds only %zu rows in the cache", n,
+                  s->last_chunk.size());
+    for (int j = 0; j + 1 < n; ++j)
+      if (emitted[j] != s->last_chunk[j + 1])
+        return fail(TS_ERR_ARG, "emitted id %d (%d) is not the id verified at that row (%d)", j, emitted[j],
+                    s->last_chunk[j + 1]);
+    s->last_chunk.clear();
+  }
   const int used = commit_ids(s, emitted, n);
   s->cache_len += used;
   s->pending = emitted[used - 1];
@@ -1381,30 +1430,38 @@ static ts_status kv_transfer(ts_model *m, ts_session *s, int layer, void *k, voi
   }
   const int Hkv = m->c.n_kv_heads, hd = m->c.head_dim;
   const size_t page_elems = (size_t)Hkv * TS_PAGE_SIZE * hd;
-  std::vector<__half> stage(page_elems);
+  const int n_pages = (n_tokens + TS_PAGE_SIZE - 1) / TS_PAGE_SIZE;
+  // one staging image of all pages, so that the copies of a layer are issued back to back and awaited once
+  std::vector<__half> stage((size_t)n_pages * page_elems);
   for (int which = 0; which < 2; ++which) {
     float *host = (float *)(which ? v : k);
     __half *pool = which ? m->v_pages(layer) : m->k_pages(layer);
-    for (int p = 0; p * TS_PAGE_SIZE < n_tokens; ++p) {
-      const int t0 = p * TS_PAGE_SIZE, nt = std::min(TS_PAGE_SIZE, n_tokens - t0);
-      __half *dev = pool + (size_t)s->pages[p] * page_elems;
-      if (to_device) {
-        std::fill(stage.begin(), stage.end(), __float2half(0.f));
-        for (int t = 0; t < nt; ++t)
-          for (int hh = 0; hh < Hkv; ++hh)
-            for (int e = 0; e < hd; ++e) {
-              const float x = host[((size_t)(t0 + t) * Hkv + hh) * hd + e];
-              stage[((size_t)hh * TS_PAGE_SIZE + t) * hd + e] = __float2half_rn(std::min(std::max(x, -65504.f), 65504.f));
-            }
-        CU_TRY(cudaMemcpyAsync(dev, stage.data(), page_elems * 2, cudaMemcpyHostToDevice, m->st));
-        CU_TRY(cudaStreamSynchronize(m->st));
-      } else {
-        CU_TRY(cudaMemcpyAsync(stage.data(), dev, page_elems * 2, cudaMemcpyDeviceToHost, m->st));
-        CU_TRY(cudaStreamSynchronize(m->st));
-        for (int t = 0; t < nt; ++t)
-          for (int hh = 0; hh < Hkv; ++hh)
-            for (int e = 0; e < hd; ++e)
-              host[((size_t)(t0 + t) * Hkv + hh) * hd + e] = __half2float(stage[((size_t)hh * TS_PAGE_SIZE + t) * hd + e]);
+    if (to_device) {
+      std::fill(stage.begin(), stage.end(), __float2half(0.f));
+      for (int t = 0; t < n_tokens; ++t) {
+        __half *pg = stage.data() + (size_t)(t / TS_PAGE_SIZE) * page_elems;
+        for (int hh = 0; hh < Hkv; ++hh) {
+          const float *src = host + ((size_t)t * Hkv + hh) * hd;
+          __half *dst = pg + ((size_t)hh * TS_PAGE_SIZE + (t % TS_PAGE_SIZE)) * hd;
+          for (int e = 0; e < hd; ++e) dst[e] = __float2half_rn(std::min(std::max(src[e], -65504.f), 65504.f));
+        }
+      }
+      for (int p = 0; p < n_pages; ++p)
+        CU_TRY(cudaMemcpyAsync(pool + (size_t)s->pages[p] * page_elems, stage.data() + (size_t)p * page_elems,
+                               page_elems * 2, cudaMemcpyHostToDevice, m->st));
+      CU_TRY(cudaStreamSynchronize(m->st));
+    } else {
+      for (int p = 0; p < n_pages; ++p)
+        CU_TRY(cudaMemcpyAsync(stage.data() + (size_t)p * page_elems, pool + (size_t)s->pages[p] * page_elems,
+                               page_elems * 2, cudaMemcpyDeviceToHost, m->st));
+      CU_TRY(cudaStreamSynchronize(m->st));
+      for (int t = 0; t < n_tokens; ++t) {
+        const __half *pg = stage.data() + (size_t)(t / TS_PAGE_SIZE) * page_elems;
+        for (int hh = 0; hh < Hkv; ++hh) {
+          float *dst = host + ((size_t)t * Hkv + hh) * hd;
+          const __half *src = pg + ((size_t)hh * TS_PAGE_SIZE + (t % TS_PAGE_SIZE)) * hd;
+          for (int e = 0; e < hd; ++e) dst[e] = __half2float(src[e]);
+        }
       }
     }
   }
@@ -1427,6 +1484,7 @@ ts_status ts_debug_set_cache(ts_session *s, int32_t cache_len, int32_t pending) 
   }
   s->cache_len = cache_len;
   s->pending = pending;
+  s->last_chunk.clear();   // whatever was verified before does not describe this context
   return TS_OK;
 }
 
@@ -1495,6 +1553,23 @@ ts_status ts_topk_cosine(ts_model *m, const void *hidden_dev, int32_t n_entries,
   return TS_OK;
 }
 
+ts_status ts_session_retrieve(ts_model *m, ts_session *s, int32_t row, int32_t K, float *scores_dev, int32_t *out_index,
+                              float *out_score, int32_t *out_k) {
+  if (!m || !s || !scores_dev || !out_index || !out_k) return fail(TS_ERR_ARG, "null argument");
+  if (s->m != m) return fail(TS_ERR_ARG, "session belongs to another model");
+  const ts_datastore *d = s->store;
+  if (!d) return fail(TS_ERR_STATE, "session has no datastore");
+  if (!d->hidden_dev) return fail(TS_ERR_STATE, "the datastore has no hidden states attached");
+  if (d->n_entries() < 1) return fail(TS_ERR_STATE, "the datastore is empty");
+  if (d->hidden_width != m->c.d_model) return fail(TS_ERR_ARG, "hidden states are %d wide, the model %d", d->hidden_width, m->c.d_model);
+  if (K < 1) return fail(TS_ERR_ARG, "K must be positive");
+  const int32_t k = std::min(std::min(K, d->n_entries()), 64);
+  ts_status st = ts_topk_cosine(m, d->hidden_dev, d->n_entries(), nullptr, row, k, scores_dev, out_index, out_score);
+  if (st) return st;
+  *out_k = k;
+  return ts_session_set_ranks(s, out_index, k);
+}
+
 ts_status ts_debug_read_buffer(ts_model *m, int32_t which, void *host_out, uint64_t bytes) {
   if (!m || !host_out) return fail(TS_ERR_ARG, "null argument");
   const Layout &L = m->L;
@@ -1541,6 +1616,12 @@ ts_status ts_debug_schedule(int32_t n_tiles, int32_t n_kblocks, int32_t n_ctas, 
     ++n;
   }
   *n_segments = n;
+  return TS_OK;
+}
+
+ts_status ts_debug_inject_device_error(ts_model *m, int32_t code) {
+  if (!m || code <= 0) return fail(TS_ERR_ARG, "bad argument");
+  m->inject_err = code;
   return TS_OK;
 }
 

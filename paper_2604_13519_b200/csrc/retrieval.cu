@@ -54,11 +54,12 @@ cosine_scores_kernel(const __nv_bfloat16 *H, int N, int d, const float *q_dev, c
 
 cudaError_t launch_topk_cosine(const __nv_bfloat16 *H, int N, int d, const float *q_dev, const __nv_bfloat16 *q_planes,
                                int plane_stride, int planes, int K, float *scores, cudaStream_t st) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce once;
+  int dev_ = -1;
+  if (once.needed(&dev_)) {
     cudaError_t e = cudaFuncSetAttribute(cosine_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    once.done(dev_);
   }
   const int per = kCosThreads / 32 * kCosRowsPerWarp;
   cosine_scores_kernel<<<(N + per - 1) / per, kCosThreads, (size_t)d * 4, st>>>(H, N, d, q_dev, q_planes, plane_stride,

@@ -74,22 +74,19 @@ TS_HD int slab_slot_of(int c, int tile, int T, int KB, uint32_t n) {
   return (unit_begin((uint32_t)c, U, active_ctas(U, n)) < (uint32_t)tile * (uint32_t)KB) ? 1 : 0;
 }
 
-// KV positions of one attention split: whole pages, balanced to within one page.
-TS_HD void split_pages(int n_pages, int n_splits, int split, int *p0, int *p1) {
-  *p0 = (int)(((int64_t)split * n_pages) / n_splits);
-  *p1 = (int)(((int64_t)(split + 1) * n_pages) / n_splits);
-}
-
-
-// The same cut in whole 64-position blocks (4 pages), so that only a sequence's last split ends in a partial block.
-// Cut points are rounded up, so a remainder goes to the first splits: the last one, which alone waits for the chunk's
-// own K/V rows and masks its last block, never gets the extra block.
-TS_HD void split_blocks(int n_pages, int n_splits, int split, int *p0, int *p1) {
-  const int nb = (n_pages + 3) >> 2;
-  const int b0 = (int)(((int64_t)split * nb + n_splits - 1) / n_splits);
-  const int b1 = (int)(((int64_t)(split + 1) * nb + n_splits - 1) / n_splits);
-  *p0 = b0 << 2;
-  *p1 = (b1 << 2) < n_pages ? (b1 << 2) : n_pages;
+// KV positions [pos_beg, pos_end) of one attention split.  Only the whole units (2^unit_shift positions: a page or a
+// 64-position block) that lie entirely inside the CACHE -- the `len` positions written by earlier steps -- are cut
+// among the splits, balanced to within one unit with the remainder going to the first splits; the last split also
+// takes everything after them: the cache's ragged tail and the chunk's own rows, up to `end`.  So every split but
+// the last holds whole, fully visible units, only the last one waits for the chunk's K/V and masks, and -- the point
+// of the rule -- the cut depends on the cached length alone: a row's blocks, their order and therefore its result
+// bits do not change with the number of rows verified beside it.
+TS_HD void split_positions(int len, int end, int n_splits, int split, int unit_shift, int *pos_beg, int *pos_end) {
+  const int nu = len >> unit_shift;
+  const int u0 = (int)(((int64_t)split * nu + n_splits - 1) / n_splits);
+  const int u1 = (int)(((int64_t)(split + 1) * nu + n_splits - 1) / n_splits);
+  *pos_beg = u0 << unit_shift;
+  *pos_end = (split == n_splits - 1) ? end : (u1 << unit_shift);
 }
 
 }  // namespace ts

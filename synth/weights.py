@@ -51,11 +51,22 @@ def _gaussian_bf16(seed: int, tid: int, rows: int, cols: int, pool) -> torch.Ten
     return t.view(rows, cols)
 
 
-def make_weights(shape: ModelShape, seed: int = MASTER_SEED, layers=None, with_globals: bool = True):
-    """dict name -> torch.bfloat16 CPU tensor [out][in]; norm gains (fp32, all ones) under
-    'l{l}.g1', 'l{l}.g2', 'gf'.  `layers` restricts generation to some layer indices; the global
-    tensors (embedding, LM head) are produced unless `with_globals` is false.  A tensor's values
-    depend only on (seed, its index in tensor_names), so a model can be generated piece by piece."""
+def _gain(shape: ModelShape, gain_seed, which: int) -> torch.Tensor:
+    """Norm gain vector: ones (the benchmark configurations), or, with a gain seed, 1 + 0.3 N(0,1) so that a test
+    can tell the gain vectors of different layers and norms apart."""
+    if gain_seed is None:
+        return torch.ones(shape.d_model, dtype=torch.float32)
+    g = np.random.Generator(np.random.Philox(key=[(int(gain_seed) << 20) ^ 0x6A17, which]))
+    return torch.from_numpy(1.0 + 0.3 * g.standard_normal(shape.d_model)).to(torch.float32)
+
+
+def make_weights(shape: ModelShape, seed: int = MASTER_SEED, layers=None, with_globals: bool = True,
+                 gain_seed=None):
+    """dict name -> torch.bfloat16 CPU tensor [out][in]; norm gains (fp32; all ones unless `gain_seed`
+    is given, then 1 + 0.3 N(0,1) per element) under 'l{l}.g1', 'l{l}.g2', 'gf'.  `layers` restricts
+    generation to some layer indices; the global tensors (embedding, LM head, final gain) are produced
+    unless `with_globals` is false.  A tensor's values depend only on (seed, its index in tensor_names),
+    so a model can be generated piece by piece."""
     w = {}
     with ThreadPoolExecutor(max_workers=os.cpu_count() or 4) as pool:
         for tid, (name, (r, c)) in enumerate(tensor_names(shape)):
@@ -68,7 +79,7 @@ def make_weights(shape: ModelShape, seed: int = MASTER_SEED, layers=None, with_g
     for l in range(shape.n_layers):
         if layers is not None and l not in layers:
             continue
-        w[f"l{l}.g1"] = torch.ones(shape.d_model, dtype=torch.float32)
-        w[f"l{l}.g2"] = torch.ones(shape.d_model, dtype=torch.float32)
-    w["gf"] = torch.ones(shape.d_model, dtype=torch.float32)
+        w[f"l{l}.g1"] = _gain(shape, gain_seed, 2 * l)
+        w[f"l{l}.g2"] = _gain(shape, gain_seed, 2 * l + 1)
+    w["gf"] = _gain(shape, gain_seed, 2 * shape.n_layers)
     return w

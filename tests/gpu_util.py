@@ -11,9 +11,12 @@ LOGIT_MEAN_ABS = 3e-3
 GAP = 0.05               # integer results may differ only where the oracle's top-2 gap is below this
 
 
+GAIN_SEED = 7            # norm gains 1 + 0.3 N(0,1): a gain vector taken from the wrong layer or norm cannot pass
+
+
 def make_pair(shape, max_batch=1, k_max=8, max_rows=None, max_ctx=1024, max_pages=None, act_split=True,
               weights=None, path=0):
-    w = weights if weights is not None else synth.make_weights(shape)
+    w = weights if weights is not None else synth.make_weights(shape, gain_seed=GAIN_SEED)
     om = oracle.OracleModel(shape, w)
     max_rows = max_rows or max_batch * k_max
     max_pages = max_pages or max_batch * ((max_ctx + 15) // 16)

@@ -187,14 +187,15 @@ def test_retrieval_heavy_batch():
         d.feed_prompt([pending])
         tid, toks = max(inv[10 * i:10 * i + 10], key=lambda e: len(e[1]))
         d.commit(toks[:12], schema.vocab.eos, 10 ** 6)
-        ts.ts_commit_forced(s, toks[:12])     # 12 generated ids: cache 500+.. grows by 12 unverified rows
+        ts.ts_verify(gm, [s], [toks[:11]])    # (a commit is checked against the chunk of the last verification)
+        ts.ts_commit_forced(s, toks[:12])     # 12 generated ids
         want, src = d.draft(63)
         got, gsrc = ts.ts_draft(s, 63)
         assert (got, gsrc) == (want, src) and src == 2
         # the oracle cache must hold the same 12 extra positions: extend it with the same K/V the GPU will see
         sess.append(s); drafts.append(got)
         refs.append((cache, toks[11], want, 500 + 37 * i))
-    # the 12 forced ids were never run through the model; reset both sides to the imported context
+    # the oracle side never saw those 12 rows; reset both sides to the imported context
     for s, (cache, p, want, n) in zip(sess, refs):
         s.set_cache(n, p)
     out = ts.ts_verify(gm, sess, drafts)
@@ -227,6 +228,65 @@ def test_argument_and_capacity_errors():
     assert e.value.code == -3
     res = ts.ts_verify(gm, [s], [[70]])[0]                 # the context is still usable
     assert res.k == 2
+    gm.close()
+
+
+def test_commit_is_checked_against_the_verified_chunk():
+    """A commit moves the cache length over rows the last verification wrote: it is refused without one, twice for
+    the same one, for more ids than rows, and for ids other than the ones those rows were computed from."""
+    shape = synth.SHAPES["tiny"]
+    om, gm = make_pair(shape, k_max=8, max_ctx=128)
+    s = ts.Session(gm, None, None)
+    ts.ts_prefill(gm, s, [70, 71, 72, 73])
+    with pytest.raises(ts.TsError) as e:
+        ts.ts_commit_forced(s, [80])                       # nothing verified yet
+    assert e.value.code == -2
+    draft = [90, 91, 92]
+    res = ts.ts_verify(gm, [s], [draft])[0]
+    with pytest.raises(ts.TsError) as e:
+        ts.ts_commit_forced(s, [90, 91, 92, 93, 94])       # 5 ids, 4 rows
+    assert e.value.code == -1
+    with pytest.raises(ts.TsError) as e:
+        ts.ts_commit_forced(s, [90, 99, 5])                # row 2 was fed 91, not 99
+    assert e.value.code == -1
+    assert s.state().cache_len == 3                        # the refused calls changed nothing
+    ts.ts_commit_forced(s, [90, 91, 5])                    # two verified drafts kept, a free last id
+    assert (s.state().cache_len, s.state().pending) == (6, 5)
+    with pytest.raises(ts.TsError) as e:
+        ts.ts_commit(s, res)                               # the same verification a second time
+    assert e.value.code == -2
+    res = ts.ts_verify(gm, [s], [[]])[0]
+    ts.ts_commit(s, res)
+    assert s.state().cache_len == 7
+    s.set_cache(3, 73)
+    with pytest.raises(ts.TsError) as e:
+        ts.ts_commit(s, res)                               # the context was replaced since
+    assert e.value.code == -2
+    gm.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_device_timeout_is_reported_and_survived(path):
+    """The host's handling of an expired device-side wait, without making the GPU wait: the status word is written on
+    the stream after the step's last kernel (no kernel sees it).  The step fails with TS_ERR_DEVICE_TIMEOUT, the
+    session is untouched, and the next step is parity-green again."""
+    shape = synth.SHAPES["1b-2l"]
+    om, gm = make_pair(shape, k_max=16, max_ctx=512, path=path)
+    cache, s, pending = synthetic_context(shape, om, gm, 200)
+    draft = _rand_draft(shape.vocab, 9, 31)
+    ref = om.verify(pending, draft, cache.clone(), want_logits=True)
+    check_step(ts.ts_verify(gm, [s], [draft])[0], gm.read_logits(0, 10), ref, "before")
+    gm.inject_device_error(3)
+    with pytest.raises(ts.TsError) as e:
+        ts.ts_verify(gm, [s], [draft])
+    assert e.value.code == -6 and "code 3" in str(e.value)
+    assert (s.state().cache_len, s.state().pending) == (200, pending)
+    with pytest.raises(ts.TsError) as e:
+        ts.ts_commit_forced(s, ref["emitted"])            # a failed step leaves nothing to commit
+    assert e.value.code == -2
+    res = ts.ts_verify(gm, [s], [draft])[0]               # the word was cleared: the same step again, clean
+    check_step(res, gm.read_logits(0, 10), ref, "after the reported timeout")
+    ts.ts_commit(s, res)
     gm.close()
 
 

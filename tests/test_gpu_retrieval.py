@@ -66,3 +66,88 @@ def test_query_from_the_last_step_is_the_final_hidden_state():
     with pytest.raises(ts.TsError):
         ts.ts_topk_cosine(gm, H.cuda(), 0)
     gm.close()
+
+
+def test_algorithm_1_retrieval_end_to_end():
+    """Algorithm 1 driven from the library's own datastore H = {(h_j, y_j)}: N historical invocations inserted with the
+    hidden state of their question's last token (device-to-device, into a matrix the test owns); then, per query,
+    h_x -> Top-10 -> I_k installed on the session -> drafts (the schema draft's tool guess and the suffix match, both
+    restricted to I_k) equal to the oracle's, which ranks its own float64 hidden states rounded to bf16."""
+    shape = synth.SHAPES["tiny"]
+    om, gm = make_pair(shape, k_max=16, max_ctx=256, path=1)
+    schema = synth.make_schema(shape.vocab, 8)
+    inv = synth.make_datastore(schema, 40)
+    sc = ts.Schema(schema.vocab, schema.tools)
+    questions = [synth.make_context(shape.vocab, 20 + i % 7, stream=100 + i) for i in range(len(inv))]
+    H = torch.zeros(len(inv) + 2, shape.d_model, dtype=torch.bfloat16, device="cuda")
+    st_c, st_o, hs_o = ts.Datastore(len(schema.tools)), oracle.Datastore(len(schema.tools)), oracle.HiddenStore()
+    with pytest.raises(ts.TsError) as e:
+        st_c.add_hidden(gm, 0, inv[0][1], inv[0][0])           # nothing attached yet
+    assert e.value.code == -2
+    st_c.attach_hidden(H)
+
+    def final_hidden(prompt):
+        cache, pending = oracle.prefill(om, prompt)
+        probe = {}
+        om.forward_chunk([pending], cache, probe=probe)
+        return oracle.rmsnorm(probe["x_final"], om.w["gf"], shape.rms_eps)[0]
+
+    for (tid, toks), q in zip(inv, questions):
+        s = ts.Session(gm, None, None)
+        ts.ts_prefill(gm, s, q)
+        ts.ts_verify(gm, [s], [[]])                             # row 0 = the question's last token
+        st_c.add_hidden(gm, 0, toks, tid)
+        s.close()
+        st_o.add(toks, tid)
+        hs_o.add(final_hidden(q))
+    with pytest.raises(ts.TsError) as e:
+        st_c.add(inv[0][1], inv[0][0])                          # an entry without its hidden state
+    assert e.value.code == -2
+    torch.cuda.synchronize()
+    want_rows = torch.stack(hs_o.rows).float()
+    got_rows = H[:len(inv)].float().cpu()
+    assert (got_rows - want_rows).abs().max() <= 2e-2 * want_rows.abs().max()
+    assert float(H[len(inv):].abs().max()) == 0.0              # rows of entries that do not exist were not written
+
+    exact = 0
+    for trial, j_star in enumerate((5, 17, 33, 0)):
+        q = list(questions[j_star])
+        q[2 + trial] = (q[2 + trial] + 1) % shape.vocab         # the stored question, one token changed
+        s = ts.Session(gm, sc, st_c)
+        ts.ts_prefill(gm, s, q)
+        ts.ts_verify(gm, [s], [[]])
+        idx, score = ts.ts_session_retrieve(gm, s, 10)
+        h_x = final_hidden(q)
+        ref_idx, ref_score = hs_o.retrieve(h_x, 10)
+        assert idx[0] == ref_idx[0] == j_star
+        assert np.allclose(score, ref_score, rtol=0, atol=1e-2)
+        s_all = oracle.cosine_scores(torch.stack(hs_o.rows), h_x)
+        for r in range(10):       # a rank may differ only between entries whose oracle scores nearly tie
+            assert idx[r] == ref_idx[r] or abs(float(s_all[idx[r]]) - ref_score[r]) < 1e-2, (r, idx, ref_idx)
+        exact += idx == ref_idx
+        s.set_ranks(ref_idx)                                    # (same candidate order on both sides from here on)
+        d = oracle.Drafter(schema, st_o, ranks=ref_idx)
+        d.feed_prompt(q)
+        # the schema draft: the tool is guessed from the best-ranked candidate
+        assert ts.ts_draft(s, 15) == d.draft(15)
+        # the suffix match, restricted to I_k: continue with the opening of the third-ranked invocation
+        toks = st_o.entries[ref_idx[2]]
+        ts.ts_verify(gm, [s], [toks[:7]])
+        ts.ts_commit_forced(s, toks[:8])
+        d.commit(toks[:8], schema.vocab.eos, 10 ** 6)
+        got, want = ts.ts_draft(s, 15), d.draft(15)
+        assert got == want and want[1] == 2 and len(want[0]) > 0
+        # an invocation outside I_k is never matched, although the whole store would match it
+        outside = next(c for c in range(len(inv)) if c not in ref_idx and len(st_o.entries[c]) > 9)
+        s2 = ts.Session(gm, sc, st_c)
+        ts.ts_prefill(gm, s2, q)
+        ts.ts_verify(gm, [s2], [st_o.entries[outside][:7]])
+        s2.set_ranks(ref_idx)
+        ts.ts_commit_forced(s2, st_o.entries[outside][:8])
+        d2 = oracle.Drafter(schema, st_o, ranks=ref_idx)
+        d2.feed_prompt(q)
+        d2.commit(st_o.entries[outside][:8], schema.vocab.eos, 10 ** 6)
+        assert ts.ts_draft(s2, 15) == d2.draft(15)
+        s.close(); s2.close()
+    assert exact >= 3
+    gm.close()

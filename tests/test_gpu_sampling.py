@@ -109,6 +109,10 @@ def test_sampled_batch_and_errors():
         ts.ts_verify_sampled(gm, [s0], [d0], 0.0, [0.5] * 4)             # temperature must be positive
     with pytest.raises(ts.TsError):
         ts.ts_verify_sampled(gm, [s0], [d0], 1.0, [0.5, 1.0, 0.1, 0.2])  # a uniform outside [0, 1)
+    with pytest.raises(ts.TsError) as e:                                   # two children of the root with one token:
+        ts.ts_verify_tree_sampled(gm, [s0], [[100, 101, 100]], [[0, 1, 0]], 1.0, [0.5] * 4)   # its weight would be removed twice
+    assert e.value.code == -1 and "same token" in str(e.value)
+    ts.ts_verify_tree(gm, [s0], [[100, 101, 100]], [[0, 1, 0]])           # (greedy acceptance takes the first of them)
     gm.close()
 
 

@@ -1,25 +1,29 @@
-"""ts_attention_static against ts_verify's own attention stage.
+"""ts_attention_static against the oracle's attention and against ts_verify's own attention stage.
 
 Some users of the library cannot allocate device memory (a plugin inside a server whose memory pool
 belongs to the host application, code running under a fixed memory budget), so they cannot provide
 the workspace a model needs.  ts_attention_static keeps its scratch in an array inside the library
 image instead.  This test feeds it what ts_verify's attention stage saw in the last layer of a step
 (the rotated queries and the layer's cache, re-paged under a shuffled block table in buffers the test
-owns) and requires the same output, on two different problems in a row so that whatever the first
-call leaves in the shared scratch must not leak into the second.
+owns) and requires (a) the oracle's attention of the same queries, keys and values, (b) the output of
+ts_verify's attention stage, a different kernel, on two different problems in a row so that whatever
+the first call leaves in the shared scratch must not leak into the second, and (c) that the device's
+free memory and torch's allocation count are the same before and after the call.
 
 Collected last on purpose: a run that stops at the first failure has then run every other test.
 """
 import pytest
 import torch
 
+import oracle
 import synth
 import paper_2604_13519_b200 as ts
 from gpu_util import make_pair, synthetic_context
 
 pytestmark = pytest.mark.gpu
 
-TOL = 1e-3     # on attention outputs of magnitude ~0.1 (the two paths normally agree bit for bit)
+TOL = 1e-3         # against ts_verify's attention stage, on outputs of magnitude ~0.1
+ORACLE_TOL = 2e-3  # against the float64 oracle: softmax weights carry 11 bits (fp16), values are N(0,1)
 
 
 def _own_pages(shape, sess, layer, n_tokens, seed):
@@ -37,21 +41,34 @@ def _own_pages(shape, sess, layer, n_tokens, seed):
     return kp.cuda(), vp.cuda(), table.view(1, -1).cuda()
 
 
-def _compare(shape, gm, sess, ctx, k, seed):
+def _compare(shape, gm, sess, ctx, k, seed, first_call=False):
     R = (gm.cfg.max_rows + 127) // 128 * 128
     Nq = shape.n_q_heads * shape.head_dim
     q = gm.read_buffer(2)[:k].cuda().contiguous()                       # fp16 [k][Nq], last layer
     want = gm.read_buffer(3).float().sum(0)[:k]                         # hi + lo planes
     kp, vp, table = _own_pages(shape, sess, shape.n_layers - 1, ctx + k, seed)
     out = torch.zeros(2, R, Nq, dtype=torch.bfloat16, device="cuda")
-    keep = ts.ts_attention_static(q, kp, vp, table, [0, k], [ctx], shape.n_q_heads, shape.n_kv_heads,
-                                  shape.head_dim, out)
+    d_cu = torch.tensor([0, k], dtype=torch.int32, device="cuda")
+    d_len = torch.tensor([ctx], dtype=torch.int32, device="cuda")
+    # every input exists now: the call itself must not take device memory, from the driver or from torch's pool
     torch.cuda.synchronize()
-    del keep
+    free0, alloc0, resv0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    ts.ts_attention_static(q, kp, vp, table, [0, k], [ctx], shape.n_q_heads, shape.n_kv_heads, shape.head_dim, out,
+                           cu_rows_dev=d_cu, seq_len_dev=d_len)
+    torch.cuda.synchronize()
+    # (the driver loads a kernel's code at its first launch in a process, which can move the free-memory figure once)
+    assert first_call or torch.cuda.mem_get_info()[0] == free0
+    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == resv0
     got = out.float().sum(0)[:k].cpu()
     err = (got - want).abs().max().item()
     assert want.abs().max().item() > 1e-3                               # the reference is not trivially zero
-    assert err <= TOL, f"ctx={ctx} k={k}: max abs difference {err:.3e}"
+    assert err <= TOL, f"ctx={ctx} k={k}: max abs difference from ts_verify's attention {err:.3e}"
+    # the oracle's attention over the same fp16 queries and the cache rows as exported (chunk rows included)
+    kk, vv = sess.export_kv(shape.n_layers - 1, ctx + k)
+    ref = oracle.attention(q.cpu().double().view(k, shape.n_q_heads, shape.head_dim), kk.double(), vv.double(),
+                           torch.arange(k) + ctx, torch.arange(ctx + k)).reshape(k, Nq)
+    err_o = (got.double() - ref).abs().max().item()
+    assert err_o <= ORACLE_TOL, f"ctx={ctx} k={k}: max abs difference from the oracle {err_o:.3e}"
 
 
 def test_static_attention_matches_verify_twice():
@@ -61,7 +78,7 @@ def test_static_attention_matches_verify_twice():
     cache, sess, pending = synthetic_context(shape, om, gm, 700)
     draft = [100 + 3 * j for j in range(31)]
     ts.ts_verify(gm, [sess], [draft])
-    _compare(shape, gm, sess, 700, 32, seed=1)
+    _compare(shape, gm, sess, 700, 32, seed=1, first_call=True)
     # second problem, right after: shorter context, ragged chunk, fewer splits
     sess2_cache, sess2, _ = synthetic_context(shape, om, gm, 85, stream=1)
     draft2 = [200 + 5 * j for j in range(6)]
