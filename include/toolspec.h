@@ -382,6 +382,13 @@ ts_status ts_debug_phase_clocks(ts_model *m, uint64_t *out, int32_t cap, int32_t
  * Host only; for testing the index arithmetic without a GPU. */
 ts_status ts_debug_schedule(int32_t n_tiles, int32_t n_kblocks, int32_t n_ctas, int32_t cta, int32_t cap,
                             int32_t *segments, int32_t *n_segments);
+/* Timeline of the last step under its normal launch configuration (programmatic dependent launch on, kernels
+ * overlapping as in production): the step is run once more with every kernel leaving four device-clock stamps
+ * (nanoseconds of the GPU's global timer): earliest CTA start, earliest and latest return from the dependency wait,
+ * latest CTA end.  stamps: host, 4 values per launch in launch order; classes: host, the launch's class as in
+ * ts_profile_step; at most cap launches are written, *n_launches receives their number.  A launch without stamps
+ * (acceptance, Top-K, sampling) reports ~0, ~0, 0, 0.  One-kernel-per-stage path only.  Synchronises the stream. */
+ts_status ts_debug_timeline(ts_model *m, uint64_t *stamps, int32_t *classes, int32_t cap, int32_t *n_launches);
 /* Make the NEXT step (ts_verify*, ts_prefill chunk) report `code` (> 0) in its device status word, as a bounded
  * device-side wait that expired would: the word is written on the model's stream after the step's last kernel and
  * before the results are read back, so no kernel sees it and nothing is left waiting.  That step then fails with

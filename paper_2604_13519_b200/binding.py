@@ -126,6 +126,7 @@ _SIGNATURES = {
     "ts_read_logits": [_P, C.c_int32, C.c_int32, C.POINTER(C.c_float)],
     "ts_debug_read_buffer": [_P, C.c_int32, _P, C.c_uint64],
     "ts_debug_inject_device_error": [_P, C.c_int32],
+    "ts_debug_timeline": [_P, C.POINTER(C.c_uint64), _I32P, C.c_int32, _I32P],
     "ts_model_counters": [_P, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64)],
     "ts_attention_static": [C.POINTER(ts_attention_args), _P],
     "ts_debug_phase_clocks": [_P, C.POINTER(C.c_uint64), C.c_int32, _I32P],
@@ -308,6 +309,23 @@ class Model:
         buf = (C.c_uint64 * 4096)()
         _check(lib().ts_debug_phase_clocks(self.h, buf, 4096, C.byref(n)))
         return np.array(buf[:3 * n.value], dtype=np.uint64).reshape(3, n.value)
+
+    def timeline(self):
+        """[(class name, start, first wait return, last wait return, end)] per launch of the last step re-run under
+        its normal launch configuration; times in microseconds from the first kernel's start."""
+        cap = 9 * self.shape.n_layers + 16
+        st = (C.c_uint64 * (4 * cap))()
+        cls = (C.c_int32 * cap)()
+        n = C.c_int32(0)
+        _check(lib().ts_debug_timeline(self.h, st, cls, cap, C.byref(n)))
+        rows, t0 = [], None
+        for i in range(min(n.value, cap)):
+            v = [st[4 * i + j] for j in range(4)]
+            if v[3] == 0:
+                continue
+            t0 = v[0] if t0 is None else t0
+            rows.append((KERNEL_CLASSES[cls[i]],) + tuple((x - t0) / 1e3 for x in v))
+        return rows
 
     def inject_device_error(self, code: int):
         """Test support: the next step reports `code` in its device status word (see toolspec.h)."""

@@ -311,6 +311,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
+  if (threadIdx.x == 0) stamp_min(a.stamp);
   pdl_launch_dependents();   // (this CTA holds its tensor memory; the dependent waits for this kernel's end anyway)
   // The step's integer inputs were copied in before the step's first kernel started, so they may be read here.
   const AttnUnit t = attn_unit_info(a, (int)blockIdx.x);
@@ -395,6 +396,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
     // ---------------------------------------------------------------- workers
     uint32_t blk = 0;
     pdl_wait();   // the rotated queries come from the previous kernel
+    if (threadIdx.x == kWorkerWarp0 * 32) stamp_waited(a.stamp);
     attn_unit_workers<HD>(a, ctl, t, smem, tmem_base, warp & 3, lane, (int)threadIdx.x - kWorkerWarp0 * 32, blk, err);
   }
   tc_fence_before();
@@ -403,6 +405,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
   }
+  if (threadIdx.x == 0 && a.stamp) stamp_max(a.stamp + 3);
 }
 
 // grid = (M, Hq), hd threads: add the leaves of one (row, query head) and emit the normalised row as bf16 (hi[, lo]).
@@ -412,12 +415,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
 // order.  NS = compile-time bound on the number of leaves.
 template <int NS>
 __global__ void attn_merge_kernel(const AttnTcArgs a) {
+  if (threadIdx.x == 0) stamp_min(a.stamp_merge);
   pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
-  pdl_wait();
   const int m = blockIdx.x, h = blockIdx.y, d = threadIdx.x, lane = threadIdx.x & 31;
-  const int seq = a.in.row_seq[m];
-  const int total = a.in.seq_len[seq] + (a.in.cu_rows[seq + 1] - a.in.cu_rows[seq]);
-  const int nl = (total + a.leaf_len - 1) / a.leaf_len;
+  const int nl = a.in.row_leaves[m];   // (a step input, on the device before the step's first kernel)
+  pdl_wait();
+  if (threadIdx.x == 0) stamp_waited(a.stamp_merge);
   const size_t base = ((size_t)m * a.Hq + h) * a.n_slots;
   const float2 ml = lane < nl ? a.attn_ml[base + lane] : make_float2(-INFINITY, 0.f);
   float t[NS];
@@ -442,6 +445,7 @@ __global__ void attn_merge_kernel(const AttnTcArgs a) {
   const size_t ld = (size_t)a.Hq * a.hd;
   a.out[(size_t)m * ld + col] = hi;
   if (a.planes == 2) a.out[((size_t)a.out_rows + m) * ld + col] = lo;
+  if (threadIdx.x == 0 && a.stamp_merge) stamp_max(a.stamp_merge + 3);
 }
 
 template <typename K>

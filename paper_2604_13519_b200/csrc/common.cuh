@@ -105,6 +105,15 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const void *tmap, int 
       : "memory");
 }
 
+// ---- optional device-clock stamps of a launch (timeline of a step under programmatic dependent launch) -------------
+// stamp[0] = earliest CTA start, [1] = earliest return from the dependency wait, [2] = latest return from it,
+// [3] = latest CTA end; nanoseconds of the global timer.  A null pointer (the normal case) costs one branch.
+__device__ __forceinline__ void stamp_min(unsigned long long *p) { if (p) atomicMin(p, global_timer_ns()); }
+__device__ __forceinline__ void stamp_max(unsigned long long *p) { if (p) atomicMax(p, global_timer_ns()); }
+__device__ __forceinline__ void stamp_waited(unsigned long long *p) {
+  if (p) { const unsigned long long t = global_timer_ns(); atomicMin(p + 1, t); atomicMax(p + 2, t); }
+}
+
 // ---- programmatic dependent launch -------------------------------------------------------------------
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() {

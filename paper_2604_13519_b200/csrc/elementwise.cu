@@ -21,22 +21,33 @@ __device__ __forceinline__ float block_sum(float v, float *red) {
   return t;
 }
 
-// One CTA per row, one float4 of the row per thread and pass (d/4 threads, at most 1024), so that the
-// loads of all split-K slabs are in flight together.  MODE 0: x = embedding row (and the row's argmax
-// slot is cleared for the LM-head epilogue).  MODE 1: x += sum of partial slabs.
+// One CTA per row.  MODE 0: x = embedding row (and the row's argmax slot is cleared for the LM-head epilogue).
+// MODE 1: x += sum of the split-K partial slabs of the preceding projection.  Then h = x * rsqrt(mean(x^2) + eps) * g
+// as bf16 (hi[, lo]) planes.  A thread owns one float4 of the row (d / 4 threads; wider rows loop), issues the loads it
+// needs together -- the gain before the dependency wait, the residual and the slabs after it -- and keeps its sum in
+// registers across the block reduction, so that nothing is read back.  (Spreading a row over a cluster of CTAs with
+// the sums of squares exchanged through distributed shared memory was measured and is not faster: the kernel's time
+// is the latency of its first access after the wait and of its exit, not the bytes one SM pulls from L2.)
 template <int MODE>
 __global__ void __launch_bounds__(kNormMaxThreads)
 norm_kernel(const int32_t *tokens, const __nv_bfloat16 *embed, const float *part, int n_splits, int part_rows,
             const float *gain, float eps, int d, float *x, __nv_bfloat16 *h, int h_rows, int planes,
-            unsigned long long *amax) {
+            unsigned long long *amax, unsigned long long *stamp) {
   __shared__ float red[32];
+  if (threadIdx.x == 0) stamp_min(stamp);
   pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
-  pdl_wait();
   const int m = blockIdx.x;
+  const int c0 = threadIdx.x * 4;
+  const bool one_pass = d <= (int)blockDim.x * 4;   // the whole row lives in the CTA's registers
+  float4 gn = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (c0 < d) gn = *reinterpret_cast<const float4 *>(gain + c0);   // (weights do not depend on the previous kernel)
+  pdl_wait();
+  if (threadIdx.x == 0) stamp_waited(stamp);
   float *xr = x + (size_t)m * d;
   float ss = 0.f;
+  float4 keep = make_float4(0.f, 0.f, 0.f, 0.f);
   if (MODE == 0 && threadIdx.x == 0) amax[m] = 0ull;
-  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
+  for (int c = c0; c < d; c += blockDim.x * 4) {
     float4 v;
     if (MODE == 0) {
       const __nv_bfloat16 *e = embed + (size_t)tokens[m] * d + c;
@@ -45,34 +56,46 @@ norm_kernel(const int32_t *tokens, const __nv_bfloat16 *embed, const float *part
       const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162 *>(&raw.y);
       v = make_float4(__low2float(a), __high2float(a), __low2float(b), __high2float(b));
     } else {
+      // all loads first (a 1024-thread CTA has 64 registers per thread: nine slabs -- what the projections of the
+      // large shapes use -- and the residual fit; further slabs take a second round), then the sum in slab order
+      constexpr int kFirst = 9;
+      float4 p[kFirst];
       v = *reinterpret_cast<const float4 *>(xr + c);
-      // two batches of six independent loads (a 1024-thread CTA has 64 registers per thread)
 #pragma unroll
-      for (int s0 = 0; s0 < kNormMaxSplits; s0 += 6) {
-        float4 p[6];
+      for (int s = 0; s < kFirst; ++s)
+        if (s < n_splits) p[s] = *reinterpret_cast<const float4 *>(part + ((size_t)s * part_rows + m) * d + c);
 #pragma unroll
-        for (int s = 0; s < 6; ++s)
-          if (s0 + s < n_splits) p[s] = *reinterpret_cast<const float4 *>(part + ((size_t)(s0 + s) * part_rows + m) * d + c);
+      for (int s = 0; s < kFirst; ++s)
+        if (s < n_splits) { v.x += p[s].x; v.y += p[s].y; v.z += p[s].z; v.w += p[s].w; }
+      if (n_splits > kFirst) {
 #pragma unroll
-        for (int s = 0; s < 6; ++s)
-          if (s0 + s < n_splits) { v.x += p[s].x; v.y += p[s].y; v.z += p[s].z; v.w += p[s].w; }
+        for (int s = kFirst; s < kNormMaxSplits; ++s)
+          if (s < n_splits) p[s - kFirst] = *reinterpret_cast<const float4 *>(part + ((size_t)s * part_rows + m) * d + c);
+#pragma unroll
+        for (int s = kFirst; s < kNormMaxSplits; ++s)
+          if (s < n_splits) { v.x += p[s - kFirst].x; v.y += p[s - kFirst].y; v.z += p[s - kFirst].z; v.w += p[s - kFirst].w; }
       }
     }
     *reinterpret_cast<float4 *>(xr + c) = v;
+    keep = v;
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   const float tot = block_sum(ss, red);
   const float r = rsqrtf(tot / (float)d + eps);
-  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
-    const float4 v = *reinterpret_cast<const float4 *>(xr + c);
-    const float4 gn = *reinterpret_cast<const float4 *>(gain + c);
-    const float o[4] = {v.x * r * gn.x, v.y * r * gn.y, v.z * r * gn.z, v.w * r * gn.w};
+  for (int c = c0; c < d; c += blockDim.x * 4) {
+    float4 v = keep, gg = gn;
+    if (!one_pass) {
+      v = *reinterpret_cast<const float4 *>(xr + c);
+      gg = *reinterpret_cast<const float4 *>(gain + c);
+    }
+    const float o[4] = {v.x * r * gg.x, v.y * r * gg.y, v.z * r * gg.z, v.w * r * gg.w};
     __nv_bfloat16 hi[4], lo[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) split_bf16(o[j], hi[j], lo[j]);
     *reinterpret_cast<uint2 *>(h + (size_t)m * d + c) = *reinterpret_cast<uint2 *>(hi);
     if (planes == 2) *reinterpret_cast<uint2 *>(h + ((size_t)h_rows + m) * d + c) = *reinterpret_cast<uint2 *>(lo);
   }
+  if (stamp) { __syncthreads(); if (threadIdx.x == 0) stamp_max(stamp + 3); }
 }
 
 template <typename K, typename... Args>
@@ -96,15 +119,16 @@ cudaError_t launch_embed_norm(const StepIn &in, const __nv_bfloat16 *embed, cons
                               int d, float *x, __nv_bfloat16 *h, int h_rows, int planes,
                               unsigned long long *amax, cudaStream_t st) {
   return launch_pdl(norm_kernel<0>, dim3(in.M), dim3(norm_threads(d)), 0, st, in.tokens, embed,
-                    (const float *)nullptr, 0, 0, gain, eps, d, x, h, h_rows, planes, amax);
+                    (const float *)nullptr, 0, 0, gain, eps, d, x, h, h_rows, planes, amax, (unsigned long long *)nullptr);
 }
 
 cudaError_t launch_add_norm(int M, int d, const float *part, int n_splits, int part_rows, const float *gain,
-                            float eps, float *x, __nv_bfloat16 *h, int h_rows, int planes, cudaStream_t st) {
+                            float eps, float *x, __nv_bfloat16 *h, int h_rows, int planes, cudaStream_t st,
+                            unsigned long long *stamp) {
   if (n_splits > kNormMaxSplits) return cudaErrorInvalidValue;
   return launch_pdl(norm_kernel<1>, dim3(M), dim3(norm_threads(d)), 0, st, (const int32_t *)nullptr,
                     (const __nv_bfloat16 *)nullptr, part, n_splits, part_rows, gain, eps, d, x, h, h_rows,
-                    planes, (unsigned long long *)nullptr);
+                    planes, (unsigned long long *)nullptr, stamp);
 }
 
 __device__ __forceinline__ __half to_half_sat(float x) {
@@ -112,24 +136,33 @@ __device__ __forceinline__ __half to_half_sat(float x) {
 }
 
 // grid = (M, Hq + 2*Hkv); one CTA of hd/2 threads per (row, head).  Thread i handles the rotary pair
-// (i, i + hd/2) of q or k heads, or elements (i, i + hd/2) of a v head.
+// (i, i + hd/2) of q or k heads, or elements (i, i + hd/2) of a v head.  Every load is issued before the first use
+// (the slabs, the row's position, sequence and slot): the kernel is two round trips to L2, not one per slab.
 __global__ void rope_kv_kernel(StepIn in, const float *part, int n_splits, int part_rows, int Hq, int Hkv, int hd,
-                               const float2 *rope_tab, __half *q_out, __half *q_lo_out, __half *k_pages, __half *v_pages) {
+                               const float2 *rope_tab, __half *q_out, __half *q_lo_out, __half *k_pages, __half *v_pages,
+                               unsigned long long *stamp) {
+  if (threadIdx.x == 0) stamp_min(stamp);
   pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
-  pdl_wait();
   const int m = blockIdx.x, head = blockIdx.y, i = threadIdx.x, half = hd >> 1;
   const int N = (Hq + 2 * Hkv) * hd;
+  // the step's integer inputs were copied in before the step's first kernel: they may be read before the wait
+  const int pos = in.pos[m], seq = in.row_seq[m], slot = in.slot[m];
+  const int page = (head >= Hq) ? in.block_tab[(size_t)seq * in.pages_per_seq + (slot >> 4)] : 0;
+  float2 cs = make_float2(1.f, 0.f);
+  if (head < Hq + Hkv) cs = rope_tab[(size_t)pos * half + i];
+  pdl_wait();
+  if (threadIdx.x == 0) stamp_waited(stamp);
   // the QKV weight rows are stored with rotary partners adjacent: feature 2i = element i, 2i+1 = element i + hd/2
   const int col = head * hd + 2 * i;
+  float2 p[kNormMaxSplits];
+#pragma unroll
+  for (int s = 0; s < kNormMaxSplits; ++s)
+    if (s < n_splits) p[s] = *reinterpret_cast<const float2 *>(part + ((size_t)s * part_rows + m) * N + col);
   float a = 0.f, b = 0.f;
-  for (int s = 0; s < n_splits; ++s) {
-    const float2 ab = *reinterpret_cast<const float2 *>(part + ((size_t)s * part_rows + m) * N + col);
-    a += ab.x;
-    b += ab.y;
-  }
-  const int pos = in.pos[m];
+#pragma unroll
+  for (int s = 0; s < kNormMaxSplits; ++s)
+    if (s < n_splits) { a += p[s].x; b += p[s].y; }
   if (head < Hq + Hkv) {
-    const float2 cs = rope_tab[(size_t)pos * half + i];
     const float ra = a * cs.x - b * cs.y;
     const float rb = b * cs.x + a * cs.y;
     a = ra; b = rb;
@@ -146,22 +179,20 @@ __global__ void rope_kv_kernel(StepIn in, const float *part, int n_splits, int p
       q_lo_out[qo + i + half] = __float2half_rn(fabsf(b) <= 65504.f ? b - __half2float(hb) : 0.f);
     }
   } else {
-    const int seq = in.row_seq[m];
-    const int slot = in.slot[m];
-    const int page = in.block_tab[(size_t)seq * in.pages_per_seq + (slot >> 4)];
     const bool is_k = head < Hq + Hkv;
     const int kh = is_k ? head - Hq : head - Hq - Hkv;
     __half *dst = (is_k ? k_pages : v_pages) + (((size_t)page * Hkv + kh) * 16 + (slot & 15)) * hd;
     dst[i] = to_half_sat(a);
     dst[i + half] = to_half_sat(b);
   }
+  if (threadIdx.x == 0) stamp_max(stamp ? stamp + 3 : nullptr);
 }
 
 cudaError_t launch_rope_kv(const StepIn &in, const float *part, int n_splits, int part_rows, int Hq, int Hkv,
                            int hd, const float2 *rope_tab, __half *q_out, __half *q_lo_out, __half *k_pages,
-                           __half *v_pages, cudaStream_t st) {
+                           __half *v_pages, cudaStream_t st, unsigned long long *stamp) {
   return launch_pdl(rope_kv_kernel, dim3(in.M, Hq + 2 * Hkv), dim3(hd / 2), 0, st, in, part, n_splits,
-                    part_rows, Hq, Hkv, hd, rope_tab, q_out, q_lo_out, k_pages, v_pages);
+                    part_rows, Hq, Hkv, hd, rope_tab, q_out, q_lo_out, k_pages, v_pages, stamp);
 }
 
 // One CTA per source row; thread i moves 16 bytes.  Block (tile, kb) of the stored matrix starts at row

@@ -71,6 +71,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
+  if (threadIdx.x == 0) stamp_min(g.stamp);
   // Let the next kernel launch now: it waits (griddepcontrol.wait) for this one to finish before it touches
   // dependent data, so only its launch latency and its own prologue (weight prefetch) move forward.  Placed after
   // this CTA holds its resources, so a waiting dependent can never starve an earlier kernel.
@@ -89,6 +90,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
         tma_load_2d(smem_u32(smem + (size_t)it * stage_bytes), &tmap_w, 0, (blockIdx.x * g.n_kblocks + kb0 + it) * kTileN, bar, pol_w);
       }
       pdl_wait();
+      stamp_waited(g.stamp);
       for (int it = 0; it < pre; ++it) {
         uint32_t bar = smem_u32(&ctl->full[it]);
         tma_load_3d(smem_u32(smem + (size_t)it * stage_bytes + kWBytes), &tmap_a, (kb0 + it) * kBlockK, m0, 0,
@@ -222,6 +224,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     tc_fence_after();
     tmem_dealloc(tmem_base, alloc_cols);
   }
+  if (threadIdx.x == 0 && g.stamp) stamp_max(g.stamp + 3);
 }
 
 static size_t gemm_smem_bytes(int stages, int planes, int Mc) {

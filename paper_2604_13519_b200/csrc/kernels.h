@@ -41,6 +41,7 @@ struct GemmArgs {
   int out_planes;
   unsigned long long *amax;  // EPI_LOGITS: [M] packed (ordered logit bits << 32 | ~token id), atomicMax
   int *err;             // device status word
+  unsigned long long *stamp;   // optional clock stamps of this launch (null = none)
 };
 
 int gemm_pick_stages(int planes, int Mc, size_t smem_budget);
@@ -60,6 +61,7 @@ struct StepIn {
   const int32_t *parent;     // [M] parent of each row inside its chunk (row index relative to the chunk; -1 = root)
   const uint32_t *anc;       // [M][2] low / high word of the row's visibility mask over its chunk: bit i = row i of
                              // the chunk is the row itself or one of its ancestors (a chain: bits 0..j)
+  const int32_t *row_leaves; // [M] attention leaves of the row's sequence: ceil((cached length + chunk rows) / leaf length)
   int pages_per_seq;
   int B, M;
 };
@@ -70,12 +72,13 @@ cudaError_t launch_embed_norm(const StepIn &in, const __nv_bfloat16 *embed, cons
                               unsigned long long *amax, cudaStream_t st);
 // x[m] += sum_s part[s][m]; h = rmsnorm(x) * gain -> bf16 (hi[, lo])
 cudaError_t launch_add_norm(int M, int d, const float *part, int n_splits, int part_rows, const float *gain,
-                            float eps, float *x, __nv_bfloat16 *h, int h_rows, int planes, cudaStream_t st);
+                            float eps, float *x, __nv_bfloat16 *h, int h_rows, int planes, cudaStream_t st,
+                            unsigned long long *stamp = nullptr);
 // qkv = sum of split-K partials; rotary on q and k; q -> fp16 [M][Hq][hd] (and, if q_lo_out is given, the rounding
 // remainder of every element as a second fp16 array of the same shape); k, v -> fp16 pages
 cudaError_t launch_rope_kv(const StepIn &in, const float *part, int n_splits, int part_rows, int Hq, int Hkv,
                            int hd, const float2 *rope_tab, __half *q_out, __half *q_lo_out, __half *k_pages,
-                           __half *v_pages, cudaStream_t st);
+                           __half *v_pages, cudaStream_t st, unsigned long long *stamp = nullptr);
 
 constexpr int kAttnMaxSplits = 32;   // KV splits per (row tile, kv head): one lane of the merge kernel each
 
@@ -120,6 +123,7 @@ struct AttnTcArgs {
   __nv_bfloat16 *out;            // [planes][out_rows][Hq*hd] merged, normalised rows as bf16 (hi[, lo])
   int out_rows, planes;
   int *err;                      // device status word
+  unsigned long long *stamp, *stamp_merge;   // optional clock stamps of the attention and the merge launch
 };
 cudaError_t launch_attention_tc(const AttnTcArgs &a, cudaStream_t st);
 cudaError_t launch_attention_tc_merge(const AttnTcArgs &a, cudaStream_t st);

@@ -56,9 +56,10 @@ struct Layout {
   // workspace (byte offsets)
   uint64_t x, h, part, q, attn_o, attn_ml, attn, act, logits, amax, rope, d_in, d_out, workspace_bytes;
   // fused single-kernel path
-  uint64_t maps, slab, ss_part, sync, phase_t;
+  uint64_t maps, slab, ss_part, sync, phase_t, stamps;
+  int max_stamps;
   int n_maps, n_counters, n_phases, max_tiles128, o_tile128_seq, o_tile128_row0;
-  int leaf_len, max_units, o_unit_tile, o_unit_leaf;   // attention leaves (see AttnTcArgs)
+  int leaf_len, max_units, o_unit_tile, o_unit_leaf, o_row_leaves;   // attention leaves (see AttnTcArgs)
   // step io (int32 offsets inside d_in / h_in)
   int o_tokens, o_pos, o_rowseq, o_cu, o_len, o_tile_seq, o_tile_row0, o_btab, in_ints;
   int o_parent, o_anc, o_path, o_uni, o_topk, o_slot;
@@ -146,6 +147,7 @@ void make_layout(const ts_model_config &c, Layout *L) {
   while ((int64_t)L->leaf_len * kMaxAttnSplits < c.max_ctx) L->leaf_len *= 2;
   L->max_units = L->max_tiles128 * kMaxAttnSplits;
   L->o_unit_tile = itake(L->max_units); L->o_unit_leaf = itake(L->max_units);
+  L->o_row_leaves = itake(c.max_rows);
   L->o_parent = itake(c.max_rows); L->o_anc = itake(2 * c.max_rows); L->o_uni = itake(c.max_rows);
   L->o_slot = itake(c.max_rows);
   L->o_btab = itake(c.max_batch * L->pages_per_seq);   // (last: only the used part is copied per step)
@@ -166,6 +168,8 @@ void make_layout(const ts_model_config &c, Layout *L) {
   L->sync = take((uint64_t)(8 + L->n_counters) * 4);
   L->n_phases = 6 * c.n_layers + 3;
   L->phase_t = take((uint64_t)3 * L->n_phases * 8);
+  L->max_stamps = 9 * c.n_layers + 16;
+  L->stamps = take((uint64_t)L->max_stamps * 4 * 8);
   L->workspace_bytes = o;
   L->host_io_bytes = align_up((uint64_t)(L->in_ints + L->out_ints) * 4, 4096);
 }
@@ -217,8 +221,16 @@ struct ts_model {
   bool profiling = false;
   std::vector<cudaEvent_t> prof_ev;
   std::vector<int> prof_cls;
+  // device-clock timeline (ts_debug_timeline): four stamps per launch of the step being recorded
+  bool timeline = false;
+  int stamp_idx = 0;
+  std::vector<int> stamp_cls;
+  unsigned long long *stamp_slot() const {
+    return (timeline && stamp_idx < L.max_stamps) ? (unsigned long long *)WS(L.stamps) + 4 * (size_t)stamp_idx : nullptr;
+  }
   void launched(int cls) {
     ++launches;
+    if (timeline) { stamp_cls.push_back(cls); ++stamp_idx; }
     if (profiling) {
       cudaEvent_t e;
       if (cudaEventCreate(&e) == cudaSuccess) {
@@ -327,6 +339,7 @@ ts_status run_gemm(ts_model *m, int epi, const CUtensorMap &tw, const CUtensorMa
   g.act_out = act_out; g.act_rows = m->L.rows_alloc; g.out_planes = m->planes;
   g.amax = amax;
   g.err = m->d_out() + m->L.o_err;
+  g.stamp = m->stamp_slot();
   if (plan) { plan->splits = splits; plan->kb_per_split = g.kb_per_split; }
   CU_TRY(ts::launch_gemm(epi, tw, ta4[mi], g, splits, m->gemm_smem_budget, m->st, m->use_pdl && !m->profiling));
   m->launched(0);
@@ -345,6 +358,7 @@ ts_status run_step_fused(ts_model *m) {
   a.in.tokens = di + L.o_tokens; a.in.pos = di + L.o_pos; a.in.row_seq = di + L.o_rowseq; a.in.cu_rows = di + L.o_cu;
   a.in.seq_len = di + L.o_len; a.in.block_tab = di + L.o_btab; a.in.pages_per_seq = L.pages_per_seq;
   a.in.parent = di + L.o_parent; a.in.anc = (const uint32_t *)(di + L.o_anc); a.in.slot = di + L.o_slot;
+  a.in.row_leaves = di + L.o_row_leaves;
   a.in.B = m->last_B; a.in.M = m->last_M;
   a.mc_index = pick_mc_index(m->last_M); a.Mc = kMcOptions[a.mc_index]; a.planes = m->planes;
   a.n_ctas = m->n_sms; a.skip_lm = (m->last_flags & TS_FLAG_SKIP_LM_HEAD) ? 1 : 0;
@@ -395,6 +409,7 @@ ts_status run_step(ts_model *m) {
   in.tokens = di + L.o_tokens; in.pos = di + L.o_pos; in.row_seq = di + L.o_rowseq; in.cu_rows = di + L.o_cu;
   in.seq_len = di + L.o_len; in.block_tab = di + L.o_btab; in.pages_per_seq = L.pages_per_seq;
   in.parent = di + L.o_parent; in.anc = (const uint32_t *)(di + L.o_anc); in.slot = di + L.o_slot;
+  in.row_leaves = di + L.o_row_leaves;
   in.B = B; in.M = M;
   float *x = (float *)m->WS(L.x);
   __nv_bfloat16 *h = (__nv_bfloat16 *)m->WS(L.h);
@@ -437,19 +452,21 @@ ts_status run_step(ts_model *m) {
   for (int l = 0; l < c.n_layers; ++l) {
     if (l > 0) {
       CU_TRY(ts::launch_add_norm(M, d, part, plan.splits, R, (const float *)m->W(L.g1[l]), c.rms_eps, x, h, R,
-                                 m->planes, m->st));
+                                 m->planes, m->st, m->stamp_slot()));
       m->launched(3);
     }
     ts_status s = run_gemm(m, ts::EPI_PARTIAL, m->tm_qkv[l], m->tm_h, L.Nqkv, d, M, part, nullptr, nullptr, &plan);
     if (s) return s;
     CU_TRY(ts::launch_rope_kv(in, part, plan.splits, R, c.n_q_heads, c.n_kv_heads, c.head_dim, rope, q,
-                              q + (size_t)R * Nq, m->k_pages(l), m->v_pages(l), m->st));
+                              q + (size_t)R * Nq, m->k_pages(l), m->v_pages(l), m->st, m->stamp_slot()));
     m->launched(4);
     aa.k_pages = m->k_pages(l); aa.v_pages = m->v_pages(l);
     if (m->fused_ok) {   // tensor-memory attention (needs the same device features as the persistent kernel)
       at.layer = l;
+      at.stamp = m->stamp_slot();
       CU_TRY(ts::launch_attention_tc(at, m->st));
       m->launched(1);
+      at.stamp_merge = m->stamp_slot();
       CU_TRY(ts::launch_attention_tc_merge(at, m->st));
     } else {
       CU_TRY(ts::launch_attention_split(aa, m->st));
@@ -460,7 +477,7 @@ ts_status run_step(ts_model *m) {
     s = run_gemm(m, ts::EPI_PARTIAL, m->tm_o[l], m->tm_attn, d, Nq, M, part, nullptr, nullptr, &plan);
     if (s) return s;
     CU_TRY(ts::launch_add_norm(M, d, part, plan.splits, R, (const float *)m->W(L.g2[l]), c.rms_eps, x, h, R,
-                               m->planes, m->st));
+                               m->planes, m->st, m->stamp_slot()));
     m->launched(3);
     // (gate-up keeps its SwiGLU epilogue and so cannot split K: 192 tiles run as 1.3 waves.  Splitting K
     // three ways with a separate SwiGLU kernel filled the waves but cost as much as it saved.)
@@ -471,7 +488,7 @@ ts_status run_step(ts_model *m) {
   }
   if (m->last_flags & TS_FLAG_SKIP_LM_HEAD) return TS_OK;
   CU_TRY(ts::launch_add_norm(M, d, part, plan.splits, R, (const float *)m->W(L.gf), c.rms_eps, x, h, R, m->planes,
-                             m->st));
+                             m->st, m->stamp_slot()));
   m->launched(3);
   unsigned long long *amax = (unsigned long long *)m->WS(L.amax);
   ts_status s = run_gemm(m, ts::EPI_LOGITS, m->tm_lm, m->tm_h, c.vocab, d, M, (float *)m->WS(L.logits), nullptr,
@@ -601,6 +618,7 @@ ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::ve
       const int k = hi[L.o_cu + i + 1] - hi[L.o_cu + i], total = hi[L.o_len + i] + k;
       const int n_leaves = (total + L.leaf_len - 1) / L.leaf_len;
       slots = std::max(slots, n_leaves);
+      for (int r = hi[L.o_cu + i]; r < hi[L.o_cu + i + 1]; ++r) hi[L.o_row_leaves + r] = n_leaves;
       for (int r0 = 0; r0 < k * G; r0 += 128) {
         hi[L.o_tile128_seq + t] = i;
         hi[L.o_tile128_row0 + t] = r0;
@@ -1616,6 +1634,30 @@ ts_status ts_debug_schedule(int32_t n_tiles, int32_t n_kblocks, int32_t n_ctas, 
     ++n;
   }
   *n_segments = n;
+  return TS_OK;
+}
+
+ts_status ts_debug_timeline(ts_model *m, uint64_t *stamps, int32_t *classes, int32_t cap, int32_t *n_launches) {
+  if (!m || !n_launches || (cap > 0 && (!stamps || !classes))) return fail(TS_ERR_ARG, "null argument");
+  if (!m->have_step) return fail(TS_ERR_STATE, "no step has been staged yet");
+  if (m->last_fused) return fail(TS_ERR_UNIMPLEMENTED, "the persistent kernel has its own clocks (ts_debug_phase_clocks)");
+  const Layout &L = m->L;
+  std::vector<unsigned long long> init((size_t)L.max_stamps * 4);
+  for (int i = 0; i < L.max_stamps; ++i) { init[4 * i] = init[4 * i + 1] = ~0ull; init[4 * i + 2] = init[4 * i + 3] = 0ull; }
+  CU_TRY(cudaMemcpyAsync(m->WS(L.stamps), init.data(), init.size() * 8, cudaMemcpyHostToDevice, m->st));
+  CU_TRY(cudaStreamSynchronize(m->st));
+  m->timeline = true; m->stamp_idx = 0; m->stamp_cls.clear();
+  ts_status st = run_step(m);
+  m->timeline = false;
+  if (st) return st;
+  CU_TRY(cudaMemcpyAsync(init.data(), m->WS(L.stamps), init.size() * 8, cudaMemcpyDeviceToHost, m->st));
+  CU_TRY(cudaStreamSynchronize(m->st));
+  const int n = std::min<int>((int)m->stamp_cls.size(), L.max_stamps);
+  *n_launches = n;
+  for (int i = 0; i < n && i < cap; ++i) {
+    classes[i] = m->stamp_cls[i];
+    for (int j = 0; j < 4; ++j) stamps[4 * i + j] = init[4 * (size_t)i + j];
+  }
   return TS_OK;
 }
 
