@@ -1,6 +1,8 @@
 // Paged grouped-query attention of the verify chunk on the 5th-generation tensor cores, as a kernel of its own.
 //
-// One CTA = one unit: (128-row tile of packed (position, query head) rows, kv head, leaf of the KV positions).
+// One unit = (128-row tile of packed (position, query head) rows, kv head, leaf of the KV positions); a CTA takes one
+// unit when the step has no more units than SMs, else it walks several (tensor memory, barriers and the K/V ring are
+// set up once and the ring keeps running across units).
 //   warp 0   K/V producer: TMA loads of 64-position blocks straight from the pages (5-d tensor map over the pool)
 //   warp 1   tensor memory allocation + tcgen05.mma issue:  S = Q K^T  (Q tile and K block K-major in shared
 //            memory, 128 x 64 fp32 result in tensor memory), then  O_blk = P V  with P read from tensor memory
@@ -11,6 +13,8 @@
 // Each leaf writes an un-normalised partial output with its (max, sum); attn_merge_kernel adds a row's leaves.
 // Every wait is bounded; on expiry the CTA records an error word and leaves through the normal exit.
 #include <cuda_fp16.h>
+
+#include <algorithm>
 
 #include "kernels.h"
 #include "schedule.h"
@@ -26,7 +30,7 @@ static constexpr int kWorkerWarp0 = 2;
 
 struct __align__(16) AttnCtl {
   uint64_t kv_full[kKvStages], kv_empty[kKvStages], q_full;
-  uint64_t s_full[2], s_empty[2], p_full[2], pv_done;
+  uint64_t s_full[2], s_empty[2], p_full[2], pv_done, o_free;
   uint32_t tmem_base;
 };
 
@@ -64,7 +68,11 @@ struct AttnUnit {
   int pos_beg, pos_end, nblk;
 };
 
-// CTA u works on pair u / Hkv (a row tile and one leaf of its sequence) for kv head u % Hkv.  The leaf's positions
+// The j-th unit of CTA c out of G: units are listed longest first and dealt out in rounds of G, every other round in
+// reverse CTA order, so that the CTA given the longest unit of one round gets the shortest of the next.
+__device__ __forceinline__ int attn_unit_of(int c, int j, int G) { return j * G + ((j & 1) ? G - 1 - c : c); }
+
+// Unit u works on pair u / Hkv (a row tile and one leaf of its sequence) for kv head u % Hkv.  The leaf's positions
 // are [leaf * leaf_len, (leaf + 1) * leaf_len), cut off at the end of the chunk: absolute positions, so the blocks a
 // row meets, and their order, do not depend on where the chunk starts or how long it is.
 __device__ __forceinline__ AttnUnit attn_unit_info(const AttnTcArgs &a, int u) {
@@ -221,8 +229,8 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
       pk1[e] = pack_h2(e2, e3);
     }
     // the previous product has to be complete before its P buffer's twin is reused and before the sums are touched
-    if (b > 0) {
-      if (ok && !mbar_wait_err(smem_u32(&ctl->pv_done), (uint32_t)(b - 1) & 1u, err)) { ok = false; atomicCAS((int *)err, 0, DEV_TIMEOUT_TMEM); }
+    if (b > 0) {   // (barrier phases are counted over all blocks of this CTA, like `blk`)
+      if (ok && !mbar_wait_err(smem_u32(&ctl->pv_done), (blk - 1) & 1u, err)) { ok = false; atomicCAS((int *)err, 0, DEV_TIMEOUT_TMEM); }
       tc_fence_after();
     }
     float f = 1.f;
@@ -252,7 +260,7 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
     if (lane == 0) mbar_arrive(smem_u32(&ctl->p_full[buf]));
     // (no CTA-wide barrier per block: a failed wait has set the error word, which ends every other wait)
   }
-  if (ok && !mbar_wait_err(smem_u32(&ctl->pv_done), (uint32_t)(t.nblk - 1) & 1u, err)) { ok = false; atomicCAS((int *)err, 0, DEV_TIMEOUT_TMEM); }
+  if (ok && !mbar_wait_err(smem_u32(&ctl->pv_done), (blk - 1) & 1u, err)) { ok = false; atomicCAS((int *)err, 0, DEV_TIMEOUT_TMEM); }
   tc_fence_after();
   if (!worker_all(ok)) return false;
 
@@ -277,6 +285,11 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
       }
     }
   }
+  // the output sums are in registers / on their way to memory: the next unit's first product may overwrite them, and
+  // its queries may be staged over this unit's (every score product of this unit has completed)
+  tc_fence_before();
+  __syncwarp();
+  if (lane == 0) mbar_arrive(smem_u32(&ctl->o_free));
   return true;
 }
 
@@ -301,6 +314,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
     }
     mbar_init(smem_u32(&ctl->q_full), 1);
     mbar_init(smem_u32(&ctl->pv_done), 1);
+    mbar_init(smem_u32(&ctl->o_free), 4);   // one arrival per worker warp
     fence_barrier_init();
   }
   if (warp == 1) {
@@ -314,82 +328,99 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
   if (threadIdx.x == 0) stamp_min(a.stamp);
   pdl_launch_dependents();   // (this CTA holds its tensor memory; the dependent waits for this kernel's end anyway)
   // The step's integer inputs were copied in before the step's first kernel started, so they may be read here.
-  const AttnUnit t = attn_unit_info(a, (int)blockIdx.x);
+  // This CTA's units: attn_unit_of(blockIdx.x, 0, 1, 2, ...).  The three roles walk the units as three loops coupled only by the barriers, whose
+  // phases are counted over all blocks (`gb`) and units (`un`) of the CTA.
+  const int n_total = a.n_units * a.Hkv;
 
   if (warp == 0) {
     // ---------------------------------------------------------------- K/V producer
-    if (lane == 0 && t.nblk > 0) {
+    if (lane == 0) {
       const uint64_t pol = policy_evict_first();
-      const int32_t *btab = a.in.block_tab + (size_t)t.seq * a.in.pages_per_seq;
-      auto load_block = [&](int b) {
-        const uint32_t st = b % kKvStages;
-        const uint32_t bar = smem_u32(&ctl->kv_full[st]);
-        mbar_expect_tx(bar, kKvBytes);
-        uint8_t *sK = smem + kQBytes + st * kKvBytes, *sV = sK + kAttnBlk * HD * 2;
-        for (int pg = 0; pg < kAttnBlk / 16; ++pg) {
-          // a page past the split's end is never visible; load the last visible page again instead
-          const int pos = min(t.pos_beg + b * kAttnBlk + pg * 16, t.pos_end - 1);
-          const int page = btab[pos >> 4];
+      uint32_t gb = 0;
+      bool waited = false, ok = true;
+      for (int j = 0; j * (int)gridDim.x < n_total && ok; ++j) {
+        const int u = attn_unit_of((int)blockIdx.x, j, (int)gridDim.x);
+        if (u >= n_total) continue;
+        const AttnUnit t = attn_unit_info(a, u);
+        const int32_t *btab = a.in.block_tab + (size_t)t.seq * a.in.pages_per_seq;
+        for (int b = 0; b < t.nblk; ++b, ++gb) {
+          // blocks wholly inside the cache of earlier steps do not depend on the previous kernel: the ring is filled
+          // with them before the dependency wait; the chunk's own K/V rows come from the previous kernel
+          if (!waited && (gb >= (uint32_t)kKvStages || t.pos_beg + (b + 1) * kAttnBlk > t.len)) { pdl_wait(); waited = true; }
+          const uint32_t st = gb % kKvStages;
+          if (gb >= (uint32_t)kKvStages &&
+              !mbar_wait_err(smem_u32(&ctl->kv_empty[st]), ((gb / kKvStages) & 1) ^ 1, err)) { atomicCAS(a.err, 0, DEV_TIMEOUT_EMPTY); ok = false; break; }
+          const uint32_t bar = smem_u32(&ctl->kv_full[st]);
+          mbar_expect_tx(bar, kKvBytes);
+          uint8_t *sK = smem + kQBytes + st * kKvBytes, *sV = sK + kAttnBlk * HD * 2;
+          for (int pg = 0; pg < kAttnBlk / 16; ++pg) {
+            // a page past the unit's end is never visible; load the last visible page again instead
+            const int pos = min(t.pos_beg + b * kAttnBlk + pg * 16, t.pos_end - 1);
+            const int page = btab[pos >> 4];
 #pragma unroll
-          for (int hh = 0; hh < (int)kHalves; ++hh) {
-            const uint32_t off = hh * (kAttnBlk * 128) + pg * 2048;
-            tma_load_5d(smem_u32(sK + off), a.map_kv, hh * 64, 0, t.kh, page, 2 * a.layer, bar, pol);
-            tma_load_5d(smem_u32(sV + off), a.map_kv, hh * 64, 0, t.kh, page, 2 * a.layer + 1, bar, pol);
+            for (int hh = 0; hh < (int)kHalves; ++hh) {
+              const uint32_t off = hh * (kAttnBlk * 128) + pg * 2048;
+              tma_load_5d(smem_u32(sK + off), a.map_kv, hh * 64, 0, t.kh, page, 2 * a.layer, bar, pol);
+              tma_load_5d(smem_u32(sV + off), a.map_kv, hh * 64, 0, t.kh, page, 2 * a.layer + 1, bar, pol);
+            }
           }
         }
-      };
-      // blocks wholly inside the cache of earlier steps do not depend on the previous kernel: fill the ring with them
-      int b = 0;
-      for (; b < min(t.nblk, kKvStages) && t.pos_beg + (b + 1) * kAttnBlk <= t.len; ++b) load_block(b);
-      pdl_wait();   // the chunk's own K/V rows come from the previous kernel
-      for (; b < t.nblk; ++b) {
-        if (!mbar_wait_err(smem_u32(&ctl->kv_empty[b % kKvStages]), ((b / kKvStages) & 1) ^ 1, err)) { atomicCAS(a.err, 0, DEV_TIMEOUT_EMPTY); break; }
-        load_block(b);
       }
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issue
-    if (lane == 0 && t.nblk > 0) {
+    if (lane == 0) {
       const uint32_t idesc_qk = umma_idesc_f16(kAttnRows, kAttnBlk, 0);
       const uint32_t idesc_pv = umma_idesc_f16(kAttnRows, HD, 1);
       const uint32_t sQ = smem_u32(smem);
       bool ok = true;
-      auto issue_pv = [&](uint32_t bi) -> bool {   // O += P V for block bi
+      uint32_t gb = 0, un = 0;
+      // O (+)= P V for block bi; `first`: the unit's first block starts the sums afresh, which needs the workers to
+      // have read the previous unit's sums out
+      auto issue_pv = [&](uint32_t bi, bool first) -> bool {
         const uint32_t pb = bi & 1, vst = bi % kKvStages;
         if (!mbar_wait_err(smem_u32(&ctl->p_full[pb]), (bi >> 1) & 1, err)) return false;
+        if (first && un > 0 && !mbar_wait_err(smem_u32(&ctl->o_free), (un - 1) & 1, err)) return false;
         tc_fence_after();
         const uint32_t sV = sQ + kQBytes + vst * kKvBytes + kAttnBlk * HD * 2;
 #pragma unroll
         for (int ks = 0; ks < kAttnBlk / 16; ++ks)   // 16 positions per instruction
           umma_f16_ts(tmem_base + kColO, tmem_base + kColP + pb * 32 + ks * 8,
-                      umma_desc_sw128_mn(sV + ks * 2048, kAttnBlk * 128), idesc_pv, (bi | ks) != 0 ? 1u : 0u);
+                      umma_desc_sw128_mn(sV + ks * 2048, kAttnBlk * 128), idesc_pv, (!first || ks != 0) ? 1u : 0u);
         umma_commit(smem_u32(&ctl->pv_done));
         umma_commit(smem_u32(&ctl->kv_empty[vst]));
         return true;
       };
-      ok = mbar_wait_err(smem_u32(&ctl->q_full), 0, err);
-      for (uint32_t b = 0; ok && b < (uint32_t)t.nblk; ++b) {
-        const uint32_t kst = b % kKvStages, st = b & 1;
-        if (!mbar_wait_err(smem_u32(&ctl->kv_full[kst]), (b / kKvStages) & 1, err)) { ok = false; break; }
-        if (!mbar_wait_err(smem_u32(&ctl->s_empty[st]), ((b >> 1) & 1) ^ 1, err)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t sK = sQ + kQBytes + kst * kKvBytes;
-        // S = Q K^T + Q_lo K^T: the remainder plane of the queries goes through the same keys into the same sums
+      for (int j = 0; j * (int)gridDim.x < n_total && ok; ++j) {
+        const int u = attn_unit_of((int)blockIdx.x, j, (int)gridDim.x);
+        if (u >= n_total) continue;
+        const AttnUnit t = attn_unit_info(a, u);
+        if (t.nblk == 0) continue;
+        ok = mbar_wait_err(smem_u32(&ctl->q_full), un & 1, err);
+        for (int b = 0; ok && b < t.nblk; ++b, ++gb) {
+          const uint32_t kst = gb % kKvStages, st = gb & 1;
+          if (!mbar_wait_err(smem_u32(&ctl->kv_full[kst]), (gb / kKvStages) & 1, err)) { ok = false; break; }
+          if (!mbar_wait_err(smem_u32(&ctl->s_empty[st]), ((gb >> 1) & 1) ^ 1, err)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sK = sQ + kQBytes + kst * kKvBytes;
+          // S = Q K^T + Q_lo K^T: the remainder plane of the queries goes through the same keys into the same sums
 #pragma unroll
-        for (int pl = 0; pl < 2; ++pl) {
+          for (int pl = 0; pl < 2; ++pl) {
 #pragma unroll
-          for (int hh = 0; hh < (int)kHalves; ++hh) {
-            const uint64_t dq = umma_desc_sw128(sQ + pl * (kAttnRows * HD * 2) + hh * (kAttnRows * 128));
-            const uint64_t dk = umma_desc_sw128(sK + hh * (kAttnBlk * 128));
+            for (int hh = 0; hh < (int)kHalves; ++hh) {
+              const uint64_t dq = umma_desc_sw128(sQ + pl * (kAttnRows * HD * 2) + hh * (kAttnRows * 128));
+              const uint64_t dk = umma_desc_sw128(sK + hh * (kAttnBlk * 128));
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              umma_bf16(tmem_base + kColS + st * 64, dq + 2 * kk, dk + 2 * kk, idesc_qk, (pl | hh | kk) != 0 ? 1u : 0u);
+              for (int kk = 0; kk < 4; ++kk)
+                umma_bf16(tmem_base + kColS + st * 64, dq + 2 * kk, dk + 2 * kk, idesc_qk, (pl | hh | kk) != 0 ? 1u : 0u);
+            }
           }
+          umma_commit(smem_u32(&ctl->s_full[st]));
+          if (b > 0) ok = issue_pv(gb - 1, b == 1);
         }
-        umma_commit(smem_u32(&ctl->s_full[st]));
-        if (b > 0) ok = issue_pv(b - 1);
+        if (ok) ok = issue_pv(gb - 1, t.nblk == 1);
+        ++un;
       }
-      if (ok) ok = issue_pv((uint32_t)t.nblk - 1);
       if (!ok) atomicCAS(a.err, 0, DEV_TIMEOUT_FULL);
     }
   } else {
@@ -397,7 +428,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
     uint32_t blk = 0;
     pdl_wait();   // the rotated queries come from the previous kernel
     if (threadIdx.x == kWorkerWarp0 * 32) stamp_waited(a.stamp);
-    attn_unit_workers<HD>(a, ctl, t, smem, tmem_base, warp & 3, lane, (int)threadIdx.x - kWorkerWarp0 * 32, blk, err);
+    bool ok = true;
+    for (int j = 0; j * (int)gridDim.x < n_total && ok; ++j) {
+      const int u = attn_unit_of((int)blockIdx.x, j, (int)gridDim.x);
+      if (u >= n_total) continue;
+      const AttnUnit t = attn_unit_info(a, u);
+      ok = attn_unit_workers<HD>(a, ctl, t, smem, tmem_base, warp & 3, lane, (int)threadIdx.x - kWorkerWarp0 * 32, blk, err);
+    }
   }
   tc_fence_before();
   __syncthreads();
@@ -486,7 +523,7 @@ cudaError_t launch_attention_tc(const AttnTcArgs &a, cudaStream_t st) {
     once.done(dev_);
   }
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(a.n_units * a.Hkv);
+  cfg.gridDim = dim3(std::min(a.n_units * a.Hkv, a.max_ctas));
   cfg.blockDim = dim3(kTcThreads);
   cfg.dynamicSmemBytes = attn_tc_smem(a.hd);
   cfg.stream = st;

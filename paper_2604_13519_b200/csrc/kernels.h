@@ -110,7 +110,8 @@ struct AttnTcArgs {
   StepIn in;
   int Hq, Hkv, hd, layer;
   int leaf_len;                  // KV positions per leaf
-  int n_units;                   // (tile, leaf) pairs of this step; the grid is n_units * Hkv CTAs
+  int n_units;                   // (tile, leaf) pairs of this step: n_units * Hkv units of work
+  int max_ctas;                  // CTAs launched at most (one per SM); a CTA walks units blockIdx.x, + gridDim.x, ...
   int n_slots;                   // partial results kept per (row, query head): the most leaves any sequence has
   const int32_t *unit_tile;      // [n_units] tile of each pair
   const int32_t *unit_leaf;      // [n_units] leaf of each pair

@@ -59,7 +59,7 @@ struct Layout {
   uint64_t maps, slab, ss_part, sync, phase_t, stamps;
   int max_stamps;
   int n_maps, n_counters, n_phases, max_tiles128, o_tile128_seq, o_tile128_row0;
-  int leaf_len, max_units, o_unit_tile, o_unit_leaf, o_row_leaves;   // attention leaves (see AttnTcArgs)
+  int max_units, o_unit_tile, o_unit_leaf, o_row_leaves;   // attention units (see AttnTcArgs)
   // step io (int32 offsets inside d_in / h_in)
   int o_tokens, o_pos, o_rowseq, o_cu, o_len, o_tile_seq, o_tile_row0, o_btab, in_ints;
   int o_parent, o_anc, o_path, o_uni, o_topk, o_slot;
@@ -141,10 +141,6 @@ void make_layout(const ts_model_config &c, Layout *L) {
   L->o_tile_seq = itake(L->max_tiles); L->o_tile_row0 = itake(L->max_tiles);
   L->max_tiles128 = c.max_batch * ((c.k_max * G + 127) / 128);
   L->o_tile128_seq = itake(L->max_tiles128); L->o_tile128_row0 = itake(L->max_tiles128);
-  // attention leaf: the smallest power-of-two number of 64-position blocks with at most kMaxAttnSplits leaves in
-  // max_ctx positions.  A constant of the model, NOT of the step: a row's bits must not depend on the step's shape.
-  L->leaf_len = 64;
-  while ((int64_t)L->leaf_len * kMaxAttnSplits < c.max_ctx) L->leaf_len *= 2;
   L->max_units = L->max_tiles128 * kMaxAttnSplits;
   L->o_unit_tile = itake(L->max_units); L->o_unit_leaf = itake(L->max_units);
   L->o_row_leaves = itake(c.max_rows);
@@ -200,6 +196,7 @@ struct ts_model {
   Layout L{};
   cudaStream_t st = nullptr;
   int planes = 1, n_sms = 148;
+  int leaf_len = 64;   // KV positions per attention leaf: a constant of the model (see AttnTcArgs), set by ts_init_model
   size_t gemm_smem_budget = 100 * 1024;
   std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_d;
   CUtensorMap tm_lm{}, tm_h[4]{}, tm_attn[4]{}, tm_act[4]{};
@@ -439,7 +436,7 @@ ts_status run_step(ts_model *m) {
 
   ts::AttnTcArgs at{};
   at.in = in; at.Hq = c.n_q_heads; at.Hkv = c.n_kv_heads; at.hd = c.head_dim;
-  at.leaf_len = L.leaf_len; at.n_units = m->last_units; at.n_slots = m->last_slots;
+  at.leaf_len = m->leaf_len; at.n_units = m->last_units; at.n_slots = m->last_slots; at.max_ctas = m->n_sms;
   at.unit_tile = di + L.o_unit_tile; at.unit_leaf = di + L.o_unit_leaf;
   at.tile_seq = di + L.o_tile128_seq; at.tile_row0 = di + L.o_tile128_row0;
   at.q = q; at.q_lo = q + (size_t)R * Nq; at.map_kv = (const CUtensorMap *)m->WS(L.maps) + (L.n_maps - 1);
@@ -616,14 +613,14 @@ ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::ve
     int slots = 1;
     for (int i : order) {
       const int k = hi[L.o_cu + i + 1] - hi[L.o_cu + i], total = hi[L.o_len + i] + k;
-      const int n_leaves = (total + L.leaf_len - 1) / L.leaf_len;
+      const int n_leaves = (total + m->leaf_len - 1) / m->leaf_len;
       slots = std::max(slots, n_leaves);
       for (int r = hi[L.o_cu + i]; r < hi[L.o_cu + i + 1]; ++r) hi[L.o_row_leaves + r] = n_leaves;
       for (int r0 = 0; r0 < k * G; r0 += 128) {
         hi[L.o_tile128_seq + t] = i;
         hi[L.o_tile128_row0 + t] = r0;
         for (int lf = 0; lf < n_leaves; ++lf)
-          units.push_back({t, lf, (std::min(total, (lf + 1) * L.leaf_len) - lf * L.leaf_len + 63) / 64});
+          units.push_back({t, lf, (std::min(total, (lf + 1) * m->leaf_len) - lf * m->leaf_len + 63) / 64});
         ++t;
       }
     }
@@ -844,6 +841,21 @@ ts_status ts_init_model(const ts_model_config *cfg, const ts_buffers *bufs, void
     m->smem_optin = (size_t)optin;
     m->fused_ok = coop != 0 && m->n_sms <= kMaxFusedCtas &&
                   ts::fused_ring_stages(m->planes, kFusedMaxRows, c.head_dim, m->smem_optin) >= 2;
+  }
+  {
+    // Attention leaf length.  A constant of the model, NOT of the step: a row's bits must not depend on the step's
+    // shape.  Chosen so that a full batch at full context gives about one unit of work per SM -- groups = (sequence,
+    // row tile, kv head) triples of a full step, leaves per group = 95% of the SMs / groups, at least 4 and at most
+    // kMaxAttnSplits -- in whole 64-position blocks: a batch-1 model gets many short leaves (its few groups must
+    // cover the SMs), a batched one a few long ones (a leaf costs a fixed start-up and one partial result per row;
+    // four per full-length sequence still let ragged batches be dealt out evenly over the SMs).
+    const int G = c.n_q_heads / c.n_kv_heads;
+    const int groups = c.max_batch * ((c.k_max * G + 127) / 128) * c.n_kv_heads;
+    const int want = std::max(4, std::min(kMaxAttnSplits, (int)(0.95 * m->n_sms) / std::max(1, groups)));
+    const int blocks = (c.max_ctx + 63) / 64;
+    int leaf_blocks = std::max(1, (blocks + want - 1) / want);
+    while ((blocks + leaf_blocks - 1) / leaf_blocks > kMaxAttnSplits) ++leaf_blocks;
+    m->leaf_len = 64 * leaf_blocks;
   }
   m->free_pages.resize(c.max_pages);
   for (int i = 0; i < c.max_pages; ++i) m->free_pages[i] = c.max_pages - 1 - i;   // hand out 0, 1, 2, ...
