@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtoolspec.so")
-SOURCES = ["model.cu", "gemm_tcgen05.cu", "attention.cu", "attention_tc.cu", "elementwise.cu", "fused.cu", "attention_static.cu", "sampling.cu", "retrieval.cu", "topk.cu", "drafter.cpp"]
+SOURCES = ["model.cu", "gemm_tcgen05.cu", "gemm_rows_tcgen05.cu", "attention.cu", "attention_tc.cu", "elementwise.cu", "fused.cu", "attention_static.cu", "sampling.cu", "retrieval.cu", "topk.cu", "drafter.cpp"]
 
 
 def _stale() -> bool:

@@ -1,0 +1,272 @@
+// The dense projections of the verify step for MANY rows (batched steps: more than 64 rows), where the work is bound by
+// the tensor cores and by the bytes an SM pulls from L2 per flop, no longer by streaming the weights:
+//     out[m][n] = sum_k act[m][k] * W[n][k]
+// Orientation: a CTA owns a chunk of 128 activation rows (operand A of the tensor-core instruction, its 128-row
+// dimension) and 256 weight rows (operand B, the instruction's N dimension); the accumulator in tensor memory is
+// 128 lanes (rows) x 256 fp32 columns (features).  The (hi, lo) bf16 planes of the activations are two instructions
+// into the SAME accumulator, so per 64-wide k-block a CTA brings in 32 KB of activations and 32 KB of weights for
+// 8.4 MFLOP -- two thirds of the bytes per flop of the weight-streaming kernel (gemm_tcgen05.cu), which at these sizes
+// is what sets the pace.  The weight matrix keeps its storage (contiguous 128 x 64 blocks, one TMA box each): a CTA's
+// 256 weight rows are two such boxes.  One CTA per SM (three 64 KB stages).
+//
+// Roles: warp 0 = TMA producer, warp 1 = TMEM allocation + MMA issue, warps 2..5 = epilogue (thread <-> row).
+// Every wait is bounded; on expiry the CTA records an error word and leaves through the normal exit.
+#include <algorithm>
+
+#include "kernels.h"
+
+namespace ts {
+
+static constexpr int kBlockK = 64;                 // k-block: 64 bf16 = 128 bytes per row
+static constexpr int kRowsM = 128;                 // activation rows per CTA
+static constexpr int kBoxN = 128;                  // weight rows per stored block (one TMA box)
+static constexpr int kTileN = 256;                 // weight rows per CTA
+static constexpr int kBoxBytes = kBoxN * kBlockK * 2;
+static constexpr int kMaxStages = 4;
+
+struct __align__(8) RowsSmemCtl {
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
+  uint64_t tmem_full;
+  uint32_t tmem_base;
+  uint32_t abort_flag;
+};
+
+template <int EPI>
+__global__ void __launch_bounds__(192, 1)
+gemm_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_a,
+                 const GemmArgs g) {
+  extern __shared__ uint8_t smem_raw[];
+  // 1024-byte alignment is required by the 128-byte swizzle pattern
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int a_bytes = g.planes * kRowsM * kBlockK * 2;
+  const int stage_bytes = a_bytes + 2 * kBoxBytes;
+  RowsSmemCtl *ctl = reinterpret_cast<RowsSmemCtl *>(smem + (size_t)g.stages * stage_bytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * kTileN;
+  const int nb = min(kTileN, g.N - n0);             // 256, or 128 for a last tile of an odd number of blocks
+  const int split = blockIdx.y;
+  const int m0 = blockIdx.z * kRowsM;
+  // balanced cut of the k-blocks into gridDim.y runs
+  const int kb0 = (int)(((long long)split * g.n_kblocks) / (int)gridDim.y);
+  const int kb1 = (int)(((long long)(split + 1) * g.n_kblocks) / (int)gridDim.y);
+  const int nkb = kb1 - kb0;
+  const int tx_bytes = a_bytes + (nb / kBoxN) * kBoxBytes;
+
+  if (warp == 0 && lane == 0) {
+    tma_prefetch_desc(&tmap_w);
+    tma_prefetch_desc(&tmap_a);
+    for (int s = 0; s < g.stages; ++s) {
+      mbar_init(smem_u32(&ctl->full[s]), 1);
+      mbar_init(smem_u32(&ctl->empty[s]), 1);
+    }
+    mbar_init(smem_u32(&ctl->tmem_full), 1);
+    ctl->abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&ctl->tmem_base), kTileN);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+  if (threadIdx.x == 0) stamp_min(g.stamp);
+  // (placed after this CTA holds its resources, so a waiting dependent can never starve an earlier kernel)
+  pdl_launch_dependents();
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0 && nkb > 0) {
+      const uint64_t pol_w = policy_evict_first(), pol_a = policy_evict_last();
+      // block (128-row block j, k-block kb) of the stored matrix = rows (j * n_kblocks + kb) * 128 .. of a [.][64] array
+      auto load_w = [&](int s, int kb) {
+        const uint32_t bar = smem_u32(&ctl->full[s]);
+        const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes + a_bytes);
+        for (int j = 0; j < nb / kBoxN; ++j)
+          tma_load_2d(dst + j * kBoxBytes, &tmap_w, 0, ((2 * (int)blockIdx.x + j) * g.n_kblocks + kb) * kBoxN, bar, pol_w);
+      };
+      const int pre = min(g.stages, nkb);
+      // weights do not depend on the previous kernel: start them before the programmatic-dependency wait
+      for (int it = 0; it < pre; ++it) {
+        mbar_expect_tx(smem_u32(&ctl->full[it]), tx_bytes);
+        load_w(it, kb0 + it);
+      }
+      pdl_wait();
+      stamp_waited(g.stamp);
+      for (int it = 0; it < pre; ++it)
+        tma_load_3d(smem_u32(smem + (size_t)it * stage_bytes), &tmap_a, (kb0 + it) * kBlockK, m0, 0,
+                    smem_u32(&ctl->full[it]), pol_a);
+      int s = (pre == g.stages) ? 0 : pre;
+      uint32_t ph = (pre == g.stages) ? 1 : 0;
+      for (int it = pre; it < nkb; ++it) {
+        if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1)) {
+          atomicExch(g.err, DEV_TIMEOUT_EMPTY);
+          break;
+        }
+        mbar_expect_tx(smem_u32(&ctl->full[s]), tx_bytes);
+        load_w(s, kb0 + it);
+        tma_load_3d(smem_u32(smem + (size_t)s * stage_bytes), &tmap_a, (kb0 + it) * kBlockK, m0, 0,
+                    smem_u32(&ctl->full[s]), pol_a);
+        if (++s == g.stages) { s = 0; ph ^= 1; }
+      }
+    } else if (lane == 0) {
+      pdl_wait();
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issue
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(kRowsM, (uint32_t)nb);
+      bool ok = true;
+      int s = 0;
+      uint32_t ph = 0;
+      for (int it = 0; it < nkb; ++it) {
+        if (!mbar_wait(smem_u32(&ctl->full[s]), ph)) {
+          atomicExch(g.err, DEV_TIMEOUT_FULL);
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+        const uint64_t db = umma_desc_sw128(sa + a_bytes);
+        // the value plane and the remainder plane of the activations into the same sums
+        for (int pl = 0; pl < g.planes; ++pl) {
+          const uint64_t da = umma_desc_sw128(sa + pl * (kRowsM * kBlockK * 2));
+#pragma unroll
+          for (int kk = 0; kk < kBlockK / 16; ++kk)   // 16 bf16 along K = 32 bytes = 2 descriptor address units
+            umma_bf16(tmem_base, da + 2 * kk, db + 2 * kk, idesc, (it | kk | pl) != 0);
+        }
+        umma_commit(smem_u32(&ctl->empty[s]));
+        if (++s == g.stages) { s = 0; ph ^= 1; }
+      }
+      if (!ok) ctl->abort_flag = 1;
+      umma_commit(smem_u32(&ctl->tmem_full));
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5): thread <-> row
+    pdl_wait();   // outputs of this kernel may still be read by the previous one's consumers
+    bool ok = true;
+    if (nkb > 0) {
+      ok = mbar_wait(smem_u32(&ctl->tmem_full), 0);
+      if (!ok && lane == 0) atomicExch(g.err, DEV_TIMEOUT_TMEM);
+    }
+    tc_fence_after();
+    ok = ok && (*reinterpret_cast<volatile uint32_t *>(&ctl->abort_flag) == 0);
+    const int q = warp & 3;                       // TMEM lane quarter this warp may read
+    const int m = m0 + q * 32 + lane;             // this thread's row
+    const bool row_ok = m < g.M;
+    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+    float best = -INFINITY;
+    int best_n = 0;
+    if (ok) {
+      for (int c0 = 0; c0 < nb; c0 += 16) {
+        uint32_t r[16];
+        float v[16];
+        if (nkb > 0) {
+          tmem_ld16(taddr + c0, r);     // (warp-wide: rows past the end read too, and write nothing)
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] = 0.f;
+        }
+        const int n = n0 + c0;
+        if constexpr (EPI == EPI_PARTIAL) {
+          if (row_ok) {
+            float4 *dst = reinterpret_cast<float4 *>(g.out + ((size_t)split * g.out_rows + m) * g.N + n);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+          }
+        } else if constexpr (EPI == EPI_LOGITS) {
+          if (row_ok) {
+            float4 *dst = reinterpret_cast<float4 *>(g.out + (size_t)m * g.N + n);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+              if (v[j] > best) { best = v[j]; best_n = n + j; }   // (ascending ids: a tie keeps the lower one)
+          }
+        } else {  // EPI_SWIGLU: even feature = gate_f, odd = up_f, f = n / 2
+          const int F = g.N >> 1, f = n >> 1;
+          __nv_bfloat16 hi[8], lo[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float gate = v[2 * j], up = v[2 * j + 1];
+            split_bf16(gate / (1.f + __expf(-gate)) * up, hi[j], lo[j]);
+          }
+          if (row_ok) {
+            *reinterpret_cast<uint4 *>(g.act_out + (size_t)m * F + f) = *reinterpret_cast<uint4 *>(hi);
+            if (g.out_planes == 2)
+              *reinterpret_cast<uint4 *>(g.act_out + ((size_t)g.act_rows + m) * F + f) = *reinterpret_cast<uint4 *>(lo);
+          }
+        }
+      }
+      if constexpr (EPI == EPI_LOGITS) {
+        if (row_ok) {
+          // order-preserving map of the float to an unsigned word; ties resolve to the lowest id
+          uint32_t u = __float_as_uint(best);
+          u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+          atomicMax(g.amax + m, ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)best_n));
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTileN);
+  }
+  if (threadIdx.x == 0 && g.stamp) stamp_max(g.stamp + 3);
+}
+
+static size_t rows_smem_bytes(int stages, int planes) {
+  return (size_t)stages * (planes * kRowsM * kBlockK * 2 + 2 * kBoxBytes) + sizeof(RowsSmemCtl) + 1024;
+}
+
+template <int EPI>
+static cudaError_t launch_rows_one(const CUtensorMap &tw, const CUtensorMap &ta, const GemmArgs &g, dim3 grid,
+                                   size_t smem, cudaStream_t st, bool pdl) {
+  static PerDeviceOnce once;
+  int dev_ = -1;
+  if (once.needed(&dev_)) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_rows_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    once.done(dev_);
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(192);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, gemm_rows_kernel<EPI>, tw, ta, g);
+}
+
+int gemm_rows_tiles(int N) { return (N + kTileN - 1) / kTileN; }
+
+// `ta` must be the activation map whose box holds 128 rows.  N must be a multiple of 128.
+cudaError_t launch_gemm_rows(int epi, const CUtensorMap &tw, const CUtensorMap &ta, GemmArgs g, int n_splits,
+                             size_t smem_limit, cudaStream_t st, bool pdl) {
+  if (n_splits < 1 || n_splits > g.n_kblocks || g.N % kBoxN) return cudaErrorInvalidValue;
+  g.Mc = kRowsM;
+  g.stages = kMaxStages;
+  while (g.stages > 2 && rows_smem_bytes(g.stages, g.planes) > smem_limit) --g.stages;
+  const size_t smem = rows_smem_bytes(g.stages, g.planes);
+  if (smem > smem_limit) return cudaErrorInvalidConfiguration;
+  dim3 grid(gemm_rows_tiles(g.N), n_splits, (g.M + kRowsM - 1) / kRowsM);
+  switch (epi) {
+    case EPI_PARTIAL: return launch_rows_one<EPI_PARTIAL>(tw, ta, g, grid, smem, st, pdl);
+    case EPI_SWIGLU: return launch_rows_one<EPI_SWIGLU>(tw, ta, g, grid, smem, st, pdl);
+    default: return launch_rows_one<EPI_LOGITS>(tw, ta, g, grid, smem, st, pdl);
+  }
+}
+
+}  // namespace ts

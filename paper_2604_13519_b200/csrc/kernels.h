@@ -48,6 +48,12 @@ int gemm_pick_stages(int planes, int Mc, size_t smem_budget);
 cudaError_t launch_gemm(int epi, const CUtensorMap &tw, const CUtensorMap &ta, GemmArgs g, int n_splits,
                         size_t smem_budget, cudaStream_t st, bool pdl);
 
+// The same projections for many rows (gemm_rows_tcgen05.cu): 128 activation rows x 256 weight rows per CTA, one CTA
+// per SM.  `ta` must be the activation map whose box holds 128 rows; g.Mc and g.stages are set by the launcher.
+int gemm_rows_tiles(int N);
+cudaError_t launch_gemm_rows(int epi, const CUtensorMap &tw, const CUtensorMap &ta, GemmArgs g, int n_splits,
+                             size_t smem_limit, cudaStream_t st, bool pdl);
+
 // Per-step inputs resident in device memory (all int32).
 struct StepIn {
   const int32_t *tokens;     // [M] chunk ids, rows of sequence i at cu_rows[i]..cu_rows[i+1]

@@ -306,9 +306,9 @@ int pick_mc_index(int M) {
 
 // split-K factor: two CTAs fit on an SM, so the grid runs in waves of 2 * n_sms CTAs; take the smallest factor
 // (at least 4 k-blocks per slice) whose last wave is at least 95% full, else the one that fills its waves best
-int pick_splits(const ts_model *m, int n_tiles, int m_chunks, int n_kblocks, bool allow) {
+int pick_splits(const ts_model *m, int n_tiles, int m_chunks, int n_kblocks, bool allow, int ctas_per_sm = 2) {
   if (!allow) return 1;
-  const int ctas = std::max(1, n_tiles * m_chunks), slots = 2 * m->n_sms;
+  const int ctas = std::max(1, n_tiles * m_chunks), slots = ctas_per_sm * m->n_sms;
   const int s_max = std::max(1, std::min(kMaxSplits, n_kblocks / 4));
   int best = 1;
   double best_eff = 0.0;
@@ -329,8 +329,12 @@ ts_status run_gemm(ts_model *m, int epi, const CUtensorMap &tw, const CUtensorMa
   ts::GemmArgs g{};
   g.N = N; g.K = K; g.M = M; g.Mc = kMcOptions[mi]; g.planes = m->planes;
   g.n_kblocks = K / 64;
+  // Up to 64 rows the step is bound by streaming the weights (weight-major kernel, two CTAs per SM); beyond, by the
+  // tensor cores and the bytes per flop an SM pulls from L2 (row-major kernel, 256 weight rows per CTA, one CTA per SM)
+  const bool many_rows = M > 64;
   const int m_chunks = (M + g.Mc - 1) / g.Mc;
-  int splits = pick_splits(m, N / 128, m_chunks, g.n_kblocks, epi == ts::EPI_PARTIAL);
+  int splits = many_rows ? pick_splits(m, ts::gemm_rows_tiles(N), m_chunks, g.n_kblocks, epi == ts::EPI_PARTIAL, 1)
+                         : pick_splits(m, N / 128, m_chunks, g.n_kblocks, epi == ts::EPI_PARTIAL);
   g.kb_per_split = (g.n_kblocks + splits - 1) / splits;   // (the kernel cuts K into `splits` balanced runs)
   g.out = out; g.out_rows = m->L.rows_alloc;
   g.act_out = act_out; g.act_rows = m->L.rows_alloc; g.out_planes = m->planes;
@@ -338,7 +342,10 @@ ts_status run_gemm(ts_model *m, int epi, const CUtensorMap &tw, const CUtensorMa
   g.err = m->d_out() + m->L.o_err;
   g.stamp = m->stamp_slot();
   if (plan) { plan->splits = splits; plan->kb_per_split = g.kb_per_split; }
-  CU_TRY(ts::launch_gemm(epi, tw, ta4[mi], g, splits, m->gemm_smem_budget, m->st, m->use_pdl && !m->profiling));
+  if (many_rows)
+    CU_TRY(ts::launch_gemm_rows(epi, tw, ta4[3], g, splits, m->smem_optin, m->st, m->use_pdl && !m->profiling));
+  else
+    CU_TRY(ts::launch_gemm(epi, tw, ta4[mi], g, splits, m->gemm_smem_budget, m->st, m->use_pdl && !m->profiling));
   m->launched(0);
   return TS_OK;
 }
