@@ -44,13 +44,16 @@ gemm_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
   RowsSmemCtl *ctl = reinterpret_cast<RowsSmemCtl *>(smem + (size_t)g.stages * stage_bytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * kTileN;
+  // grid = (row chunks, weight tiles, K slices): the row chunks of one (tile, slice) are neighbours in launch order, so
+  // they run at the same time and all but the first find the weight blocks in L2
+  const int tile = blockIdx.y;
+  const int n0 = tile * kTileN;
   const int nb = min(kTileN, g.N - n0);             // 256, or 128 for a last tile of an odd number of blocks
-  const int split = blockIdx.y;
-  const int m0 = blockIdx.z * kRowsM;
-  // balanced cut of the k-blocks into gridDim.y runs
-  const int kb0 = (int)(((long long)split * g.n_kblocks) / (int)gridDim.y);
-  const int kb1 = (int)(((long long)(split + 1) * g.n_kblocks) / (int)gridDim.y);
+  const int split = blockIdx.z;
+  const int m0 = blockIdx.x * kRowsM;
+  // balanced cut of the k-blocks into gridDim.z runs
+  const int kb0 = (int)(((long long)split * g.n_kblocks) / (int)gridDim.z);
+  const int kb1 = (int)(((long long)(split + 1) * g.n_kblocks) / (int)gridDim.z);
   const int nkb = kb1 - kb0;
   const int tx_bytes = a_bytes + (nb / kBoxN) * kBoxBytes;
 
@@ -86,7 +89,7 @@ gemm_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
         const uint32_t bar = smem_u32(&ctl->full[s]);
         const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes + a_bytes);
         for (int j = 0; j < nb / kBoxN; ++j)
-          tma_load_2d(dst + j * kBoxBytes, &tmap_w, 0, ((2 * (int)blockIdx.x + j) * g.n_kblocks + kb) * kBoxN, bar, pol_w);
+          tma_load_2d(dst + j * kBoxBytes, &tmap_w, 0, ((2 * tile + j) * g.n_kblocks + kb) * kBoxN, bar, pol_w);
       };
       const int pre = min(g.stages, nkb);
       // weights do not depend on the previous kernel: start them before the programmatic-dependency wait
@@ -261,7 +264,7 @@ cudaError_t launch_gemm_rows(int epi, const CUtensorMap &tw, const CUtensorMap &
   while (g.stages > 2 && rows_smem_bytes(g.stages, g.planes) > smem_limit) --g.stages;
   const size_t smem = rows_smem_bytes(g.stages, g.planes);
   if (smem > smem_limit) return cudaErrorInvalidConfiguration;
-  dim3 grid(gemm_rows_tiles(g.N), n_splits, (g.M + kRowsM - 1) / kRowsM);
+  dim3 grid((g.M + kRowsM - 1) / kRowsM, gemm_rows_tiles(g.N), n_splits);
   switch (epi) {
     case EPI_PARTIAL: return launch_rows_one<EPI_PARTIAL>(tw, ta, g, grid, smem, st, pdl);
     case EPI_SWIGLU: return launch_rows_one<EPI_SWIGLU>(tw, ta, g, grid, smem, st, pdl);
