@@ -4,9 +4,11 @@
 // unit when the step has no more units than SMs, else it walks several (tensor memory, barriers and the K/V ring are
 // set up once and the ring keeps running across units).
 //   warp 0   K/V producer: TMA loads of 64-position blocks straight from the pages (5-d tensor map over the pool)
-//   warp 1   tensor memory allocation + tcgen05.mma issue:  S = Q K^T  (Q tile and K block K-major in shared
-//            memory, 128 x 64 fp32 result in tensor memory), then  O_blk = P V  with P read from tensor memory
-//            (fp16) and the V block read MN-major from the same [position][64 elements] image K uses
+//   warp 1   tensor memory allocation + tcgen05.mma issue:  S = Q K^T  (the unit's queries sit in tensor memory as
+//            the row operand -- re-reading a 128-row query tile from shared memory for every 64-position block was
+//            what bounded the kernel -- the K block K-major in shared memory, 128 x 64 fp32 result in tensor
+//            memory), then  O_blk = P V  with P read from tensor memory (fp16) and the V block read MN-major from
+//            the same [position][64 elements] image K uses
 //   warps 2..5  one row per thread: maximum over the block's 64 scores, P = exp2(S - reference maximum) written back
 //            to tensor memory as fp16.  The output sums stay in tensor memory (every P V adds to them); the
 //            reference maximum follows the running one in steps, and only then is the row of sums multiplied down
@@ -23,14 +25,14 @@ namespace ts {
 
 static constexpr int kAttnRows = 128;   // packed rows per unit
 static constexpr int kAttnBlk = 64;     // kv positions per block
-static constexpr int kKvStages = 4;     // K/V blocks in flight
+static constexpr int kKvStages = 6;     // K/V blocks in the ring (three are held by issued products, the rest are in flight)
 static constexpr int kTcThreads = 192;
 static constexpr int kWorkers = 128;
 static constexpr int kWorkerWarp0 = 2;
 
 struct __align__(16) AttnCtl {
   uint64_t kv_full[kKvStages], kv_empty[kKvStages], q_full;
-  uint64_t s_full[2], s_empty[2], p_full[2], pv_done, o_free;
+  uint64_t s_full[2], s_empty[2], p_full[2], pv_done[2], o_free;
   uint32_t tmem_base;
 };
 
@@ -47,7 +49,6 @@ __device__ __forceinline__ bool worker_all(bool ok) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ bool mbar_wait_err(uint32_t bar, uint32_t parity, const int *err) {
   uint64_t t0 = 0;
   for (uint32_t it = 0;; ++it) {
@@ -98,19 +99,18 @@ __device__ __forceinline__ AttnUnit attn_unit_info(const AttnTcArgs &a, int u) {
 static constexpr int kColS = 0;      // two score buffers of 64 columns
 static constexpr int kColP = 128;    // two probability buffers of 32 columns (fp16 pairs)
 static constexpr int kColO = 192;    // the output sums: head_dim columns, accumulated over the unit's blocks
+static constexpr int kColQ = 320;    // the unit's queries, fp16 pairs: head_dim / 2 columns of values, then as many of remainders
 static constexpr float kRescaleStep = 8.f;   // the reference maximum follows the running one in steps of 2^8
 
-__device__ __forceinline__ void cp_async16z(uint32_t dst, const void *src, bool valid) {
-  const int sz = valid ? 16 : 0;
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
-}
-__device__ __forceinline__ void cp_commit_wait_all() {
-  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
-}
 // 2^x for x <= 0 (and 0 for -inf); tiny results flush to zero
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float y;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
   return y;
 }
 __device__ __forceinline__ uint32_t pack_h2(float x, float y) {
@@ -122,7 +122,7 @@ __device__ __forceinline__ uint32_t pack_h2(float x, float y) {
 // block's 64 scores, writes the 64 probabilities back as fp16 and, rarely, rescales the row's output sums.
 // `blk` counts K/V blocks over all units of this CTA (buffer index and barrier parity come from it).
 template <int HD>
-__device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *ctl, const AttnUnit &t, uint8_t *sQ, uint32_t tmem_base,
+__device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *ctl, const AttnUnit &t, uint32_t tmem_base,
                                                   int q, int lane, int wtid, uint32_t &blk, const int *err) {
   constexpr int CH = HD / 8;          // 16-byte chunks per row
   const int row = q * 32 + lane;      // row of the tile
@@ -134,24 +134,36 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
     if (valid) a.attn_ml[ob] = make_float2(-INFINITY, 0.f);
     return true;
   }
-  // ---- stage Q: [128 rows][64 elements] images with the 128-byte swizzle, one per 64-element half, first of the
-  // values, then of their rounding remainders -------------------------------------------------------------
-  for (int idx = wtid; idx < kAttnRows * CH; idx += kWorkers) {
-    const int r = idx / CH, c = idx % CH;
-    const int prr = t.row0 + r;
-    const bool v = r < t.rows_here;
-    const int jj = v ? prr / t.G : 0, gg = v ? prr % t.G : 0;
-    const size_t so = ((size_t)(t.r_beg + jj) * a.Hq + t.kh * t.G + gg) * HD + c * 8;
-    const uint32_t dst = smem_u32(sQ) + (c >> 3) * (kAttnRows * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4);
-    cp_async16z(dst, a.q + so, v);
-    cp_async16z(dst + kAttnRows * HD * 2, a.q_lo + so, v);
+  // ---- stage Q into tensor memory: the score product reads its row operand there (thread <-> row, an fp16 pair
+  // per column: head_dim / 2 columns of values, then as many of rounding remainders), so per block only the keys
+  // and values come through shared memory.  Every score product of the CTA's previous unit has completed (its
+  // last scores were read before that unit's sums were drained), so the columns may be overwritten.
+  const uint32_t tq = tmem_base + ((uint32_t)(q * 32) << 16);
+  {
+    const size_t so = ((size_t)(t.r_beg + j) * a.Hq + t.kh * t.G + gq) * HD;
+#pragma unroll
+    for (int pl = 0; pl < 2; ++pl) {
+      const uint4 *src = reinterpret_cast<const uint4 *>((pl ? a.q_lo : a.q) + so);
+      uint4 v[CH];
+#pragma unroll
+      for (int c = 0; c < CH; ++c) v[c] = valid ? src[c] : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+      for (int c4 = 0; c4 < CH / 4; ++c4) {
+        uint32_t r[16];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          r[4 * e] = v[4 * c4 + e].x; r[4 * e + 1] = v[4 * c4 + e].y;
+          r[4 * e + 2] = v[4 * c4 + e].z; r[4 * e + 3] = v[4 * c4 + e].w;
+        }
+        tmem_st16(tq + kColQ + pl * (HD / 2) + c4 * 16, r);
+      }
+    }
+    tmem_wait_st();
   }
-  cp_commit_wait_all();
-  fence_proxy_async_all();   // generic-proxy writes -> tcgen05 (async proxy) reads
+  tc_fence_before();
   worker_sync();
   if (wtid == 0) mbar_arrive(smem_u32(&ctl->q_full));
 
-  const uint32_t tq = tmem_base + ((uint32_t)(q * 32) << 16);
   // Visibility: the whole cache, and of the chunk the rows named by this row's mask (itself and its ancestors in
   // the draft tree; in a chain, rows 0..j), up to the end of this split.
   const int lim_all = min(t.len, t.pos_end) - 1;   // every row sees every position up to here
@@ -207,8 +219,9 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
     }
     float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-    for (int e = 0; e < 64; e += 4) {
-      mx0 = fmaxf(mx0, sc[e]); mx1 = fmaxf(mx1, sc[e + 1]); mx2 = fmaxf(mx2, sc[e + 2]); mx3 = fmaxf(mx3, sc[e + 3]);
+    for (int e = 0; e < 64; e += 8) {   // three-input maxima: half the instructions of pairwise ones
+      mx0 = max3(mx0, sc[e], sc[e + 1]); mx1 = max3(mx1, sc[e + 2], sc[e + 3]);
+      mx2 = max3(mx2, sc[e + 4], sc[e + 5]); mx3 = max3(mx3, sc[e + 6], sc[e + 7]);
     }
     // block maximum in the log2 domain: scores times log2(e)/sqrt(head_dim), folded into one multiply-add per score
     const float m_blk = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale;
@@ -228,13 +241,15 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
       pk0[e] = pack_h2(e0, e1);
       pk1[e] = pack_h2(e2, e3);
     }
-    // the previous product has to be complete before its P buffer's twin is reused and before the sums are touched
-    if (b > 0) {   // (barrier phases are counted over all blocks of this CTA, like `blk`)
-      if (ok && !mbar_wait_err(smem_u32(&ctl->pv_done), (blk - 1) & 1u, err)) { ok = false; atomicCAS((int *)err, 0, DEV_TIMEOUT_TMEM); }
-      tc_fence_after();
-    }
+    // This block's P buffer last fed product b - 2, which is complete: the scores of this block were committed after
+    // it by the same thread, and a commit covers everything issued before it.  Only multiplying the sums down needs
+    // more -- product b - 1 complete -- so that is the only case that waits.  The products of even and of odd blocks
+    // complete phases of barriers of their own: a waiter is then never more than one phase behind (product b - 3,
+    // the previous one on the same barrier, is known complete), which a parity wait needs.
     float f = 1.f;
     if (b > 0 && __any_sync(0xffffffffu, raise)) {       // tensor-memory accesses are warp-wide: lanes that stay use f = 1
+      if (ok && !mbar_wait_err(smem_u32(&ctl->pv_done[(blk - 1) & 1u]), ((blk - 1) >> 1) & 1u, err)) { ok = false; atomicCAS((int *)err, 0, DEV_TIMEOUT_TMEM); }
+      tc_fence_after();
       if (raise) f = ex2_approx(m_old - ref);            // exp2(-inf) = 0: nothing was summed before the first finite maximum
 #pragma unroll
       for (int i = 0; i < HD / 32; ++i) {
@@ -260,7 +275,8 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
     if (lane == 0) mbar_arrive(smem_u32(&ctl->p_full[buf]));
     // (no CTA-wide barrier per block: a failed wait has set the error word, which ends every other wait)
   }
-  if (ok && !mbar_wait_err(smem_u32(&ctl->pv_done), (blk - 1) & 1u, err)) { ok = false; atomicCAS((int *)err, 0, DEV_TIMEOUT_TMEM); }
+  // the unit's last product (and with it every earlier one)
+  if (ok && !mbar_wait_err(smem_u32(&ctl->pv_done[(blk - 1) & 1u]), ((blk - 1) >> 1) & 1u, err)) { ok = false; atomicCAS((int *)err, 0, DEV_TIMEOUT_TMEM); }
   tc_fence_after();
   if (!worker_all(ok)) return false;
 
@@ -286,7 +302,7 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
     }
   }
   // the output sums are in registers / on their way to memory: the next unit's first product may overwrite them, and
-  // its queries may be staged over this unit's (every score product of this unit has completed)
+  // its queries may be written over this unit's (every score product of this unit has completed)
   tc_fence_before();
   __syncwarp();
   if (lane == 0) mbar_arrive(smem_u32(&ctl->o_free));
@@ -297,8 +313,8 @@ template <int HD>
 __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_constant__ AttnTcArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  constexpr uint32_t kQBytes = 2u * kAttnRows * HD * 2, kKvBytes = 2u * kAttnBlk * HD * 2, kHalves = HD / 64;   // Q: two planes
-  AttnCtl *ctl = reinterpret_cast<AttnCtl *>(smem + kQBytes + kKvStages * kKvBytes);
+  constexpr uint32_t kKvBytes = 2u * kAttnBlk * HD * 2, kHalves = HD / 64;
+  AttnCtl *ctl = reinterpret_cast<AttnCtl *>(smem + kKvStages * kKvBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int *err = a.err;
 
@@ -311,9 +327,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
       mbar_init(smem_u32(&ctl->s_full[b]), 1);
       mbar_init(smem_u32(&ctl->s_empty[b]), 4);
       mbar_init(smem_u32(&ctl->p_full[b]), 4);
+      mbar_init(smem_u32(&ctl->pv_done[b]), 1);
     }
     mbar_init(smem_u32(&ctl->q_full), 1);
-    mbar_init(smem_u32(&ctl->pv_done), 1);
     mbar_init(smem_u32(&ctl->o_free), 4);   // one arrival per worker warp
     fence_barrier_init();
   }
@@ -352,7 +368,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
               !mbar_wait_err(smem_u32(&ctl->kv_empty[st]), ((gb / kKvStages) & 1) ^ 1, err)) { atomicCAS(a.err, 0, DEV_TIMEOUT_EMPTY); ok = false; break; }
           const uint32_t bar = smem_u32(&ctl->kv_full[st]);
           mbar_expect_tx(bar, kKvBytes);
-          uint8_t *sK = smem + kQBytes + st * kKvBytes, *sV = sK + kAttnBlk * HD * 2;
+          uint8_t *sK = smem + st * kKvBytes, *sV = sK + kAttnBlk * HD * 2;
           for (int pg = 0; pg < kAttnBlk / 16; ++pg) {
             // a page past the unit's end is never visible; load the last visible page again instead
             const int pos = min(t.pos_beg + b * kAttnBlk + pg * 16, t.pos_end - 1);
@@ -369,59 +385,82 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issue
-    if (lane == 0) {
+    // The whole warp walks the loops and the waits together; one elected lane issues each tensor-core instruction and
+    // each commit (the loop state is then the same in every lane, which lets the compiler keep descriptors and
+    // addresses in uniform registers: a lone lane issued an instruction every ~50 cycles, too slow for 20 small
+    // instructions per 64-position block).
+    {
       const uint32_t idesc_qk = umma_idesc_f16(kAttnRows, kAttnBlk, 0);
       const uint32_t idesc_pv = umma_idesc_f16(kAttnRows, HD, 1);
-      const uint32_t sQ = smem_u32(smem);
+      const uint32_t sKV = smem_u32(smem);
       bool ok = true;
       uint32_t gb = 0, un = 0;
+      // a wait that ran out in one lane ends the loops of all lanes together (elect.sync names the full warp)
+      auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, mbar_wait_err(bar, parity, err));
+      };
       // O (+)= P V for block bi; `first`: the unit's first block starts the sums afresh, which needs the workers to
       // have read the previous unit's sums out
       auto issue_pv = [&](uint32_t bi, bool first) -> bool {
         const uint32_t pb = bi & 1, vst = bi % kKvStages;
-        if (!mbar_wait_err(smem_u32(&ctl->p_full[pb]), (bi >> 1) & 1, err)) return false;
-        if (first && un > 0 && !mbar_wait_err(smem_u32(&ctl->o_free), (un - 1) & 1, err)) return false;
+        if (!wait_all(smem_u32(&ctl->p_full[pb]), (bi >> 1) & 1)) return false;
+        if (first && un > 0 && !wait_all(smem_u32(&ctl->o_free), (un - 1) & 1)) return false;
         tc_fence_after();
-        const uint32_t sV = sQ + kQBytes + vst * kKvBytes + kAttnBlk * HD * 2;
+        const uint32_t sV = sKV + vst * kKvBytes + kAttnBlk * HD * 2;
 #pragma unroll
         for (int ks = 0; ks < kAttnBlk / 16; ++ks)   // 16 positions per instruction
-          umma_f16_ts(tmem_base + kColO, tmem_base + kColP + pb * 32 + ks * 8,
-                      umma_desc_sw128_mn(sV + ks * 2048, kAttnBlk * 128), idesc_pv, (!first || ks != 0) ? 1u : 0u);
-        umma_commit(smem_u32(&ctl->pv_done));
-        umma_commit(smem_u32(&ctl->kv_empty[vst]));
+          if (elect_one())
+            umma_f16_ts(tmem_base + kColO, tmem_base + kColP + pb * 32 + ks * 8,
+                        umma_desc_sw128_mn(sV + ks * 2048, kAttnBlk * 128), idesc_pv, (!first || ks != 0) ? 1u : 0u);
+        if (elect_one()) {
+          umma_commit(smem_u32(&ctl->pv_done[pb]));
+          umma_commit(smem_u32(&ctl->kv_empty[vst]));
+        }
+        __syncwarp();
         return true;
       };
+      // S = Q K^T + Q_lo K^T for block g (counted over the CTA's blocks): the remainder plane of the queries goes
+      // through the same keys into the same sums; the queries are read from tensor memory (8 columns = 16 elements
+      // per instruction)
+      auto issue_qk = [&](uint32_t g) -> bool {
+        const uint32_t kst = g % kKvStages, st = g & 1;
+        if (!wait_all(smem_u32(&ctl->kv_full[kst]), (g / kKvStages) & 1)) return false;
+        if (!wait_all(smem_u32(&ctl->s_empty[st]), ((g >> 1) & 1) ^ 1)) return false;
+        tc_fence_after();
+        const uint32_t sK = sKV + kst * kKvBytes;
+#pragma unroll
+        for (int pl = 0; pl < 2; ++pl) {
+#pragma unroll
+          for (int hh = 0; hh < (int)kHalves; ++hh) {
+            const uint64_t dk = umma_desc_sw128(sK + hh * (kAttnBlk * 128));
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              if (elect_one())
+                umma_f16_ts(tmem_base + kColS + st * 64, tmem_base + kColQ + pl * (HD / 2) + hh * 32 + kk * 8, dk + 2 * kk,
+                            idesc_qk, (pl | hh | kk) != 0 ? 1u : 0u);
+          }
+        }
+        if (elect_one()) umma_commit(smem_u32(&ctl->s_full[st]));
+        __syncwarp();
+        return true;
+      };
+      // Issue order within a unit: S(0), then for every block b: S(b + 1), O += P(b) V(b).  The scores run one block
+      // ahead of the block the workers are on, so a worker finds its scores complete when it gets to them, and the
+      // product of block b waits only for that block's probabilities.
       for (int j = 0; j * (int)gridDim.x < n_total && ok; ++j) {
         const int u = attn_unit_of((int)blockIdx.x, j, (int)gridDim.x);
         if (u >= n_total) continue;
         const AttnUnit t = attn_unit_info(a, u);
         if (t.nblk == 0) continue;
-        ok = mbar_wait_err(smem_u32(&ctl->q_full), un & 1, err);
+        ok = wait_all(smem_u32(&ctl->q_full), un & 1);
+        if (ok) ok = issue_qk(gb);
         for (int b = 0; ok && b < t.nblk; ++b, ++gb) {
-          const uint32_t kst = gb % kKvStages, st = gb & 1;
-          if (!mbar_wait_err(smem_u32(&ctl->kv_full[kst]), (gb / kKvStages) & 1, err)) { ok = false; break; }
-          if (!mbar_wait_err(smem_u32(&ctl->s_empty[st]), ((gb >> 1) & 1) ^ 1, err)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t sK = sQ + kQBytes + kst * kKvBytes;
-          // S = Q K^T + Q_lo K^T: the remainder plane of the queries goes through the same keys into the same sums
-#pragma unroll
-          for (int pl = 0; pl < 2; ++pl) {
-#pragma unroll
-            for (int hh = 0; hh < (int)kHalves; ++hh) {
-              const uint64_t dq = umma_desc_sw128(sQ + pl * (kAttnRows * HD * 2) + hh * (kAttnRows * 128));
-              const uint64_t dk = umma_desc_sw128(sK + hh * (kAttnBlk * 128));
-#pragma unroll
-              for (int kk = 0; kk < 4; ++kk)
-                umma_bf16(tmem_base + kColS + st * 64, dq + 2 * kk, dk + 2 * kk, idesc_qk, (pl | hh | kk) != 0 ? 1u : 0u);
-            }
-          }
-          umma_commit(smem_u32(&ctl->s_full[st]));
-          if (b > 0) ok = issue_pv(gb - 1, b == 1);
+          if (b + 1 < t.nblk) ok = issue_qk(gb + 1);
+          if (ok) ok = issue_pv(gb, b == 0);
         }
-        if (ok) ok = issue_pv(gb - 1, t.nblk == 1);
         ++un;
       }
-      if (!ok) atomicCAS(a.err, 0, DEV_TIMEOUT_FULL);
+      if (!ok && lane == 0) atomicCAS(a.err, 0, DEV_TIMEOUT_FULL);
     }
   } else {
     // ---------------------------------------------------------------- workers
@@ -433,7 +472,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
       const int u = attn_unit_of((int)blockIdx.x, j, (int)gridDim.x);
       if (u >= n_total) continue;
       const AttnUnit t = attn_unit_info(a, u);
-      ok = attn_unit_workers<HD>(a, ctl, t, smem, tmem_base, warp & 3, lane, (int)threadIdx.x - kWorkerWarp0 * 32, blk, err);
+      ok = attn_unit_workers<HD>(a, ctl, t, tmem_base, warp & 3, lane, (int)threadIdx.x - kWorkerWarp0 * 32, blk, err);
     }
   }
   tc_fence_before();
@@ -509,7 +548,7 @@ cudaError_t launch_attention_tc_merge(const AttnTcArgs &a, cudaStream_t st) {
 }
 
 static size_t attn_tc_smem(int hd) {
-  return 1024 + (size_t)2 * kAttnRows * hd * 2 + (size_t)kKvStages * 2 * kAttnBlk * hd * 2 + sizeof(AttnCtl) + 64;
+  return 1024 + (size_t)kKvStages * 2 * kAttnBlk * hd * 2 + sizeof(AttnCtl) + 64;
 }
 
 cudaError_t launch_attention_tc(const AttnTcArgs &a, cudaStream_t st) {
