@@ -12,6 +12,11 @@
 // Roles: warp 0 = TMA producer, warp 1 = TMEM allocation + MMA issue, warps 2..5 = epilogue (thread <-> row).
 // Every wait is bounded; on expiry the CTA records an error word and leaves through the normal exit.
 #include <algorithm>
+#include <functional>
+#include <map>
+#include <mutex>
+#include <tuple>
+#include <vector>
 
 #include "kernels.h"
 
@@ -46,9 +51,12 @@ gemm_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // grid = (row chunks, weight tiles, K slices): the row chunks of one (tile, slice) are neighbours in launch order, so
   // they run at the same time and all but the first find the weight blocks in L2
+  // the first n_wide tiles hold two stored 128-row weight blocks, the tiles after them one (the launcher mixes the
+  // widths so that the last wave of CTAs is short instead of nearly empty)
   const int tile = blockIdx.y;
-  const int n0 = tile * kTileN;
-  const int nb = min(kTileN, g.N - n0);             // 256, or 128 for a last tile of an odd number of blocks
+  const int blk0 = tile < g.n_wide ? 2 * tile : g.n_wide + tile;   // the tile's first weight block
+  const int n0 = blk0 * kBoxN;
+  const int nb = tile < g.n_wide ? kTileN : kBoxN;
   const int split = blockIdx.z;
   const int m0 = blockIdx.x * kRowsM;
   // balanced cut of the k-blocks into gridDim.z runs
@@ -89,7 +97,7 @@ gemm_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
         const uint32_t bar = smem_u32(&ctl->full[s]);
         const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes + a_bytes);
         for (int j = 0; j < nb / kBoxN; ++j)
-          tma_load_2d(dst + j * kBoxBytes, &tmap_w, 0, ((2 * tile + j) * g.n_kblocks + kb) * kBoxN, bar, pol_w);
+          tma_load_2d(dst + j * kBoxBytes, &tmap_w, 0, ((blk0 + j) * g.n_kblocks + kb) * kBoxN, bar, pol_w);
       };
       const int pre = min(g.stages, nkb);
       // weights do not depend on the previous kernel: start them before the programmatic-dependency wait
@@ -255,16 +263,51 @@ static cudaError_t launch_rows_one(const CUtensorMap &tw, const CUtensorMap &ta,
 
 int gemm_rows_tiles(int N) { return (N + kTileN - 1) / kTileN; }
 
+// How many of a projection's `blocks` stored weight blocks go into 256-row tiles (two blocks) when the launch has
+// `chunks` row chunks and one CTA per SM: the rest become 128-row tiles, launched last.  A 128-row tile costs about
+// 0.6 of a 256-row one (half the flops, three quarters of the bytes through shared memory).  The CTAs start in launch
+// order on whichever SM frees up first; the count with the shortest finish wins, ties go to fewer narrow tiles.
+static int pick_wide_tiles(int blocks, int chunks, int n_sms) {
+  static std::mutex mu;
+  static std::map<std::tuple<int, int, int>, int> memo;
+  std::lock_guard<std::mutex> lk(mu);
+  const auto key = std::make_tuple(blocks, chunks, n_sms);
+  auto it = memo.find(key);
+  if (it != memo.end()) return it->second;
+  const int x_max = blocks / 2;
+  int best_x = x_max;
+  double best_t = 1e30;
+  std::vector<double> sm(n_sms);
+  for (int x = x_max; x >= 0 && x >= x_max - 2 * n_sms; --x) {
+    std::fill(sm.begin(), sm.end(), 0.0);
+    std::make_heap(sm.begin(), sm.end(), std::greater<double>());
+    const int tiles = x + (blocks - 2 * x);
+    for (int t = 0; t < tiles; ++t)
+      for (int c = 0; c < chunks; ++c) {
+        std::pop_heap(sm.begin(), sm.end(), std::greater<double>());
+        sm.back() += t < x ? 1.0 : 0.6;
+        std::push_heap(sm.begin(), sm.end(), std::greater<double>());
+      }
+    const double finish = *std::max_element(sm.begin(), sm.end());
+    if (finish < best_t - 1e-9) { best_t = finish; best_x = x; }
+  }
+  memo[key] = best_x;
+  return best_x;
+}
+
 // `ta` must be the activation map whose box holds 128 rows.  N must be a multiple of 128.
 cudaError_t launch_gemm_rows(int epi, const CUtensorMap &tw, const CUtensorMap &ta, GemmArgs g, int n_splits,
-                             size_t smem_limit, cudaStream_t st, bool pdl) {
+                             size_t smem_limit, int n_sms, cudaStream_t st, bool pdl) {
   if (n_splits < 1 || n_splits > g.n_kblocks || g.N % kBoxN) return cudaErrorInvalidValue;
   g.Mc = kRowsM;
   g.stages = kMaxStages;
   while (g.stages > 2 && rows_smem_bytes(g.stages, g.planes) > smem_limit) --g.stages;
   const size_t smem = rows_smem_bytes(g.stages, g.planes);
   if (smem > smem_limit) return cudaErrorInvalidConfiguration;
-  dim3 grid((g.M + kRowsM - 1) / kRowsM, gemm_rows_tiles(g.N), n_splits);
+  const int blocks = g.N / kBoxN, chunks = (g.M + kRowsM - 1) / kRowsM;
+  // split-K launches are already cut to fill their waves; the others may mix tile widths
+  g.n_wide = n_splits > 1 ? blocks / 2 : pick_wide_tiles(blocks, chunks, n_sms);
+  dim3 grid(chunks, g.n_wide + (blocks - 2 * g.n_wide), n_splits);
   switch (epi) {
     case EPI_PARTIAL: return launch_rows_one<EPI_PARTIAL>(tw, ta, g, grid, smem, st, pdl);
     case EPI_SWIGLU: return launch_rows_one<EPI_SWIGLU>(tw, ta, g, grid, smem, st, pdl);

@@ -34,6 +34,7 @@ struct GemmArgs {
   int n_kblocks;        // K / 64
   int kb_per_split;     // k-blocks per split-K slice
   int stages;           // filled in by the launcher
+  int n_wide;           // many-rows kernel: weight tiles of 256 rows (the tiles after them have 128); filled in by the launcher
   float *out;           // EPI_PARTIAL: [splits][out_rows][N]; EPI_LOGITS: [M][N]
   int out_rows;
   __nv_bfloat16 *act_out;  // EPI_SWIGLU: [out_planes][act_rows][N/2]
@@ -52,7 +53,7 @@ cudaError_t launch_gemm(int epi, const CUtensorMap &tw, const CUtensorMap &ta, G
 // per SM.  `ta` must be the activation map whose box holds 128 rows; g.Mc and g.stages are set by the launcher.
 int gemm_rows_tiles(int N);
 cudaError_t launch_gemm_rows(int epi, const CUtensorMap &tw, const CUtensorMap &ta, GemmArgs g, int n_splits,
-                             size_t smem_limit, cudaStream_t st, bool pdl);
+                             size_t smem_limit, int n_sms, cudaStream_t st, bool pdl);
 
 // Per-step inputs resident in device memory (all int32).
 struct StepIn {

@@ -343,7 +343,7 @@ ts_status run_gemm(ts_model *m, int epi, const CUtensorMap &tw, const CUtensorMa
   g.stamp = m->stamp_slot();
   if (plan) { plan->splits = splits; plan->kb_per_split = g.kb_per_split; }
   if (many_rows)
-    CU_TRY(ts::launch_gemm_rows(epi, tw, ta4[3], g, splits, m->smem_optin, m->st, m->use_pdl && !m->profiling));
+    CU_TRY(ts::launch_gemm_rows(epi, tw, ta4[3], g, splits, m->smem_optin, m->n_sms, m->st, m->use_pdl && !m->profiling));
   else
     CU_TRY(ts::launch_gemm(epi, tw, ta4[mi], g, splits, m->gemm_smem_budget, m->st, m->use_pdl && !m->profiling));
   m->launched(0);
