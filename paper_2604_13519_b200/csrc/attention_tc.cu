@@ -123,13 +123,21 @@ __device__ __forceinline__ uint32_t pack_h2(float x, float y) {
 // `blk` counts K/V blocks over all units of this CTA (buffer index and barrier parity come from it).
 template <int HD>
 __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *ctl, const AttnUnit &t, uint32_t tmem_base,
-                                                  int q, int lane, int wtid, uint32_t &blk, const int *err) {
+                                                  int q, int lane, int wtid, uint32_t &blk, bool &waited, const int *err) {
   constexpr int CH = HD / 8;          // 16-byte chunks per row
   const int row = q * 32 + lane;      // row of the tile
   const int pr = t.row0 + row;        // packed row of the sequence
   const bool valid = row < t.rows_here;
   const int j = valid ? pr / t.G : 0, gq = valid ? pr % t.G : 0;
   const size_t ob = ((size_t)(t.r_beg + j) * a.Hq + t.kh * t.G + gq) * a.n_slots + t.leaf;
+  // (a step input like the unit tables: read before the dependency wait)
+  const unsigned long long anc = ((unsigned long long)a.in.anc[2 * (t.r_beg + j) + 1] << 32) | a.in.anc[2 * (t.r_beg + j)];
+  // the rotated queries come from the previous kernel; everything above was on the device before the step began
+  if (!waited) {
+    pdl_wait();
+    waited = true;
+    if (wtid == 0) stamp_waited(a.stamp);
+  }
   if (t.nblk == 0) {   // no position in this leaf: mark it empty
     if (valid) a.attn_ml[ob] = make_float2(-INFINITY, 0.f);
     return true;
@@ -141,19 +149,24 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
   const uint32_t tq = tmem_base + ((uint32_t)(q * 32) << 16);
   {
     const size_t so = ((size_t)(t.r_beg + j) * a.Hq + t.kh * t.G + gq) * HD;
+    // all loads of both planes are issued before the first use: one round trip to L2, where the previous kernel has
+    // just written the rows
+    const uint4 *src0 = reinterpret_cast<const uint4 *>(a.q + so), *src1 = reinterpret_cast<const uint4 *>(a.q_lo + so);
+    uint4 v[2][CH];
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+      v[0][c] = valid ? src0[c] : make_uint4(0u, 0u, 0u, 0u);
+      v[1][c] = valid ? src1[c] : make_uint4(0u, 0u, 0u, 0u);
+    }
 #pragma unroll
     for (int pl = 0; pl < 2; ++pl) {
-      const uint4 *src = reinterpret_cast<const uint4 *>((pl ? a.q_lo : a.q) + so);
-      uint4 v[CH];
-#pragma unroll
-      for (int c = 0; c < CH; ++c) v[c] = valid ? src[c] : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
       for (int c4 = 0; c4 < CH / 4; ++c4) {
         uint32_t r[16];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          r[4 * e] = v[4 * c4 + e].x; r[4 * e + 1] = v[4 * c4 + e].y;
-          r[4 * e + 2] = v[4 * c4 + e].z; r[4 * e + 3] = v[4 * c4 + e].w;
+          r[4 * e] = v[pl][4 * c4 + e].x; r[4 * e + 1] = v[pl][4 * c4 + e].y;
+          r[4 * e + 2] = v[pl][4 * c4 + e].z; r[4 * e + 3] = v[pl][4 * c4 + e].w;
         }
         tmem_st16(tq + kColQ + pl * (HD / 2) + c4 * 16, r);
       }
@@ -167,7 +180,6 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
   // Visibility: the whole cache, and of the chunk the rows named by this row's mask (itself and its ancestors in
   // the draft tree; in a chain, rows 0..j), up to the end of this split.
   const int lim_all = min(t.len, t.pos_end) - 1;   // every row sees every position up to here
-  const unsigned long long anc = ((unsigned long long)a.in.anc[2 * (t.r_beg + j) + 1] << 32) | a.in.anc[2 * (t.r_beg + j)];
   const float scale = rsqrtf((float)HD) * 1.4426950408889634f;
   // The output sums stay in tensor memory: every product P V adds to them.  Probabilities are taken against a
   // reference maximum m_ref that follows the running maximum lazily: only when a block's maximum exceeds it by
@@ -465,15 +477,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
   } else {
     // ---------------------------------------------------------------- workers
     uint32_t blk = 0;
-    pdl_wait();   // the rotated queries come from the previous kernel
-    if (threadIdx.x == kWorkerWarp0 * 32) stamp_waited(a.stamp);
-    bool ok = true;
+    bool ok = true, waited = false;
     for (int j = 0; j * (int)gridDim.x < n_total && ok; ++j) {
       const int u = attn_unit_of((int)blockIdx.x, j, (int)gridDim.x);
       if (u >= n_total) continue;
       const AttnUnit t = attn_unit_info(a, u);
-      ok = attn_unit_workers<HD>(a, ctl, t, tmem_base, warp & 3, lane, (int)threadIdx.x - kWorkerWarp0 * 32, blk, err);
+      ok = attn_unit_workers<HD>(a, ctl, t, tmem_base, warp & 3, lane, (int)threadIdx.x - kWorkerWarp0 * 32, blk, waited, err);
     }
+    if (!waited) pdl_wait();
   }
   tc_fence_before();
   __syncthreads();
