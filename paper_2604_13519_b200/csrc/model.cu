@@ -321,6 +321,26 @@ int pick_splits(const ts_model *m, int n_tiles, int m_chunks, int n_kblocks, boo
   return best;
 }
 
+// split-K factor of the many-rows kernel (one CTA per SM, 128 x 256 output tile per CTA).  A CTA there costs about
+// 13 k-blocks' worth of time besides its k-blocks (set-up, the first loads, 128 KB of partial sums written out), and
+// every slice adds a slab of partial sums that the next kernel reads back: take the factor with the smallest
+//   waves * (k-blocks per CTA + 13) + 2.5 * slices
+// (measured on the 8B shape with 256 rows: 9 slices of 7 k-blocks in two waves took 29.5 us for the O projection,
+// 4 slices of 16 in one wave 21 us, and the norm after it reads 4 slabs instead of 9).
+int pick_splits_rows(const ts_model *m, int n_tiles, int m_chunks, int n_kblocks, bool allow) {
+  if (!allow) return 1;
+  const int ctas = std::max(1, n_tiles * m_chunks);
+  const int s_max = std::max(1, std::min(kMaxSplits, n_kblocks / 4));
+  int best = 1;
+  double best_cost = 1e30;
+  for (int s = 1; s <= s_max; ++s) {
+    const int waves = (ctas * s + m->n_sms - 1) / m->n_sms;
+    const double cost = waves * ((double)n_kblocks / s + 13.0) + 2.5 * s;
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
+  }
+  return best;
+}
+
 struct GemmPlan { int splits, kb_per_split; };
 
 ts_status run_gemm(ts_model *m, int epi, const CUtensorMap &tw, const CUtensorMap *ta4, int N, int K, int M,
@@ -333,7 +353,7 @@ ts_status run_gemm(ts_model *m, int epi, const CUtensorMap &tw, const CUtensorMa
   // tensor cores and the bytes per flop an SM pulls from L2 (row-major kernel, 256 weight rows per CTA, one CTA per SM)
   const bool many_rows = M > 64;
   const int m_chunks = (M + g.Mc - 1) / g.Mc;
-  int splits = many_rows ? pick_splits(m, ts::gemm_rows_tiles(N), m_chunks, g.n_kblocks, epi == ts::EPI_PARTIAL, 1)
+  int splits = many_rows ? pick_splits_rows(m, ts::gemm_rows_tiles(N), m_chunks, g.n_kblocks, epi == ts::EPI_PARTIAL)
                          : pick_splits(m, N / 128, m_chunks, g.n_kblocks, epi == ts::EPI_PARTIAL);
   g.kb_per_split = (g.n_kblocks + splits - 1) / splits;   // (the kernel cuts K into `splits` balanced runs)
   g.out = out; g.out_rows = m->L.rows_alloc;
