@@ -294,7 +294,7 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
 
   // ---- partial result of this split: un-normalised output, its reference maximum (log2 domain), sum -------
   {
-    float4 *dst = reinterpret_cast<float4 *>(a.attn_o + ob * HD);
+    float *dst = a.attn_o + ob * HD;
     if (valid) a.attn_ml[ob] = make_float2(m_ref, l_run);
 #pragma unroll
     for (int i = 0; i < HD / 32; ++i) {
@@ -302,14 +302,11 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
       tmem_ld16(tq + kColO + i * 32, r0);      // (warp-wide: rows past the tile's end read too, and write nothing)
       tmem_ld16(tq + kColO + i * 32 + 16, r1);
       tmem_wait_ld();
-      if (valid) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          dst[i * 8 + e] = make_float4(__uint_as_float(r0[4 * e]), __uint_as_float(r0[4 * e + 1]),
-                                       __uint_as_float(r0[4 * e + 2]), __uint_as_float(r0[4 * e + 3]));
-          dst[i * 8 + 4 + e] = make_float4(__uint_as_float(r1[4 * e]), __uint_as_float(r1[4 * e + 1]),
-                                           __uint_as_float(r1[4 * e + 2]), __uint_as_float(r1[4 * e + 3]));
-        }
+      if (valid) {   // whole 32-byte sectors per lane: the lanes of a warp write 32 different rows
+        st_global_v8(dst + i * 32, r0);
+        st_global_v8(dst + i * 32 + 8, r0 + 8);
+        st_global_v8(dst + i * 32 + 16, r1);
+        st_global_v8(dst + i * 32 + 24, r1 + 8);
       }
     }
   }

@@ -114,6 +114,13 @@ __device__ __forceinline__ void stamp_waited(unsigned long long *p) {
   if (p) { const unsigned long long t = global_timer_ns(); atomicMin(p + 1, t); atomicMax(p + 2, t); }
 }
 
+// 32 bytes (one whole sector) per lane in one store; `p` must be 32-byte aligned
+__device__ __forceinline__ void st_global_v8(float *p, const uint32_t *r) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
+
 // ---- programmatic dependent launch -------------------------------------------------------------------
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() {

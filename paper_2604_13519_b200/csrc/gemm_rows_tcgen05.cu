@@ -182,20 +182,21 @@ gemm_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
           for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
         } else {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) v[j] = 0.f;
+          for (int j = 0; j < 16; ++j) { v[j] = 0.f; r[j] = 0u; }
         }
         const int n = n0 + c0;
         if constexpr (EPI == EPI_PARTIAL) {
           if (row_ok) {
-            float4 *dst = reinterpret_cast<float4 *>(g.out + ((size_t)split * g.out_rows + m) * g.N + n);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            // (a row's 64 bytes as two whole 32-byte sectors: the lanes of a warp write 32 different rows)
+            float *dst = g.out + ((size_t)split * g.out_rows + m) * g.N + n;
+            st_global_v8(dst, r);
+            st_global_v8(dst + 8, r + 8);
           }
         } else if constexpr (EPI == EPI_LOGITS) {
           if (row_ok) {
-            float4 *dst = reinterpret_cast<float4 *>(g.out + (size_t)m * g.N + n);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            float *dst = g.out + (size_t)m * g.N + n;
+            st_global_v8(dst, r);
+            st_global_v8(dst + 8, r + 8);
 #pragma unroll
             for (int j = 0; j < 16; ++j)
               if (v[j] > best) { best = v[j]; best_n = n + j; }   // (ascending ids: a tie keeps the lower one)
