@@ -124,7 +124,6 @@ __device__ __forceinline__ uint32_t pack_h2(float x, float y) {
 template <int HD>
 __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *ctl, const AttnUnit &t, uint32_t tmem_base,
                                                   int q, int lane, int wtid, uint32_t &blk, bool &waited, const int *err) {
-  constexpr int CH = HD / 8;          // 16-byte chunks per row
   const int row = q * 32 + lane;      // row of the tile
   const int pr = t.row0 + row;        // packed row of the sequence
   const bool valid = row < t.rows_here;
@@ -151,23 +150,25 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
     const size_t so = ((size_t)(t.r_beg + j) * a.Hq + t.kh * t.G + gq) * HD;
     // all loads of both planes are issued before the first use: one round trip to L2, where the previous kernel has
     // just written the rows
-    const uint4 *src0 = reinterpret_cast<const uint4 *>(a.q + so), *src1 = reinterpret_cast<const uint4 *>(a.q_lo + so);
-    uint4 v[2][CH];
+    // (32 bytes per lane and load: the lanes of a warp read 32 different rows)
+    uint32_t v[2][HD / 2];
+    if (valid) {
 #pragma unroll
-    for (int c = 0; c < CH; ++c) {
-      v[0][c] = valid ? src0[c] : make_uint4(0u, 0u, 0u, 0u);
-      v[1][c] = valid ? src1[c] : make_uint4(0u, 0u, 0u, 0u);
+      for (int c = 0; c < HD / 16; ++c) {
+        ld_global_v8(a.q + so + c * 16, &v[0][c * 8]);
+        ld_global_v8(a.q_lo + so + c * 16, &v[1][c * 8]);
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < HD / 2; ++c) v[0][c] = v[1][c] = 0u;
     }
 #pragma unroll
     for (int pl = 0; pl < 2; ++pl) {
 #pragma unroll
-      for (int c4 = 0; c4 < CH / 4; ++c4) {
+      for (int c4 = 0; c4 < HD / 32; ++c4) {
         uint32_t r[16];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          r[4 * e] = v[pl][4 * c4 + e].x; r[4 * e + 1] = v[pl][4 * c4 + e].y;
-          r[4 * e + 2] = v[pl][4 * c4 + e].z; r[4 * e + 3] = v[pl][4 * c4 + e].w;
-        }
+        for (int e = 0; e < 16; ++e) r[e] = v[pl][c4 * 16 + e];
         tmem_st16(tq + kColQ + pl * (HD / 2) + c4 * 16, r);
       }
     }

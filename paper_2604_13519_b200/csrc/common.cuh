@@ -121,6 +121,14 @@ __device__ __forceinline__ void st_global_v8(float *p, const uint32_t *r) {
                : "memory");
 }
 
+// 32 bytes per lane in one load; `p` must be 32-byte aligned
+__device__ __forceinline__ void ld_global_v8(const void *p, uint32_t *r) {
+  asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "l"(p)
+               : "memory");
+}
+
 // ---- programmatic dependent launch -------------------------------------------------------------------
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() {

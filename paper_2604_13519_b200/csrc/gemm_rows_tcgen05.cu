@@ -171,6 +171,7 @@ gemm_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
     float best = -INFINITY;
     int best_n = 0;
+    __align__(16) __nv_bfloat16 hi16[16], lo16[16];   // EPI_SWIGLU: the features of two iterations
     if (ok) {
       for (int c0 = 0; c0 < nb; c0 += 16) {
         uint32_t r[16];
@@ -202,17 +203,23 @@ gemm_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
               if (v[j] > best) { best = v[j]; best_n = n + j; }   // (ascending ids: a tie keeps the lower one)
           }
         } else {  // EPI_SWIGLU: even feature = gate_f, odd = up_f, f = n / 2
-          const int F = g.N >> 1, f = n >> 1;
-          __nv_bfloat16 hi[8], lo[8];
+          // 16 accumulator columns give 8 features = 16 bytes per plane; two iterations are put together so that a
+          // lane writes a whole 32-byte sector (nb is a multiple of 32)
+          const int F = g.N >> 1;
+          const int half = (c0 >> 4) & 1;
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const float gate = v[2 * j], up = v[2 * j + 1];
-            split_bf16(gate / (1.f + __expf(-gate)) * up, hi[j], lo[j]);
+            __nv_bfloat16 h, l;
+            split_bf16(gate / (1.f + __expf(-gate)) * up, h, l);
+            if (half == 0) { hi16[j] = h; lo16[j] = l; } else { hi16[8 + j] = h; lo16[8 + j] = l; }
           }
-          if (row_ok) {
-            *reinterpret_cast<uint4 *>(g.act_out + (size_t)m * F + f) = *reinterpret_cast<uint4 *>(hi);
+          if (half == 1 && row_ok) {
+            const int f = (n - 16) >> 1;
+            st_global_v8(reinterpret_cast<float *>(g.act_out + (size_t)m * F + f), reinterpret_cast<const uint32_t *>(hi16));
             if (g.out_planes == 2)
-              *reinterpret_cast<uint4 *>(g.act_out + ((size_t)g.act_rows + m) * F + f) = *reinterpret_cast<uint4 *>(lo);
+              st_global_v8(reinterpret_cast<float *>(g.act_out + ((size_t)g.act_rows + m) * F + f),
+                           reinterpret_cast<const uint32_t *>(lo16));
           }
         }
       }
