@@ -493,51 +493,79 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
   if (threadIdx.x == 0 && a.stamp) stamp_max(a.stamp + 3);
 }
 
-// grid = (M, Hq), hd threads: add the leaves of one (row, query head) and emit the normalised row as bf16 (hi[, lo]).
-// The row's sequence has n_leaves = ceil((cached length + chunk rows) / leaf_len) leaves, all of them written (a
-// leaf the row cannot see carries sum 0 and gets weight 0).  Lane s of each warp turns leaf s's (max, sum) into a
-// weight; every thread loads its output element of all leaves at once (one round trip to L2) and adds them in leaf
-// order.  NS = compile-time bound on the number of leaves.
-template <int NS>
+// grid = (M, Hq / 4), 4 warps: a warp adds the leaves of one (row, query head) and emits the normalised row as bf16
+// (hi[, lo]); lane i owns hd / 32 consecutive elements.  The row's sequence has n_leaves = ceil((cached length +
+// chunk rows) / leaf_len) leaves, all of them written (a leaf the row cannot see carries sum 0 and gets weight 0).
+// Lane s turns leaf s's (max, sum) into a weight; every lane loads its elements of all leaves at once (one round trip
+// to L2, 16 bytes per lane and leaf) and adds them in leaf order.  NS = compile-time bound on the number of leaves.
+template <int NS, int VW>
 __global__ void attn_merge_kernel(const AttnTcArgs a) {
   if (threadIdx.x == 0) stamp_min(a.stamp_merge);
   pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
-  const int m = blockIdx.x, h = blockIdx.y, d = threadIdx.x, lane = threadIdx.x & 31;
+  const int m = blockIdx.x, h = blockIdx.y * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   const int nl = a.in.row_leaves[m];   // (a step input, on the device before the step's first kernel)
   pdl_wait();
   if (threadIdx.x == 0) stamp_waited(a.stamp_merge);
+  if (h >= a.Hq) return;
   const size_t base = ((size_t)m * a.Hq + h) * a.n_slots;
   const float2 ml = lane < nl ? a.attn_ml[base + lane] : make_float2(-INFINITY, 0.f);
-  float t[NS];
+  float t[NS][VW];
 #pragma unroll
-  for (int s = 0; s < NS; ++s) t[s] = (s < nl) ? a.attn_o[(base + s) * a.hd + d] : 0.f;
+  for (int s = 0; s < NS; ++s) {
+    if (s < nl) {
+      const float *src = a.attn_o + (base + s) * a.hd + lane * VW;
+      if constexpr (VW == 4) {
+        const float4 v = *reinterpret_cast<const float4 *>(src);
+        t[s][0] = v.x; t[s][1] = v.y; t[s][2] = v.z; t[s][3] = v.w;
+      } else {
+        const float2 v = *reinterpret_cast<const float2 *>(src);
+        t[s][0] = v.x; t[s][1] = v.y;
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < VW; ++e) t[s][e] = 0.f;
+    }
+  }
   float mx = ml.y > 0.f ? ml.x : -INFINITY;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
   float w = ml.y > 0.f ? exp2f(ml.x - mx) : 0.f;
   // the denominator: leaf by leaf in leaf order (a shuffle tree would pair lanes differently as leaves are added)
-  float den = 0.f, num = 0.f;
+  float den = 0.f, num[VW];
+#pragma unroll
+  for (int e = 0; e < VW; ++e) num[e] = 0.f;
 #pragma unroll
   for (int s = 0; s < NS; ++s) {
     const float ws = __shfl_sync(0xffffffffu, w, s);
     const float ls = __shfl_sync(0xffffffffu, ml.y, s);
-    if (ws != 0.f) { den += ws * ls; num += ws * t[s]; }
+    if (ws != 0.f) {
+      den += ws * ls;
+#pragma unroll
+      for (int e = 0; e < VW; ++e) num[e] += ws * t[s][e];
+    }
   }
-  num *= 1.f / den;
-  __nv_bfloat16 hi, lo;
-  split_bf16(num, hi, lo);
-  const size_t col = (size_t)h * a.hd + d;
+  const float inv = 1.f / den;
+  __align__(8) __nv_bfloat16 hi[VW], lo[VW];
+#pragma unroll
+  for (int e = 0; e < VW; ++e) split_bf16(num[e] * inv, hi[e], lo[e]);
+  const size_t col = (size_t)h * a.hd + lane * VW;
   const size_t ld = (size_t)a.Hq * a.hd;
-  a.out[(size_t)m * ld + col] = hi;
-  if (a.planes == 2) a.out[((size_t)a.out_rows + m) * ld + col] = lo;
+  __nv_bfloat16 *o_hi = a.out + (size_t)m * ld + col, *o_lo = a.out + ((size_t)a.out_rows + m) * ld + col;
+  if constexpr (VW == 4) {
+    *reinterpret_cast<uint2 *>(o_hi) = *reinterpret_cast<const uint2 *>(hi);
+    if (a.planes == 2) *reinterpret_cast<uint2 *>(o_lo) = *reinterpret_cast<const uint2 *>(lo);
+  } else {
+    *reinterpret_cast<uint32_t *>(o_hi) = *reinterpret_cast<const uint32_t *>(hi);
+    if (a.planes == 2) *reinterpret_cast<uint32_t *>(o_lo) = *reinterpret_cast<const uint32_t *>(lo);
+  }
   if (threadIdx.x == 0 && a.stamp_merge) stamp_max(a.stamp_merge + 3);
 }
 
 template <typename K>
 static cudaError_t launch_merge_pdl(K kernel, const AttnTcArgs &a, cudaStream_t st) {
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(a.in.M, a.Hq);
-  cfg.blockDim = dim3(a.hd);
+  cfg.gridDim = dim3(a.in.M, (a.Hq + 3) / 4);
+  cfg.blockDim = dim3(128);
   cfg.stream = st;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -549,11 +577,18 @@ static cudaError_t launch_merge_pdl(K kernel, const AttnTcArgs &a, cudaStream_t 
 
 cudaError_t launch_attention_tc_merge(const AttnTcArgs &a, cudaStream_t st) {
   if (a.n_slots < 1 || a.n_slots > kAttnMaxSplits) return cudaErrorInvalidValue;
-  if (a.n_slots <= 2) return launch_merge_pdl(attn_merge_kernel<2>, a, st);
-  if (a.n_slots <= 4) return launch_merge_pdl(attn_merge_kernel<4>, a, st);
-  if (a.n_slots <= 8) return launch_merge_pdl(attn_merge_kernel<8>, a, st);
-  if (a.n_slots <= 16) return launch_merge_pdl(attn_merge_kernel<16>, a, st);
-  return launch_merge_pdl(attn_merge_kernel<32>, a, st);
+  if (a.hd == 128) {
+    if (a.n_slots <= 2) return launch_merge_pdl(attn_merge_kernel<2, 4>, a, st);
+    if (a.n_slots <= 4) return launch_merge_pdl(attn_merge_kernel<4, 4>, a, st);
+    if (a.n_slots <= 8) return launch_merge_pdl(attn_merge_kernel<8, 4>, a, st);
+    if (a.n_slots <= 16) return launch_merge_pdl(attn_merge_kernel<16, 4>, a, st);
+    return launch_merge_pdl(attn_merge_kernel<32, 4>, a, st);
+  }
+  if (a.n_slots <= 2) return launch_merge_pdl(attn_merge_kernel<2, 2>, a, st);
+  if (a.n_slots <= 4) return launch_merge_pdl(attn_merge_kernel<4, 2>, a, st);
+  if (a.n_slots <= 8) return launch_merge_pdl(attn_merge_kernel<8, 2>, a, st);
+  if (a.n_slots <= 16) return launch_merge_pdl(attn_merge_kernel<16, 2>, a, st);
+  return launch_merge_pdl(attn_merge_kernel<32, 2>, a, st);
 }
 
 static size_t attn_tc_smem(int hd) {

@@ -135,6 +135,8 @@ __device__ __forceinline__ __half to_half_sat(float x) {
   return __float2half_rn(fminf(fmaxf(x, -65504.f), 65504.f));
 }
 
+static constexpr int kRopeWideRows = 128;   // steps of at least this many rows take the wide kernel (no faster below)
+
 // grid = (M, Hq + 2*Hkv); one CTA of hd/2 threads per (row, head).  Thread i handles the rotary pair
 // (i, i + hd/2) of q or k heads, or elements (i, i + hd/2) of a v head.  Every load is issued before the first use
 // (the slabs, the row's position, sequence and slot): the kernel is two round trips to L2, not one per slab.
@@ -188,9 +190,91 @@ __global__ void rope_kv_kernel(StepIn in, const float *part, int n_splits, int p
   if (threadIdx.x == 0) stamp_max(stamp ? stamp + 3 : nullptr);
 }
 
+// The same for steps of many rows: grid = (M, ceil(heads / 16)), block = (hd / 8, 16): a thread handles FOUR
+// neighbouring rotary pairs of one head (32 bytes per slab in one load, 8-byte stores), so a 256-row step is 768 CTAs
+// of 256 threads instead of 12 288 CTAs of 64 -- less than one wave of resident threads instead of nearly three.  The
+// sums are taken in the same order as above: the results are the same bits.
+__global__ void rope_kv_wide_kernel(StepIn in, const float *part, int n_splits, int part_rows, int Hq, int Hkv, int hd,
+                                    const float2 *rope_tab, __half *q_out, __half *q_lo_out, __half *k_pages,
+                                    __half *v_pages, unsigned long long *stamp) {
+  if (threadIdx.x == 0 && threadIdx.y == 0) stamp_min(stamp);
+  pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
+  const int m = blockIdx.x, head = blockIdx.y * blockDim.y + threadIdx.y, i0 = 4 * threadIdx.x, half = hd >> 1;
+  const int n_heads = Hq + 2 * Hkv, N = n_heads * hd;
+  const bool live = head < n_heads;
+  // the step's integer inputs were copied in before the step's first kernel: they may be read before the wait
+  const int pos = in.pos[m], seq = in.row_seq[m], slot = in.slot[m];
+  const int page = (live && head >= Hq) ? in.block_tab[(size_t)seq * in.pages_per_seq + (slot >> 4)] : 0;
+  float2 cs[4] = {make_float2(1.f, 0.f), make_float2(1.f, 0.f), make_float2(1.f, 0.f), make_float2(1.f, 0.f)};
+  if (live && head < Hq + Hkv) {
+    const float4 *t = reinterpret_cast<const float4 *>(rope_tab + (size_t)pos * half + i0);
+    const float4 t0 = t[0], t1 = t[1];
+    cs[0] = make_float2(t0.x, t0.y); cs[1] = make_float2(t0.z, t0.w);
+    cs[2] = make_float2(t1.x, t1.y); cs[3] = make_float2(t1.z, t1.w);
+  }
+  pdl_wait();
+  if (threadIdx.x == 0 && threadIdx.y == 0) stamp_waited(stamp);
+  if (live) {
+    // the QKV weight rows are stored with rotary partners adjacent: feature 2i = element i, 2i+1 = element i + hd/2
+    const int col = head * hd + 2 * i0;
+    float4 p[kNormMaxSplits][2];
+#pragma unroll
+    for (int s = 0; s < kNormMaxSplits; ++s)
+      if (s < n_splits) {
+        const float4 *src = reinterpret_cast<const float4 *>(part + ((size_t)s * part_rows + m) * N + col);
+        p[s][0] = src[0];
+        p[s][1] = src[1];
+      }
+    float a[4] = {0.f, 0.f, 0.f, 0.f}, b[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int s = 0; s < kNormMaxSplits; ++s)
+      if (s < n_splits) {
+        a[0] += p[s][0].x; b[0] += p[s][0].y; a[1] += p[s][0].z; b[1] += p[s][0].w;
+        a[2] += p[s][1].x; b[2] += p[s][1].y; a[3] += p[s][1].z; b[3] += p[s][1].w;
+      }
+    if (head < Hq + Hkv) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float ra = a[j] * cs[j].x - b[j] * cs[j].y;
+        const float rb = b[j] * cs[j].x + a[j] * cs[j].y;
+        a[j] = ra; b[j] = rb;
+      }
+    }
+    __align__(8) __half ha[4], hb[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { ha[j] = to_half_sat(a[j]); hb[j] = to_half_sat(b[j]); }
+    if (head < Hq) {
+      // the query as an fp16 pair (value, rounding remainder), as in rope_kv_kernel
+      const size_t qo = ((size_t)m * Hq + head) * hd + i0;
+      *reinterpret_cast<uint2 *>(q_out + qo) = *reinterpret_cast<const uint2 *>(ha);
+      *reinterpret_cast<uint2 *>(q_out + qo + half) = *reinterpret_cast<const uint2 *>(hb);
+      if (q_lo_out) {
+        __align__(8) __half la[4], lb[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          la[j] = __float2half_rn(fabsf(a[j]) <= 65504.f ? a[j] - __half2float(ha[j]) : 0.f);
+          lb[j] = __float2half_rn(fabsf(b[j]) <= 65504.f ? b[j] - __half2float(hb[j]) : 0.f);
+        }
+        *reinterpret_cast<uint2 *>(q_lo_out + qo) = *reinterpret_cast<const uint2 *>(la);
+        *reinterpret_cast<uint2 *>(q_lo_out + qo + half) = *reinterpret_cast<const uint2 *>(lb);
+      }
+    } else {
+      const bool is_k = head < Hq + Hkv;
+      const int kh = is_k ? head - Hq : head - Hq - Hkv;
+      __half *dst = (is_k ? k_pages : v_pages) + (((size_t)page * Hkv + kh) * 16 + (slot & 15)) * hd + i0;
+      *reinterpret_cast<uint2 *>(dst) = *reinterpret_cast<const uint2 *>(ha);
+      *reinterpret_cast<uint2 *>(dst + half) = *reinterpret_cast<const uint2 *>(hb);
+    }
+  }
+  if (threadIdx.x == 0 && threadIdx.y == 0) stamp_max(stamp ? stamp + 3 : nullptr);
+}
+
 cudaError_t launch_rope_kv(const StepIn &in, const float *part, int n_splits, int part_rows, int Hq, int Hkv,
                            int hd, const float2 *rope_tab, __half *q_out, __half *q_lo_out, __half *k_pages,
                            __half *v_pages, cudaStream_t st, unsigned long long *stamp) {
+  if (in.M >= kRopeWideRows && hd % 8 == 0)
+    return launch_pdl(rope_kv_wide_kernel, dim3(in.M, (Hq + 2 * Hkv + 15) / 16), dim3(hd / 8, 16), 0, st, in, part,
+                      n_splits, part_rows, Hq, Hkv, hd, rope_tab, q_out, q_lo_out, k_pages, v_pages, stamp);
   return launch_pdl(rope_kv_kernel, dim3(in.M, Hq + 2 * Hkv), dim3(hd / 2), 0, st, in, part, n_splits,
                     part_rows, Hq, Hkv, hd, rope_tab, q_out, q_lo_out, k_pages, v_pages, stamp);
 }
