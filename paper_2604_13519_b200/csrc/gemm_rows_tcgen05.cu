@@ -9,7 +9,8 @@
 // is what sets the pace.  The weight matrix keeps its storage (contiguous 128 x 64 blocks, one TMA box each): a CTA's
 // 256 weight rows are two such boxes.  One CTA per SM (three 64 KB stages).
 //
-// Roles: warp 0 = TMA producer, warp 1 = TMEM allocation + MMA issue, warps 2..5 = epilogue (thread <-> row).
+// Roles: warp 0 = TMA producer, warp 1 = TMEM allocation + MMA issue, warps 2..9 = epilogue (thread <-> row, two
+// warps per row quarter, half of the columns each).
 // Every wait is bounded; on expiry the CTA records an error word and leaves through the normal exit.
 #include <algorithm>
 #include <functional>
@@ -38,7 +39,7 @@ struct __align__(8) RowsSmemCtl {
 };
 
 template <int EPI>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(320, 1)
 gemm_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_a,
                  const GemmArgs g) {
   extern __shared__ uint8_t smem_raw[];
@@ -156,7 +157,7 @@ gemm_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
       umma_commit(smem_u32(&ctl->tmem_full));
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5): thread <-> row
+    // ------------------------------------------------------------------ epilogue (warps 2..9): thread <-> row
     pdl_wait();   // outputs of this kernel may still be read by the previous one's consumers
     bool ok = true;
     if (nkb > 0) {
@@ -171,56 +172,97 @@ gemm_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
     float best = -INFINITY;
     int best_n = 0;
-    __align__(16) __nv_bfloat16 hi16[16], lo16[16];   // EPI_SWIGLU: the features of two iterations
+    // Results leave through shared memory so that global stores are whole lines: a thread owns a ROW of the
+    // accumulator, so storing from registers makes the 32 lanes of a warp write 32 different lines per instruction
+    // (4 us for the 128 KB of a tile).  Each warp stages 32 rows x 128 bytes (16-byte chunks, slot = chunk ^ (row & 7):
+    // conflict-free both ways) in the ring's shared memory -- free by now: every load was consumed by a product that
+    // has completed -- and writes them back 4 rows x 128 bytes per instruction.
+    // Eight epilogue warps: warps 2..5 take the first half of the tile's columns, warps 6..9 the second (two warps
+    // per tensor-memory lane quarter).
+    const int eh = (warp - 2) >> 2, c_beg = eh * (nb >> 1), c_end = c_beg + (nb >> 1);
+    const uint32_t stg = smem_u32(smem) + (warp - 2) * 4096;
+    const int rr = lane >> 3, slot = lane & 7;   // read-back: rows rr, rr + 4, ...; 16-byte slot of the row
     if (ok) {
-      for (int c0 = 0; c0 < nb; c0 += 16) {
-        uint32_t r[16];
-        float v[16];
-        if (nkb > 0) {
-          tmem_ld16(taddr + c0, r);     // (warp-wide: rows past the end read too, and write nothing)
-          tmem_wait_ld();
+      if constexpr (EPI != EPI_SWIGLU) {
+        for (int c0 = c_beg; c0 < c_end; c0 += 32) {
+          uint32_t r[32];
+          if (nkb > 0) {
+            tmem_ld16(taddr + c0, *reinterpret_cast<uint32_t(*)[16]>(r));     // (warp-wide: rows past the end read too)
+            tmem_ld16(taddr + c0 + 16, *reinterpret_cast<uint32_t(*)[16]>(r + 16));
+            tmem_wait_ld();
+          } else {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
-        } else {
+            for (int j = 0; j < 32; ++j) r[j] = 0u;
+          }
+          const int n = n0 + c0;
+          if constexpr (EPI == EPI_LOGITS) {
+            if (row_ok) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) { v[j] = 0.f; r[j] = 0u; }
+              for (int j = 0; j < 32; ++j) {
+                const float v = __uint_as_float(r[j]);
+                if (v > best) { best = v; best_n = n + j; }   // (ascending ids: a tie keeps the lower one)
+              }
+            }
+          }
+#pragma unroll
+          for (int c = 0; c < 8; ++c)
+            st_shared_v4(stg + lane * 128 + ((c ^ (lane & 7)) << 4), r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int R = i * 4 + rr, mr = m0 + q * 32 + R;
+            const uint4 v = ld_shared_v4(stg + R * 128 + ((slot ^ (R & 7)) << 4));
+            if (mr < g.M) {
+              float *dst = (EPI == EPI_PARTIAL ? g.out + ((size_t)split * g.out_rows + mr) * g.N : g.out + (size_t)mr * g.N) + n + slot * 4;
+              *reinterpret_cast<uint4 *>(dst) = v;
+            }
+          }
+          __syncwarp();
         }
-        const int n = n0 + c0;
-        if constexpr (EPI == EPI_PARTIAL) {
-          if (row_ok) {
-            // (a row's 64 bytes as two whole 32-byte sectors: the lanes of a warp write 32 different rows)
-            float *dst = g.out + ((size_t)split * g.out_rows + m) * g.N + n;
-            st_global_v8(dst, r);
-            st_global_v8(dst + 8, r + 8);
-          }
-        } else if constexpr (EPI == EPI_LOGITS) {
-          if (row_ok) {
-            float *dst = g.out + (size_t)m * g.N + n;
-            st_global_v8(dst, r);
-            st_global_v8(dst + 8, r + 8);
+      } else {
+        // EPI_SWIGLU: even feature = gate_f, odd = up_f, f = n / 2.  64 accumulator columns give 32 features: 64 bytes
+        // of the value plane (slots 0..3 of the staged row) and 64 of the remainder plane (slots 4..7).
+        const int F = g.N >> 1;
+        for (int c0 = c_beg; c0 < c_end; c0 += 64) {
+          uint32_t hi[16], lo[16];   // 32 features per plane, two bf16 per word
 #pragma unroll
-            for (int j = 0; j < 16; ++j)
-              if (v[j] > best) { best = v[j]; best_n = n + j; }   // (ascending ids: a tie keeps the lower one)
-          }
-        } else {  // EPI_SWIGLU: even feature = gate_f, odd = up_f, f = n / 2
-          // 16 accumulator columns give 8 features = 16 bytes per plane; two iterations are put together so that a
-          // lane writes a whole 32-byte sector (nb is a multiple of 32)
-          const int F = g.N >> 1;
-          const int half = (c0 >> 4) & 1;
+          for (int part = 0; part < 4; ++part) {
+            uint32_t r[16];
+            if (nkb > 0) {
+              tmem_ld16(taddr + c0 + part * 16, r);
+              tmem_wait_ld();
+            } else {
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const float gate = v[2 * j], up = v[2 * j + 1];
-            __nv_bfloat16 h, l;
-            split_bf16(gate / (1.f + __expf(-gate)) * up, h, l);
-            if (half == 0) { hi16[j] = h; lo16[j] = l; } else { hi16[8 + j] = h; lo16[8 + j] = l; }
+              for (int j = 0; j < 16; ++j) r[j] = 0u;
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              __nv_bfloat16 h0, l0, h1, l1;
+              const float g0 = __uint_as_float(r[4 * j]), u0 = __uint_as_float(r[4 * j + 1]);
+              const float g1 = __uint_as_float(r[4 * j + 2]), u1 = __uint_as_float(r[4 * j + 3]);
+              split_bf16(g0 / (1.f + __expf(-g0)) * u0, h0, l0);
+              split_bf16(g1 / (1.f + __expf(-g1)) * u1, h1, l1);
+              hi[part * 4 + j] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+              lo[part * 4 + j] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+            }
           }
-          if (half == 1 && row_ok) {
-            const int f = (n - 16) >> 1;
-            st_global_v8(reinterpret_cast<float *>(g.act_out + (size_t)m * F + f), reinterpret_cast<const uint32_t *>(hi16));
-            if (g.out_planes == 2)
-              st_global_v8(reinterpret_cast<float *>(g.act_out + ((size_t)g.act_rows + m) * F + f),
-                           reinterpret_cast<const uint32_t *>(lo16));
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            st_shared_v4(stg + lane * 128 + ((c ^ (lane & 7)) << 4), hi[4 * c], hi[4 * c + 1], hi[4 * c + 2], hi[4 * c + 3]);
+            st_shared_v4(stg + lane * 128 + (((c + 4) ^ (lane & 7)) << 4), lo[4 * c], lo[4 * c + 1], lo[4 * c + 2], lo[4 * c + 3]);
           }
+          __syncwarp();
+          const int f = (n0 + c0) >> 1;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int R = i * 4 + rr, mr = m0 + q * 32 + R;
+            const uint4 v = ld_shared_v4(stg + R * 128 + ((slot ^ (R & 7)) << 4));
+            if (mr < g.M && (slot < 4 || g.out_planes == 2)) {
+              __nv_bfloat16 *dst = g.act_out + ((size_t)(slot < 4 ? 0 : g.act_rows) + mr) * F + f + (slot & 3) * 8;
+              *reinterpret_cast<uint4 *>(dst) = v;
+            }
+          }
+          __syncwarp();
         }
       }
       if constexpr (EPI == EPI_LOGITS) {
@@ -258,7 +300,7 @@ static cudaError_t launch_rows_one(const CUtensorMap &tw, const CUtensorMap &ta,
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = grid;
-  cfg.blockDim = dim3(192);
+  cfg.blockDim = dim3(320);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute at[1];
