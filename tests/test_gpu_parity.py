@@ -150,6 +150,31 @@ def test_ragged_batch():
     gm.close()
 
 
+@pytest.mark.parametrize("name", ["8b-2l", "1b-2l"])
+@pytest.mark.parametrize("ks", [[32, 32, 1], [40, 33, 30], [64, 64], [64, 64, 1], [64, 64, 64, 64], [33, 64, 64, 64, 64, 11]],
+                         ids=lambda ks: f"{sum(ks)}rows")
+def test_row_counts_around_the_projection_kernels_switch(name, ks):
+    """Steps of 65, 103, 128, 129, 256 and 300 rows: the first size past the weight-streaming projection kernel, one
+    partly filled 128-row chunk, exactly one chunk, one row into a second chunk, two full chunks (the case in which the
+    many-rows kernel mixes tile widths and cuts K by its cost model), and three chunks with a ragged last one."""
+    shape = synth.SHAPES[name]
+    lens = [70, 333, 1024, 129, 640, 17][:len(ks)]
+    om, gm = make_pair(shape, max_batch=len(ks), k_max=64, max_rows=sum(ks), max_ctx=1024 + 128)
+    sess, drafts, refs = [], [], []
+    for i, (n, k) in enumerate(zip(lens, ks)):
+        cache, s, pending = synthetic_context(shape, om, gm, n, stream=i, pending=300 + i)
+        draft = _rand_draft(shape.vocab, k - 1, 70 + i)
+        sess.append(s); drafts.append(draft)
+        refs.append(om.verify(pending, draft, cache, want_logits=True))
+    out = ts.ts_verify(gm, sess, drafts)
+    row = 0
+    for i, (res, ref) in enumerate(zip(out, refs)):
+        assert res.first_row == row and res.k == ks[i]
+        check_step(res, gm.read_logits(row, res.k), ref, f"{name}, {sum(ks)} rows, seq {i}")
+        row += res.k
+    gm.close()
+
+
 def test_sixteen_sessions_512_rows():
     """The largest step of the batched configuration: 16 sessions x k = 32 = 512 rows (four 128-row chunks in every
     projection, 16 attention row tiles), ragged contexts from a few tokens to two thousand."""
