@@ -873,12 +873,14 @@ ts_status ts_init_model(const ts_model_config *cfg, const ts_buffers *bufs, void
     // Attention leaf length.  A constant of the model, NOT of the step: a row's bits must not depend on the step's
     // shape.  Chosen so that a full batch at full context gives about one unit of work per SM -- groups = (sequence,
     // row tile, kv head) triples of a full step, leaves per group = 95% of the SMs / groups, at least 4 and at most
-    // kMaxAttnSplits -- in whole 64-position blocks: a batch-1 model gets many short leaves (its few groups must
+    // 16 -- in whole 64-position blocks: a batch-1 model gets many short leaves (its few groups must
     // cover the SMs), a batched one a few long ones (a leaf costs a fixed start-up and one partial result per row;
     // four per full-length sequence still let ragged batches be dealt out evenly over the SMs).
     const int G = c.n_q_heads / c.n_kv_heads;
     const int groups = c.max_batch * ((c.k_max * G + 127) / 128) * c.n_kv_heads;
-    const int want = std::max(4, std::min(kMaxAttnSplits, (int)(0.95 * m->n_sms) / std::max(1, groups)));
+    // (at most 16: the merge kernel is unrolled over 2, 4, 8, 16 or 32 leaves, and 17 leaves cost it a fifth more
+    // than 15 while the attention kernel gains nothing)
+    const int want = std::max(4, std::min(16, (int)(0.95 * m->n_sms) / std::max(1, groups)));
     const int blocks = (c.max_ctx + 63) / 64;
     int leaf_blocks = std::max(1, (blocks + want - 1) / want);
     while ((blocks + leaf_blocks - 1) / leaf_blocks > kMaxAttnSplits) ++leaf_blocks;
