@@ -10,8 +10,10 @@
 //            memory), then  O_blk = P V  with P read from tensor memory (fp16) and the V block read MN-major from
 //            the same [position][64 elements] image K uses
 //   warps 2..5  one row per thread: maximum over the block's 64 scores, P = exp2(S - reference maximum) written back
-//            to tensor memory as fp16.  The output sums stay in tensor memory (every P V adds to them); the
-//            reference maximum follows the running one in steps, and only then is the row of sums multiplied down
+//            to tensor memory as an fp16 (value, rounding remainder) pair -- the second product adds both, so the 11
+//            bits of fp16 do not limit the weights (a single fp16 P was the largest error of the whole step).  The
+//            output sums stay in tensor memory (every P V adds to them); the reference maximum follows the running
+//            one in steps, and only then is the row of sums multiplied down
 // Each leaf writes an un-normalised partial output with its (max, sum); attn_merge_kernel adds a row's leaves.
 // Every wait is bounded; on expiry the CTA records an error word and leaves through the normal exit.
 #include <cuda_fp16.h>
@@ -97,8 +99,9 @@ __device__ __forceinline__ AttnUnit attn_unit_info(const AttnTcArgs &a, int u) {
 
 // tensor-memory columns of the attention phase (they lie over the projection accumulators, which are idle then)
 static constexpr int kColS = 0;      // two score buffers of 64 columns
-static constexpr int kColP = 128;    // two probability buffers of 32 columns (fp16 pairs)
+static constexpr int kColP = 128;    // two probability buffers of 32 columns (fp16, two per column)
 static constexpr int kColO = 192;    // the output sums: head_dim columns, accumulated over the unit's blocks
+static constexpr int kColPL = 448;   // the probabilities' rounding remainders: two buffers of 32 columns
 static constexpr int kColQ = 320;    // the unit's queries, fp16 pairs: head_dim / 2 columns of values, then as many of remainders
 static constexpr float kRescaleStep = 8.f;   // the reference maximum follows the running one in steps of 2^8
 
@@ -243,7 +246,7 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
     if (raise) m_ref = m_blk;
     const float ref = (m_ref == -INFINITY) ? 0.f : m_ref;
     float sum0 = 0.f, sum1 = 0.f;
-    uint32_t pk0[16], pk1[16];
+    uint32_t pk0[16], pk1[16], pl0[16], pl1[16];
 #pragma unroll
     for (int e = 0; e < 16; ++e) {
       const float e0 = ex2_approx(fmaf(sc[2 * e], scale, -ref));
@@ -251,8 +254,11 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
       const float e2 = ex2_approx(fmaf(sc[32 + 2 * e], scale, -ref));
       const float e3 = ex2_approx(fmaf(sc[32 + 2 * e + 1], scale, -ref));
       sum0 += e0 + e2; sum1 += e1 + e3;
-      pk0[e] = pack_h2(e0, e1);
-      pk1[e] = pack_h2(e2, e3);
+      const __half2 h01 = __floats2half2_rn(e0, e1), h23 = __floats2half2_rn(e2, e3);
+      pk0[e] = *reinterpret_cast<const uint32_t *>(&h01);
+      pk1[e] = *reinterpret_cast<const uint32_t *>(&h23);
+      pl0[e] = pack_h2(e0 - __low2float(h01), e1 - __high2float(h01));
+      pl1[e] = pack_h2(e2 - __low2float(h23), e3 - __high2float(h23));
     }
     // This block's P buffer last fed product b - 2, which is complete: the scores of this block were committed after
     // it by the same thread, and a commit covers everything issued before it.  Only multiplying the sums down needs
@@ -282,6 +288,8 @@ __device__ __forceinline__ bool attn_unit_workers(const AttnTcArgs &a, AttnCtl *
     l_run = l_run * f + (sum0 + sum1);
     tmem_st16(tq + kColP + buf * 32, pk0);
     tmem_st16(tq + kColP + buf * 32 + 16, pk1);
+    tmem_st16(tq + kColPL + buf * 32, pl0);
+    tmem_st16(tq + kColPL + buf * 32 + 16, pl1);
     tmem_wait_st();
     tc_fence_before();
     __syncwarp();
@@ -418,10 +426,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         tc_fence_after();
         const uint32_t sV = sKV + vst * kKvBytes + kAttnBlk * HD * 2;
 #pragma unroll
-        for (int ks = 0; ks < kAttnBlk / 16; ++ks)   // 16 positions per instruction
+        for (int ks = 0; ks < kAttnBlk / 16; ++ks) {   // 16 positions per instruction: values, then remainders
           if (elect_one())
             umma_f16_ts(tmem_base + kColO, tmem_base + kColP + pb * 32 + ks * 8,
                         umma_desc_sw128_mn(sV + ks * 2048, kAttnBlk * 128), idesc_pv, (!first || ks != 0) ? 1u : 0u);
+          if (elect_one())
+            umma_f16_ts(tmem_base + kColO, tmem_base + kColPL + pb * 32 + ks * 8,
+                        umma_desc_sw128_mn(sV + ks * 2048, kAttnBlk * 128), idesc_pv, 1u);
+        }
         if (elect_one()) {
           umma_commit(smem_u32(&ctl->pv_done[pb]));
           umma_commit(smem_u32(&ctl->kv_empty[vst]));
