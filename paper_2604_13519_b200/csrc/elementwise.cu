@@ -280,7 +280,7 @@ cudaError_t launch_rope_kv(const StepIn &in, const float *part, int n_splits, in
 }
 
 // One CTA per source row; thread i moves 16 bytes.  Block (tile, kb) of the stored matrix starts at row
-// (tile * K/64 + kb) * 128 of a [.][64] array.
+// w_block(tile, kb) * 128 of a [.][64] array.
 __global__ void retile_kernel(const __nv_bfloat16 *src, int r0, int K, RowMap rm, __nv_bfloat16 *dst) {
   const int r = r0 + blockIdx.x;
   int row;
@@ -294,7 +294,7 @@ __global__ void retile_kernel(const __nv_bfloat16 *src, int r0, int K, RowMap rm
   const uint4 *s = reinterpret_cast<const uint4 *>(src + (size_t)blockIdx.x * K);
   for (int i = threadIdx.x; i < K / 8; i += blockDim.x) {
     const int kb = i >> 3, c = i & 7;
-    uint4 *d = reinterpret_cast<uint4 *>(dst + ((size_t)(tile * KB + kb) * 128 + rr) * 64) + c;
+    uint4 *d = reinterpret_cast<uint4 *>(dst + ((size_t)w_block(tile, kb, rm.tiles, KB) * 128 + rr) * 64) + c;
     *d = s[i];
   }
 }

@@ -595,8 +595,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_verify_kernel(const __grid_
             if (!ok) { atomicCAS(err, 0, DEV_TIMEOUT_EMPTY); break; }
             const uint32_t bar = smem_u32(&ctl->full[s]);
             mbar_expect_tx(bar, kWBytes);
-            // one block of the stored matrix = 16 contiguous KB = rows (tile * KB + kb) * 128 .. of a [.][64] array
-            tma_load_2d(smem_u32(smem + (size_t)s * stage_bytes), &a.maps[o.map_w], 0, (sg.tile * o.KB + kb) * kTileN, bar, pol_w);
+            // one block of the stored matrix = 16 contiguous KB = rows w_block(tile, kb) * 128 .. of a [.][64] array
+            tma_load_2d(smem_u32(smem + (size_t)s * stage_bytes), &a.maps[o.map_w], 0, w_block(sg.tile, kb, o.T, o.KB) * kTileN, bar, pol_w);
           }
         }
       }

@@ -93,12 +93,12 @@ gemm_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     // ------------------------------------------------------------------ producer
     if (lane == 0 && nkb > 0) {
       const uint64_t pol_w = policy_evict_first(), pol_a = policy_evict_last();
-      // block (128-row block j, k-block kb) of the stored matrix = rows (j * n_kblocks + kb) * 128 .. of a [.][64] array
+      // block (128-row block j, k-block kb) of the stored matrix = rows w_block(j, kb) * 128 .. of a [.][64] array
       auto load_w = [&](int s, int kb) {
         const uint32_t bar = smem_u32(&ctl->full[s]);
         const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes + a_bytes);
         for (int j = 0; j < nb / kBoxN; ++j)
-          tma_load_2d(dst + j * kBoxBytes, &tmap_w, 0, ((blk0 + j) * g.n_kblocks + kb) * kBoxN, bar, pol_w);
+          tma_load_2d(dst + j * kBoxBytes, &tmap_w, 0, w_block(blk0 + j, kb, g.N / kBoxN, g.n_kblocks) * kBoxN, bar, pol_w);
       };
       const int pre = min(g.stages, nkb);
       // weights do not depend on the previous kernel: start them before the programmatic-dependency wait

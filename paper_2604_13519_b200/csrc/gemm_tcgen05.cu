@@ -87,7 +87,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
       for (int it = 0; it < pre; ++it) {
         uint32_t bar = smem_u32(&ctl->full[it]);
         mbar_expect_tx(bar, stage_bytes);
-        tma_load_2d(smem_u32(smem + (size_t)it * stage_bytes), &tmap_w, 0, (blockIdx.x * g.n_kblocks + kb0 + it) * kTileN, bar, pol_w);
+        tma_load_2d(smem_u32(smem + (size_t)it * stage_bytes), &tmap_w, 0, w_block(blockIdx.x, kb0 + it, (g.N + kTileN - 1) / kTileN, g.n_kblocks) * kTileN, bar, pol_w);
       }
       pdl_wait();
       stamp_waited(g.stamp);
@@ -108,7 +108,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
         uint32_t bar = smem_u32(&ctl->full[s]);
         mbar_expect_tx(bar, stage_bytes);
         uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
-        tma_load_2d(dst, &tmap_w, 0, (blockIdx.x * g.n_kblocks + kb0 + it) * kTileN, bar, pol_w);
+        tma_load_2d(dst, &tmap_w, 0, w_block(blockIdx.x, kb0 + it, (g.N + kTileN - 1) / kTileN, g.n_kblocks) * kTileN, bar, pol_w);
         tma_load_3d(dst + kWBytes, &tmap_a, (kb0 + it) * kBlockK, m0, 0, bar, pol_a);
         if (++s == g.stages) { s = 0; ph ^= 1; }
       }

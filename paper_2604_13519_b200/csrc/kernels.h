@@ -187,7 +187,11 @@ cudaError_t launch_kv_compact(const CompactArgs &a, cudaStream_t st);
 
 // Where a source row of an uploaded matrix goes in the stored matrix: row r -> base + r * mul, or, with
 // hd != 0, base + (r / hd) * hd + p(r % hd) with p(e) = 2e for e < hd/2 and 2(e - hd/2) + 1 otherwise.
-struct RowMap { int base, mul, hd; };
+struct RowMap { int base, mul, hd, tiles; };   // tiles = 128-row blocks of the whole stored matrix
+// Index of block (128-row tile, 64-wide k-block) of a stored projection matrix, in units of 128 x 64 blocks: k-block
+// major, so that the CTAs of one launch, which walk the k-blocks of neighbouring tiles in step, read one contiguous
+// region of memory at a time instead of as many regions a tile's length apart as there are CTAs.
+__host__ __device__ inline int w_block(int tile, int kb, int tiles, int kblocks) { (void)kblocks; return kb * tiles + tile; }
 // Scatter n_rows source rows (row-major, K columns, first one being row r0 of the uploaded matrix) into the
 // 128 x 64-block storage of the stored matrix.
 cudaError_t launch_retile(const __nv_bfloat16 *src, int n_rows, int r0, int K, RowMap rm, __nv_bfloat16 *dst,

@@ -913,20 +913,20 @@ ts_status ts_load_tensor(ts_model *m, int32_t kind, int32_t layer, const void *h
   int64_t er = 0, ec = 0;
   uint8_t *dst = nullptr;
   size_t esz = 2;
-  ts::RowMap rm{0, 1, 0};
+  ts::RowMap rm{0, 1, 0, 0};
   switch (kind) {
     case TS_W_EMBED: er = c.vocab; ec = d; dst = m->W(L.embed); break;
-    case TS_W_LM_HEAD: er = c.vocab; ec = d; dst = m->W(L.lm_head); break;
+    case TS_W_LM_HEAD: er = c.vocab; ec = d; dst = m->W(L.lm_head); rm.tiles = (c.vocab + 127) / 128; break;
     case TS_W_FINAL_GAIN: er = 1; ec = d; dst = m->W(L.gf); esz = 4; break;
     case TS_W_GAIN1: er = 1; ec = d; dst = m->W(L.g1[layer]); esz = 4; break;
     case TS_W_GAIN2: er = 1; ec = d; dst = m->W(L.g2[layer]); esz = 4; break;
-    case TS_W_Q: er = Nq; ec = d; dst = m->W(L.wqkv[layer]); rm.base = 0; rm.hd = (int)hd; break;
-    case TS_W_K: er = Nkv; ec = d; dst = m->W(L.wqkv[layer]); rm.base = (int)Nq; rm.hd = (int)hd; break;
-    case TS_W_V: er = Nkv; ec = d; dst = m->W(L.wqkv[layer]); rm.base = (int)(Nq + Nkv); rm.hd = (int)hd; break;
-    case TS_W_O: er = d; ec = Nq; dst = m->W(L.wo[layer]); break;
-    case TS_W_GATE: er = F; ec = d; dst = m->W(L.wgu[layer]); rm.mul = 2; break;               // even rows
-    case TS_W_UP: er = F; ec = d; dst = m->W(L.wgu[layer]); rm.mul = 2; rm.base = 1; break;    // odd rows
-    case TS_W_DOWN: er = d; ec = F; dst = m->W(L.wd[layer]); break;
+    case TS_W_Q: er = Nq; ec = d; dst = m->W(L.wqkv[layer]); rm.base = 0; rm.hd = (int)hd; rm.tiles = L.Nqkv / 128; break;
+    case TS_W_K: er = Nkv; ec = d; dst = m->W(L.wqkv[layer]); rm.base = (int)Nq; rm.hd = (int)hd; rm.tiles = L.Nqkv / 128; break;
+    case TS_W_V: er = Nkv; ec = d; dst = m->W(L.wqkv[layer]); rm.base = (int)(Nq + Nkv); rm.hd = (int)hd; rm.tiles = L.Nqkv / 128; break;
+    case TS_W_O: er = d; ec = Nq; dst = m->W(L.wo[layer]); rm.tiles = (int)(d / 128); break;
+    case TS_W_GATE: er = F; ec = d; dst = m->W(L.wgu[layer]); rm.mul = 2; rm.tiles = (int)(2 * F / 128); break;               // even rows
+    case TS_W_UP: er = F; ec = d; dst = m->W(L.wgu[layer]); rm.mul = 2; rm.base = 1; rm.tiles = (int)(2 * F / 128); break;    // odd rows
+    case TS_W_DOWN: er = d; ec = F; dst = m->W(L.wd[layer]); rm.tiles = (int)(d / 128); break;
     default: return fail(TS_ERR_ARG, "unknown tensor kind %d", kind);
   }
   if (rows != er || cols != ec) return fail(TS_ERR_ARG, "tensor kind %d: expected %lld x %lld, got %lld x %lld", kind,
