@@ -129,32 +129,39 @@ gemm_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issue
-    if (lane == 0) {
+    // The whole warp walks the loop and the waits; one elected lane issues the instructions of a k-block and its commit.
+    {
       const uint32_t idesc = umma_idesc_bf16(kRowsM, (uint32_t)nb);
       bool ok = true;
       int s = 0;
       uint32_t ph = 0;
       for (int it = 0; it < nkb; ++it) {
-        if (!mbar_wait(smem_u32(&ctl->full[s]), ph)) {
-          atomicExch(g.err, DEV_TIMEOUT_FULL);
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl->full[s]), ph))) {   // (all lanes leave together)
+          if (lane == 0) atomicExch(g.err, DEV_TIMEOUT_FULL);
           ok = false;
           break;
         }
         tc_fence_after();
         const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
         const uint64_t db = umma_desc_sw128(sa + a_bytes);
-        // the value plane and the remainder plane of the activations into the same sums
-        for (int pl = 0; pl < g.planes; ++pl) {
-          const uint64_t da = umma_desc_sw128(sa + pl * (kRowsM * kBlockK * 2));
+        if (elect_one()) {
+          // the value plane and the remainder plane of the activations into the same sums
+          for (int pl = 0; pl < g.planes; ++pl) {
+            const uint64_t da = umma_desc_sw128(sa + pl * (kRowsM * kBlockK * 2));
 #pragma unroll
-          for (int kk = 0; kk < kBlockK / 16; ++kk)   // 16 bf16 along K = 32 bytes = 2 descriptor address units
-            umma_bf16(tmem_base, da + 2 * kk, db + 2 * kk, idesc, (it | kk | pl) != 0);
+            for (int kk = 0; kk < kBlockK / 16; ++kk)   // 16 bf16 along K = 32 bytes = 2 descriptor address units
+              umma_bf16(tmem_base, da + 2 * kk, db + 2 * kk, idesc, (it | kk | pl) != 0);
+          }
+          umma_commit(smem_u32(&ctl->empty[s]));
         }
-        umma_commit(smem_u32(&ctl->empty[s]));
+        __syncwarp();
         if (++s == g.stages) { s = 0; ph ^= 1; }
       }
-      if (!ok) ctl->abort_flag = 1;
-      umma_commit(smem_u32(&ctl->tmem_full));
+      if (elect_one()) {
+        if (!ok) ctl->abort_flag = 1;
+        umma_commit(smem_u32(&ctl->tmem_full));
+      }
+      __syncwarp();
     }
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..9): thread <-> row
