@@ -47,7 +47,10 @@ enum {
   TS_ERR_TOKEN_RANGE = -5,    /* token id outside [0, vocab) */
   TS_ERR_DEVICE_TIMEOUT = -6, /* a bounded device-side wait expired; the context stays usable */
   TS_ERR_CUDA = -7,           /* CUDA runtime/driver error, or no device */
-  TS_ERR_UNIMPLEMENTED = -8
+  TS_ERR_UNIMPLEMENTED = -8,
+  TS_ERR_DEVICE_BOUNDS = -9   /* debug build of the library only (compiled with TS_DEBUG_BOUNDS): a kernel found an index
+                                 from the step's inputs outside its range and skipped the access; the context stays
+                                 usable */
 };
 
 typedef struct ts_model ts_model;
@@ -392,8 +395,9 @@ ts_status ts_debug_timeline(ts_model *m, uint64_t *stamps, int32_t *classes, int
 /* Make the NEXT step (ts_verify*, ts_prefill chunk) report `code` (> 0) in its device status word, as a bounded
  * device-side wait that expired would: the word is written on the model's stream after the step's last kernel and
  * before the results are read back, so no kernel sees it and nothing is left waiting.  That step then fails with
- * TS_ERR_DEVICE_TIMEOUT, the library clears the word and the persistent kernel's counters, and later steps run
- * normally.  For testing the host's handling of a device timeout without making a GPU wait. */
+ * TS_ERR_DEVICE_TIMEOUT (codes below 64) or TS_ERR_DEVICE_BOUNDS (64 + the number of a debug-build index check), the
+ * library clears the word and the persistent kernel's counters, and later steps run normally.  For testing the
+ * host's handling of a device timeout, or of a failed index check, without making a GPU wait or go out of range. */
 ts_status ts_debug_inject_device_error(ts_model *m, int32_t code);
 /* Counters: kernels launched since ts_init_model, bytes copied host->device and device->host by
  * ts_verify since then. */

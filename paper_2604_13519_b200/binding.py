@@ -10,6 +10,7 @@ from typing import List, Optional, Sequence
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libtoolspec.so")
+DEBUG_LIB_PATH = os.path.join(_HERE, "libtoolspec_dbg.so")   # built with every device-side index check compiled in
 
 TS_K_MAX = 64
 TS_PAGE_SIZE = 16
@@ -19,7 +20,7 @@ TS_TOPK = 8
 
 STATUS = {0: "TS_OK", -1: "TS_ERR_ARG", -2: "TS_ERR_STATE", -3: "TS_ERR_OOM_PAGES",
           -4: "TS_ERR_K_TOO_LARGE", -5: "TS_ERR_TOKEN_RANGE", -6: "TS_ERR_DEVICE_TIMEOUT",
-          -7: "TS_ERR_CUDA", -8: "TS_ERR_UNIMPLEMENTED"}
+          -7: "TS_ERR_CUDA", -8: "TS_ERR_UNIMPLEMENTED", -9: "TS_ERR_DEVICE_BOUNDS"}
 
 (TS_W_EMBED, TS_W_LM_HEAD, TS_W_FINAL_GAIN, TS_W_Q, TS_W_K, TS_W_V, TS_W_O, TS_W_GATE, TS_W_UP,
  TS_W_DOWN, TS_W_GAIN1, TS_W_GAIN2) = range(12)
@@ -135,6 +136,16 @@ _SIGNATURES = {
 EXPORTED = sorted(list(_SIGNATURES) + ["ts_last_error"])
 
 _lib = None
+
+
+def use_debug_library():
+    """Load the library's debug build (`python -m paper_2604_13519_b200.build --debug-bounds`) instead of the release
+    one: the same code with every index a kernel takes from the step's inputs checked on the device; a failed check
+    makes the step return TS_ERR_DEVICE_BOUNDS.  Has to be called before the library is first used in the process."""
+    global LIB_PATH
+    if _lib is not None:
+        raise RuntimeError("the library is already loaded")
+    LIB_PATH = DEBUG_LIB_PATH
 
 
 def lib():

@@ -86,6 +86,10 @@ __device__ __forceinline__ AttnUnit attn_unit_info(const AttnTcArgs &a, int u) {
   t.leaf = a.unit_leaf[pair];
   t.G = a.Hq / a.Hkv;
   t.seq = a.tile_seq[t.tile];
+  if (!ts_in_range(a.in.ck, CHK_UNIT, t.seq, a.in.B) || !ts_in_range(a.in.ck, CHK_UNIT, t.leaf, a.n_slots)) {
+    t.seq = 0;   // (debug build: the failed check is on record; go on with indices that are in range)
+    t.leaf = 0;
+  }
   t.row0 = a.tile_row0[t.tile];
   t.r_beg = a.in.cu_rows[t.seq];
   const int k_i = a.in.cu_rows[t.seq + 1] - t.r_beg;
@@ -390,7 +394,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
           for (int pg = 0; pg < kAttnBlk / 16; ++pg) {
             // a page past the unit's end is never visible; load the last visible page again instead
             const int pos = min(t.pos_beg + b * kAttnBlk + pg * 16, t.pos_end - 1);
-            const int page = btab[pos >> 4];
+            int page = btab[pos >> 4];
+            if (!ts_in_range(a.in.ck, CHK_PAGE_ATTN, page, a.in.ck.max_pages)) page = 0;
 #pragma unroll
             for (int hh = 0; hh < (int)kHalves; ++hh) {
               const uint32_t off = hh * (kAttnBlk * 128) + pg * 2048;
@@ -515,7 +520,8 @@ __global__ void attn_merge_kernel(const AttnTcArgs a) {
   if (threadIdx.x == 0) stamp_min(a.stamp_merge);
   pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
   const int m = blockIdx.x, h = blockIdx.y * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-  const int nl = a.in.row_leaves[m];   // (a step input, on the device before the step's first kernel)
+  int nl = a.in.row_leaves[m];   // (a step input, on the device before the step's first kernel)
+  if (!ts_in_range(a.in.ck, CHK_LEAVES, nl, a.n_slots + 1)) nl = 0;
   pdl_wait();
   if (threadIdx.x == 0) stamp_waited(a.stamp_merge);
   if (h >= a.Hq) return;

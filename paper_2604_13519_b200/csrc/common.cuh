@@ -8,7 +8,29 @@
 namespace ts {
 
 // error codes written to the device status word by bounded waits
-enum : int { DEV_OK = 0, DEV_TIMEOUT_FULL = 1, DEV_TIMEOUT_EMPTY = 2, DEV_TIMEOUT_TMEM = 3, DEV_TIMEOUT_GRID = 4 };
+enum : int { DEV_OK = 0, DEV_TIMEOUT_FULL = 1, DEV_TIMEOUT_EMPTY = 2, DEV_TIMEOUT_TMEM = 3, DEV_TIMEOUT_GRID = 4,
+             DEV_BOUNDS = 64 };   // DEV_BOUNDS + check number: an index check of the debug build failed
+
+// Index checks of the debug build (-DTS_DEBUG_BOUNDS; the memory checker tools are not available everywhere): every
+// index a kernel takes from the step's inputs -- token ids, positions, page ids, leaf counts, parents, unit tables --
+// is compared with its range before it is used; a failed check leaves DEV_BOUNDS + its number in the step's status
+// word and the access is skipped.  The host validates the same inputs before a step is staged, so no check is
+// expected to fail; the release build compiles the checks away.
+enum : int { CHK_TOKEN = 1, CHK_POSITION = 2, CHK_PAGE_APPEND = 3, CHK_PAGE_ATTN = 4, CHK_LEAVES = 5, CHK_PARENT = 6,
+             CHK_PAGE_COMPACT = 7, CHK_UNIT = 8 };
+struct BoundsCheck {
+  int *err;                        // the step's status word (null: no checks)
+  int vocab, max_pages, max_ctx;   // ranges of token ids, page ids and positions
+};
+#ifdef TS_DEBUG_BOUNDS
+__device__ __forceinline__ bool ts_in_range(const BoundsCheck &bc, int check, long long v, long long lim) {
+  if (bc.err == nullptr || (v >= 0 && v < lim)) return true;
+  atomicCAS(bc.err, 0, DEV_BOUNDS + check);
+  return false;
+}
+#else
+__device__ __forceinline__ bool ts_in_range(const BoundsCheck &, int, long long, long long) { return true; }
+#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));

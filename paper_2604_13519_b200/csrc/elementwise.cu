@@ -32,7 +32,7 @@ template <int MODE>
 __global__ void __launch_bounds__(kNormMaxThreads)
 norm_kernel(const int32_t *tokens, const __nv_bfloat16 *embed, const float *part, int n_splits, int part_rows,
             const float *gain, float eps, int d, float *x, __nv_bfloat16 *h, int h_rows, int planes,
-            unsigned long long *amax, unsigned long long *stamp) {
+            unsigned long long *amax, unsigned long long *stamp, BoundsCheck bc) {
   __shared__ float red[32];
   if (threadIdx.x == 0) stamp_min(stamp);
   pdl_launch_dependents();   // the dependent kernel waits for this one's end before touching its data
@@ -50,7 +50,8 @@ norm_kernel(const int32_t *tokens, const __nv_bfloat16 *embed, const float *part
   for (int c = c0; c < d; c += blockDim.x * 4) {
     float4 v;
     if (MODE == 0) {
-      const __nv_bfloat16 *e = embed + (size_t)tokens[m] * d + c;
+      const int tok = tokens[m];
+      const __nv_bfloat16 *e = embed + (size_t)(ts_in_range(bc, CHK_TOKEN, tok, bc.vocab) ? tok : 0) * d + c;
       const uint2 raw = *reinterpret_cast<const uint2 *>(e);
       const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162 *>(&raw.x);
       const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162 *>(&raw.y);
@@ -119,7 +120,7 @@ cudaError_t launch_embed_norm(const StepIn &in, const __nv_bfloat16 *embed, cons
                               int d, float *x, __nv_bfloat16 *h, int h_rows, int planes,
                               unsigned long long *amax, cudaStream_t st) {
   return launch_pdl(norm_kernel<0>, dim3(in.M), dim3(norm_threads(d)), 0, st, in.tokens, embed,
-                    (const float *)nullptr, 0, 0, gain, eps, d, x, h, h_rows, planes, amax, (unsigned long long *)nullptr);
+                    (const float *)nullptr, 0, 0, gain, eps, d, x, h, h_rows, planes, amax, (unsigned long long *)nullptr, in.ck);
 }
 
 cudaError_t launch_add_norm(int M, int d, const float *part, int n_splits, int part_rows, const float *gain,
@@ -128,7 +129,7 @@ cudaError_t launch_add_norm(int M, int d, const float *part, int n_splits, int p
   if (n_splits > kNormMaxSplits) return cudaErrorInvalidValue;
   return launch_pdl(norm_kernel<1>, dim3(M), dim3(norm_threads(d)), 0, st, (const int32_t *)nullptr,
                     (const __nv_bfloat16 *)nullptr, part, n_splits, part_rows, gain, eps, d, x, h, h_rows,
-                    planes, (unsigned long long *)nullptr, stamp);
+                    planes, (unsigned long long *)nullptr, stamp, BoundsCheck{});
 }
 
 __device__ __forceinline__ __half to_half_sat(float x) {
@@ -150,8 +151,10 @@ __global__ void rope_kv_kernel(StepIn in, const float *part, int n_splits, int p
   // the step's integer inputs were copied in before the step's first kernel: they may be read before the wait
   const int pos = in.pos[m], seq = in.row_seq[m], slot = in.slot[m];
   const int page = (head >= Hq) ? in.block_tab[(size_t)seq * in.pages_per_seq + (slot >> 4)] : 0;
+  const bool pos_ok = ts_in_range(in.ck, CHK_POSITION, pos, in.ck.max_ctx);
+  const bool page_ok = ts_in_range(in.ck, CHK_PAGE_APPEND, page, in.ck.max_pages);
   float2 cs = make_float2(1.f, 0.f);
-  if (head < Hq + Hkv) cs = rope_tab[(size_t)pos * half + i];
+  if (head < Hq + Hkv && pos_ok) cs = rope_tab[(size_t)pos * half + i];
   pdl_wait();
   if (threadIdx.x == 0) stamp_waited(stamp);
   // the QKV weight rows are stored with rotary partners adjacent: feature 2i = element i, 2i+1 = element i + hd/2
@@ -180,7 +183,7 @@ __global__ void rope_kv_kernel(StepIn in, const float *part, int n_splits, int p
       q_lo_out[qo + i] = __float2half_rn(fabsf(a) <= 65504.f ? a - __half2float(ha) : 0.f);
       q_lo_out[qo + i + half] = __float2half_rn(fabsf(b) <= 65504.f ? b - __half2float(hb) : 0.f);
     }
-  } else {
+  } else if (page_ok) {
     const bool is_k = head < Hq + Hkv;
     const int kh = is_k ? head - Hq : head - Hq - Hkv;
     __half *dst = (is_k ? k_pages : v_pages) + (((size_t)page * Hkv + kh) * 16 + (slot & 15)) * hd;
@@ -205,8 +208,10 @@ __global__ void rope_kv_wide_kernel(StepIn in, const float *part, int n_splits, 
   // the step's integer inputs were copied in before the step's first kernel: they may be read before the wait
   const int pos = in.pos[m], seq = in.row_seq[m], slot = in.slot[m];
   const int page = (live && head >= Hq) ? in.block_tab[(size_t)seq * in.pages_per_seq + (slot >> 4)] : 0;
+  const bool pos_ok = ts_in_range(in.ck, CHK_POSITION, pos, in.ck.max_ctx);
+  const bool page_ok = ts_in_range(in.ck, CHK_PAGE_APPEND, page, in.ck.max_pages);
   float2 cs[4] = {make_float2(1.f, 0.f), make_float2(1.f, 0.f), make_float2(1.f, 0.f), make_float2(1.f, 0.f)};
-  if (live && head < Hq + Hkv) {
+  if (live && head < Hq + Hkv && pos_ok) {
     const float4 *t = reinterpret_cast<const float4 *>(rope_tab + (size_t)pos * half + i0);
     const float4 t0 = t[0], t1 = t[1];
     cs[0] = make_float2(t0.x, t0.y); cs[1] = make_float2(t0.z, t0.w);
@@ -258,7 +263,7 @@ __global__ void rope_kv_wide_kernel(StepIn in, const float *part, int n_splits, 
         *reinterpret_cast<uint2 *>(q_lo_out + qo) = *reinterpret_cast<const uint2 *>(la);
         *reinterpret_cast<uint2 *>(q_lo_out + qo + half) = *reinterpret_cast<const uint2 *>(lb);
       }
-    } else {
+    } else if (page_ok) {
       const bool is_k = head < Hq + Hkv;
       const int kh = is_k ? head - Hq : head - Hq - Hkv;
       __half *dst = (is_k ? k_pages : v_pages) + (((size_t)page * Hkv + kh) * 16 + (slot & 15)) * hd + i0;
@@ -317,8 +322,11 @@ accept_kernel(AcceptArgs a) {
   pdl_wait();
   const int seq = blockIdx.x;
   const int r0 = a.in.cu_rows[seq], r1 = a.in.cu_rows[seq + 1];
-  for (int r = r0 + threadIdx.x; r < r1; r += blockDim.x)
+  for (int r = r0 + threadIdx.x; r < r1; r += blockDim.x) {
     a.argmax[r] = (int32_t)(0xFFFFFFFFu - (uint32_t)(a.amax[r] & 0xFFFFFFFFull));
+    // (a row's parent precedes it in its chunk; -1 marks the root)
+    ts_in_range(a.in.ck, CHK_PARENT, (long long)a.in.parent[r] + 1, r - r0 + 1);
+  }
   __syncthreads();
   if (threadIdx.x == 0) {
     const int k = r1 - r0;
@@ -356,8 +364,12 @@ __global__ void kv_compact_kernel(CompactArgs a) {
   for (int j = 1; j <= l; ++j) {
     const int src = len + path[j], dst = len + j;
     if (src == dst) continue;
-    const size_t so = (((size_t)btab[src >> 4] * a.Hkv + kh) * 16 + (src & 15)) * a.hd + i;
-    const size_t dof = (((size_t)btab[dst >> 4] * a.Hkv + kh) * 16 + (dst & 15)) * a.hd + i;
+    const int ps = btab[src >> 4], pd = btab[dst >> 4];
+    if (!ts_in_range(a.in.ck, CHK_PAGE_COMPACT, ps, a.in.ck.max_pages) ||
+        !ts_in_range(a.in.ck, CHK_PAGE_COMPACT, pd, a.in.ck.max_pages))
+      continue;
+    const size_t so = (((size_t)ps * a.Hkv + kh) * 16 + (src & 15)) * a.hd + i;
+    const size_t dof = (((size_t)pd * a.Hkv + kh) * 16 + (dst & 15)) * a.hd + i;
     kp[dof] = kp[so];
     kp[a.v_offset + dof] = kp[a.v_offset + so];
   }

@@ -71,6 +71,7 @@ struct StepIn {
   const int32_t *row_leaves; // [M] attention leaves of the row's sequence: ceil((cached length + chunk rows) / leaf length)
   int pages_per_seq;
   int B, M;
+  BoundsCheck ck;            // ranges for the debug build's index checks
 };
 
 // x[m] = E[tokens[m]]; h = rmsnorm(x) * gain -> bf16 (hi[, lo])

@@ -435,6 +435,7 @@ ts_status run_step(ts_model *m) {
   in.parent = di + L.o_parent; in.anc = (const uint32_t *)(di + L.o_anc); in.slot = di + L.o_slot;
   in.row_leaves = di + L.o_row_leaves;
   in.B = B; in.M = M;
+  in.ck.err = m->d_out() + L.o_err; in.ck.vocab = c.vocab; in.ck.max_pages = c.max_pages; in.ck.max_ctx = c.max_ctx;
   float *x = (float *)m->WS(L.x);
   __nv_bfloat16 *h = (__nv_bfloat16 *)m->WS(L.h);
   float *part = (float *)m->WS(L.part);
@@ -712,6 +713,8 @@ ts_status stage_and_run(ts_model *m, ts_session *const *ss, int B, const std::ve
   if (dev_err != 0) {
     cudaMemsetAsync(m->d_out() + L.o_err, 0, 4, m->st);
     cudaMemsetAsync(m->WS(L.sync), 0, (size_t)(8 + L.n_counters) * 4, m->st);   // the fused kernel left its counters mid-step
+    if (dev_err >= ts::DEV_BOUNDS)
+      return fail(TS_ERR_DEVICE_BOUNDS, "an index check of the debug build failed on the device (check %d)", dev_err - ts::DEV_BOUNDS);
     return fail(TS_ERR_DEVICE_TIMEOUT, "a bounded device-side wait expired (code %d)", dev_err);
   }
   return TS_OK;

@@ -315,6 +315,24 @@ def test_device_timeout_is_reported_and_survived(path):
     gm.close()
 
 
+def test_device_index_check_is_reported_and_survived():
+    """The host's handling of a failed index check of the debug build, exercised the same way (a status word written
+    after the step's last kernel; the release build's kernels contain no checks): TS_ERR_DEVICE_BOUNDS with the check's
+    number, session untouched, next step clean."""
+    shape = synth.SHAPES["1b-2l"]
+    om, gm = make_pair(shape, k_max=16, max_ctx=512)
+    cache, s, pending = synthetic_context(shape, om, gm, 200)
+    draft = _rand_draft(shape.vocab, 9, 31)
+    ref = om.verify(pending, draft, cache.clone(), want_logits=True)
+    gm.inject_device_error(64 + 4)
+    with pytest.raises(ts.TsError) as e:
+        ts.ts_verify(gm, [s], [draft])
+    assert e.value.code == -9 and "check 4" in str(e.value)
+    assert (s.state().cache_len, s.state().pending) == (200, pending)
+    check_step(ts.ts_verify(gm, [s], [draft])[0], gm.read_logits(0, 10), ref, "after the reported index check")
+    gm.close()
+
+
 def test_small_batch_fused():
     """Several short sequences in one step of the persistent kernel (ragged k, ragged contexts)."""
     shape = synth.SHAPES["1b-2l"]

@@ -31,6 +31,20 @@ def test_exports_every_declared_symbol():
     assert declared == set(B.EXPORTED)
 
 
+def test_debug_library_builds_and_exports_the_same_symbols():
+    """The debug build (every index a kernel takes from the step's inputs checked on the device) is the same library
+    compiled with TS_DEBUG_BOUNDS: it must build and export every declared entry point."""
+    from paper_2604_13519_b200 import build
+    path = build.build(debug_bounds=True)
+    assert path == B.DEBUG_LIB_PATH and os.path.exists(path)
+    L = C.CDLL(path)
+    for name in B.EXPORTED:
+        assert hasattr(L, name), name
+    assert B.STATUS[-9] == "TS_ERR_DEVICE_BOUNDS"
+    hdr = open(os.path.join(ROOT, "include", "toolspec.h")).read()
+    assert re.search(r"TS_ERR_DEVICE_BOUNDS\s*=\s*-9", hdr)
+
+
 def test_buffer_sizes_and_argument_errors():
     c = B.ts_model_config()
     s = synth.SHAPES["8b"]
