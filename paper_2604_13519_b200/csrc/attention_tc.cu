@@ -372,7 +372,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
 
   if (warp == 0) {
     // ---------------------------------------------------------------- K/V producer
-    if (lane == 0) {
+    // (the whole warp walks the loops and the waits; an elected lane issues a block's sixteen copies -- a lone lane
+    // in a divergent branch needs about 50 cycles per copy instruction, more than half of a block's time)
+    {
       const uint64_t pol = policy_evict_first();
       uint32_t gb = 0;
       bool waited = false, ok = true;
@@ -387,22 +389,37 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
           if (!waited && (gb >= (uint32_t)kKvStages || t.pos_beg + (b + 1) * kAttnBlk > t.len)) { pdl_wait(); waited = true; }
           const uint32_t st = gb % kKvStages;
           if (gb >= (uint32_t)kKvStages &&
-              !mbar_wait_err(smem_u32(&ctl->kv_empty[st]), ((gb / kKvStages) & 1) ^ 1, err)) { atomicCAS(a.err, 0, DEV_TIMEOUT_EMPTY); ok = false; break; }
+              !__all_sync(0xffffffffu, mbar_wait_err(smem_u32(&ctl->kv_empty[st]), ((gb / kKvStages) & 1) ^ 1, err))) {
+            if (lane == 0) atomicCAS(a.err, 0, DEV_TIMEOUT_EMPTY);
+            ok = false;
+            break;
+          }
           const uint32_t bar = smem_u32(&ctl->kv_full[st]);
-          mbar_expect_tx(bar, kKvBytes);
           uint8_t *sK = smem + st * kKvBytes, *sV = sK + kAttnBlk * HD * 2;
-          for (int pg = 0; pg < kAttnBlk / 16; ++pg) {
-            // a page past the unit's end is never visible; load the last visible page again instead
-            const int pos = min(t.pos_beg + b * kAttnBlk + pg * 16, t.pos_end - 1);
-            int page = btab[pos >> 4];
+          // lane pg looks its page up (a page past the unit's end is never visible: the last visible page is loaded
+          // again instead); the elected lane gets the four ids by shuffle
+          int page = 0;
+          if (lane < kAttnBlk / 16) {
+            const int pos = min(t.pos_beg + b * kAttnBlk + lane * 16, t.pos_end - 1);
+            page = btab[pos >> 4];
             if (!ts_in_range(a.in.ck, CHK_PAGE_ATTN, page, a.in.ck.max_pages)) page = 0;
+          }
+          int pages[kAttnBlk / 16];
 #pragma unroll
-            for (int hh = 0; hh < (int)kHalves; ++hh) {
-              const uint32_t off = hh * (kAttnBlk * 128) + pg * 2048;
-              tma_load_5d(smem_u32(sK + off), a.map_kv, hh * 64, 0, t.kh, page, 2 * a.layer, bar, pol);
-              tma_load_5d(smem_u32(sV + off), a.map_kv, hh * 64, 0, t.kh, page, 2 * a.layer + 1, bar, pol);
+          for (int pg = 0; pg < kAttnBlk / 16; ++pg) pages[pg] = __shfl_sync(0xffffffffu, page, pg);
+          if (elect_one()) {
+            mbar_expect_tx(bar, kKvBytes);
+#pragma unroll
+            for (int pg = 0; pg < kAttnBlk / 16; ++pg) {
+#pragma unroll
+              for (int hh = 0; hh < (int)kHalves; ++hh) {
+                const uint32_t off = hh * (kAttnBlk * 128) + pg * 2048;
+                tma_load_5d(smem_u32(sK + off), a.map_kv, hh * 64, 0, t.kh, pages[pg], 2 * a.layer, bar, pol);
+                tma_load_5d(smem_u32(sV + off), a.map_kv, hh * 64, 0, t.kh, pages[pg], 2 * a.layer + 1, bar, pol);
+              }
             }
           }
+          __syncwarp();
         }
       }
     }
